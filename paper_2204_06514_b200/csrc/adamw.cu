@@ -1,0 +1,142 @@
+// Multi-tensor AdamW over float32 master weights (step U).  HBM-bound: 128-bit
+// loads and stores, one pass, writes the bf16 compute copy in the same pass.
+// Algorithmic traffic per element: read w, m, v, g (16 B) + write w, m, v
+// (12 B) + write bf16 copy (2 B) = 30 B.
+#include "common.cuh"
+
+namespace {
+
+constexpr int MAX_T = 40;              // tensors per launch (kernel-parameter space)
+constexpr int CHUNK = 4096;            // elements per block iteration
+constexpr int THREADS = 256;
+
+struct AdamTensor {
+  float* w; float* m; float* v; const void* g; bf16* wc;
+  unsigned long long n;
+  float wd;
+  unsigned int first_chunk;            // prefix sum of chunk counts
+};
+struct AdamBatch {
+  AdamTensor t[MAX_T];
+  int n_tensors;
+  unsigned int total_chunks;
+};
+
+struct AdamScalars { float lr, b1, b2, eps, inv_bc1, inv_bc2; };
+
+template <bool G_BF16>
+__device__ __forceinline__ void adam_elem(float& w, float& m, float& v, float g, float wd,
+                                          const AdamScalars& s) {
+  m = s.b1 * m + (1.f - s.b1) * g;
+  v = s.b2 * v + (1.f - s.b2) * g * g;
+  float mh = m * s.inv_bc1;
+  float vh = v * s.inv_bc2;
+  w = w - s.lr * wd * w - s.lr * mh / (sqrtf(vh) + s.eps);
+}
+
+template <bool G_BF16>
+__global__ void __launch_bounds__(THREADS)
+adamw_kernel(const __grid_constant__ AdamBatch batch, AdamScalars sc) {
+  for (unsigned int chunk = blockIdx.x; chunk < batch.total_chunks; chunk += gridDim.x) {
+    // find the tensor this chunk belongs to (few tensors: linear scan from a binary start)
+    int lo = 0, hi = batch.n_tensors - 1;
+    while (lo < hi) {
+      int mid = (lo + hi + 1) >> 1;
+      if (batch.t[mid].first_chunk <= chunk) lo = mid; else hi = mid - 1;
+    }
+    const AdamTensor& t = batch.t[lo];
+    unsigned long long base = (unsigned long long)(chunk - t.first_chunk) * CHUNK;
+    unsigned long long end = base + CHUNK < t.n ? base + CHUNK : t.n;
+    const bool vec_ok = ((t.n & 3ull) == 0);
+    if (vec_ok) {
+      for (unsigned long long e = base + 4ull * threadIdx.x; e < end; e += 4ull * THREADS) {
+        float4 w = *reinterpret_cast<const float4*>(t.w + e);
+        float4 m = *reinterpret_cast<const float4*>(t.m + e);
+        float4 v = *reinterpret_cast<const float4*>(t.v + e);
+        float4 g;
+        if (G_BF16) {
+          uint2 raw = *reinterpret_cast<const uint2*>((const bf16*)t.g + e);
+          float2 a = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&raw.x));
+          float2 b = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&raw.y));
+          g = make_float4(a.x, a.y, b.x, b.y);
+        } else {
+          g = *reinterpret_cast<const float4*>((const float*)t.g + e);
+        }
+        adam_elem<G_BF16>(w.x, m.x, v.x, g.x, t.wd, sc);
+        adam_elem<G_BF16>(w.y, m.y, v.y, g.y, t.wd, sc);
+        adam_elem<G_BF16>(w.z, m.z, v.z, g.z, t.wd, sc);
+        adam_elem<G_BF16>(w.w, m.w, v.w, g.w, t.wd, sc);
+        *reinterpret_cast<float4*>(t.w + e) = w;
+        *reinterpret_cast<float4*>(t.m + e) = m;
+        *reinterpret_cast<float4*>(t.v + e) = v;
+        if (t.wc) {
+          uint2 o;
+          *reinterpret_cast<__nv_bfloat162*>(&o.x) = __floats2bfloat162_rn(w.x, w.y);
+          *reinterpret_cast<__nv_bfloat162*>(&o.y) = __floats2bfloat162_rn(w.z, w.w);
+          *reinterpret_cast<uint2*>(t.wc + e) = o;
+        }
+      }
+    } else {
+      for (unsigned long long e = base + threadIdx.x; e < end; e += THREADS) {
+        float w = t.w[e], m = t.m[e], v = t.v[e];
+        float g = G_BF16 ? __bfloat162float(((const bf16*)t.g)[e]) : ((const float*)t.g)[e];
+        adam_elem<G_BF16>(w, m, v, g, t.wd, sc);
+        t.w[e] = w; t.m[e] = m; t.v[e] = v;
+        if (t.wc) t.wc[e] = __float2bfloat16_rn(w);
+      }
+    }
+  }
+}
+
+}  // namespace
+
+fax_status fax_adamw_launch(fax_ctx* ctx, const fax_adamw_tensor* tensors, int n, const fax_adamw_hparams* hp) {
+  if (!tensors || !hp || n < 0) return FAX_ERR_INVALID_ARG;
+  if (hp->step < 1 || !(hp->beta1 >= 0.f && hp->beta1 < 1.f) || !(hp->beta2 >= 0.f && hp->beta2 < 1.f))
+    return FAX_ERR_INVALID_ARG;
+  AdamScalars sc;
+  sc.lr = hp->lr; sc.b1 = hp->beta1; sc.b2 = hp->beta2; sc.eps = hp->eps;
+  sc.inv_bc1 = (float)(1.0 / (1.0 - pow((double)hp->beta1, (double)hp->step)));
+  sc.inv_bc2 = (float)(1.0 / (1.0 - pow((double)hp->beta2, (double)hp->step)));
+  for (int i = 0; i < n; ++i) {
+    const fax_adamw_tensor& t = tensors[i];
+    if (!t.w || !t.m || !t.v || !t.g) return FAX_ERR_INVALID_ARG;
+    if (!fax_aligned(t.w, 16) || !fax_aligned(t.m, 16) || !fax_aligned(t.v, 16) || !fax_aligned(t.g, 16) ||
+        (t.w_compute && !fax_aligned(t.w_compute, 8)))
+      return FAX_ERR_INVALID_ARG;
+  }
+  int i = 0;
+  while (i < n) {
+    AdamBatch batch;
+    int k = 0;
+    unsigned long long chunks = 0;
+    while (i < n && k < MAX_T) {
+      const fax_adamw_tensor& t = tensors[i++];
+      if (t.n == 0) continue;
+      unsigned long long c = (t.n + CHUNK - 1) / CHUNK;
+      if (chunks + c > 0xffffffffull) { --i; break; }
+      batch.t[k].w = t.w; batch.t[k].m = t.m; batch.t[k].v = t.v; batch.t[k].g = t.g;
+      batch.t[k].wc = (bf16*)t.w_compute; batch.t[k].n = t.n; batch.t[k].wd = t.weight_decay;
+      batch.t[k].first_chunk = (unsigned int)chunks;
+      chunks += c;
+      ++k;
+    }
+    if (k == 0) { if (i < n && chunks == 0 && tensors[i].n > 0) return FAX_ERR_UNSUPPORTED_SHAPE; continue; }
+    batch.n_tensors = k;
+    batch.total_chunks = (unsigned int)chunks;
+    unsigned long long want = chunks;
+    unsigned int grid = (unsigned int)(want < (unsigned long long)ctx->sm_count * 16 ? want : ctx->sm_count * 16);
+    if (hp->grad_is_bf16)
+      adamw_kernel<true><<<grid, THREADS, 0, ctx->stream>>>(batch, sc);
+    else
+      adamw_kernel<false><<<grid, THREADS, 0, ctx->stream>>>(batch, sc);
+    FAX_TRY(fax_after_launch(ctx));
+  }
+  return FAX_OK;
+}
+
+extern "C" fax_status fax_adamw_step(fax_ctx* ctx, const fax_adamw_tensor* tensors, int32_t n_tensors,
+                                     const fax_adamw_hparams* hp) {
+  if (!ctx) return FAX_ERR_INVALID_ARG;
+  return fax_adamw_launch(ctx, tensors, n_tensors, hp);
+}

@@ -1,0 +1,79 @@
+// Context lifetime, status strings and the device status word.
+#include "common.cuh"
+
+extern "C" const char* fax_status_string(fax_status s) {
+  switch (s) {
+    case FAX_OK: return "FAX_OK";
+    case FAX_ERR_INVALID_ARG: return "FAX_ERR_INVALID_ARG";
+    case FAX_ERR_UNSUPPORTED_SHAPE: return "FAX_ERR_UNSUPPORTED_SHAPE";
+    case FAX_ERR_WORKSPACE_TOO_SMALL: return "FAX_ERR_WORKSPACE_TOO_SMALL";
+    case FAX_ERR_CUDA: return "FAX_ERR_CUDA";
+    case FAX_ERR_ARCH: return "FAX_ERR_ARCH";
+    case FAX_ERR_TIMEOUT: return "FAX_ERR_TIMEOUT";
+    default: return "FAX_ERR_UNKNOWN";
+  }
+}
+
+extern "C" fax_status fax_create(fax_ctx** out, int32_t device_ordinal, void* cuda_stream) {
+  if (!out) return FAX_ERR_INVALID_ARG;
+  *out = nullptr;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess || device_ordinal < 0 || device_ordinal >= count) {
+    (void)cudaGetLastError();
+    return FAX_ERR_CUDA;
+  }
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device_ordinal) != cudaSuccess) return FAX_ERR_CUDA;
+  if (prop.major != 10) return FAX_ERR_ARCH;
+  if (cudaSetDevice(device_ordinal) != cudaSuccess) return FAX_ERR_CUDA;
+  fax_ctx* c = new fax_ctx();
+  c->device = device_ordinal;
+  c->stream = (cudaStream_t)cuda_stream;
+  c->last_cuda_error = 0;
+  c->launches = 0;
+  c->sm_count = prop.multiProcessorCount;
+  c->dev_status = nullptr;
+  c->encode_tiled = nullptr;
+  if (cudaMalloc((void**)&c->dev_status, 64) != cudaSuccess ||
+      cudaMemset(c->dev_status, 0, 64) != cudaSuccess) {
+    delete c;
+    return FAX_ERR_CUDA;
+  }
+  cudaDriverEntryPointQueryResult qres;
+  void* fn = nullptr;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess || fn == nullptr) {
+    (void)cudaGetLastError();
+    cudaFree(c->dev_status);
+    delete c;
+    return FAX_ERR_CUDA;
+  }
+  c->encode_tiled = fn;
+  *out = c;
+  return FAX_OK;
+}
+
+extern "C" fax_status fax_destroy(fax_ctx* ctx) {
+  if (!ctx) return FAX_ERR_INVALID_ARG;
+  cudaSetDevice(ctx->device);
+  cudaStreamSynchronize(ctx->stream);
+  if (ctx->dev_status) cudaFree(ctx->dev_status);
+  delete ctx;
+  return FAX_OK;
+}
+
+extern "C" int32_t fax_last_cuda_error(const fax_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
+extern "C" uint64_t fax_launch_count(const fax_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+extern "C" fax_status fax_check_device_status(fax_ctx* ctx, int32_t* detail_host) {
+  if (!ctx) return FAX_ERR_INVALID_ARG;
+  int32_t h[2] = {0, 0};
+  FAX_CUDA_TRY(ctx, cudaStreamSynchronize(ctx->stream));
+  FAX_CUDA_TRY(ctx, cudaMemcpy(h, ctx->dev_status, sizeof(h), cudaMemcpyDeviceToHost));
+  if (detail_host) *detail_host = h[1];
+  if (h[0] != 0) {
+    FAX_CUDA_TRY(ctx, cudaMemset(ctx->dev_status, 0, 8));
+    return FAX_ERR_TIMEOUT;
+  }
+  return FAX_OK;
+}

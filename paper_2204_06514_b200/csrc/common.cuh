@@ -1,0 +1,160 @@
+// Shared host/device helpers of the CUDA library: context, status handling,
+// launch bookkeeping and small numeric utilities.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "../../include/fax.h"
+
+typedef __nv_bfloat16 bf16;
+
+// Device status block owned by the context: word 0 = error flag, word 1 = detail.
+struct fax_ctx {
+  int device;
+  cudaStream_t stream;
+  int32_t* dev_status;       // 2 x int32 on the device
+  int32_t last_cuda_error;
+  uint64_t launches;
+  int sm_count;
+  void* encode_tiled;        // cuTensorMapEncodeTiled, resolved at create
+};
+
+#define FAX_CUDA_TRY(ctx, expr)                                   \
+  do {                                                            \
+    cudaError_t e__ = (expr);                                     \
+    if (e__ != cudaSuccess) {                                     \
+      (ctx)->last_cuda_error = (int32_t)e__;                      \
+      return FAX_ERR_CUDA;                                        \
+    }                                                             \
+  } while (0)
+
+#define FAX_TRY(expr)                                             \
+  do {                                                            \
+    fax_status s__ = (expr);                                      \
+    if (s__ != FAX_OK) return s__;                                \
+  } while (0)
+
+// Count a launch and pick up a launch-configuration error without syncing.
+static inline fax_status fax_after_launch(fax_ctx* ctx) {
+  ctx->launches++;
+  cudaError_t e = cudaPeekAtLastError();
+  if (e != cudaSuccess) {
+    ctx->last_cuda_error = (int32_t)e;
+    (void)cudaGetLastError();
+    return FAX_ERR_CUDA;
+  }
+  return FAX_OK;
+}
+
+static inline bool fax_aligned(const void* p, size_t a) { return ((uintptr_t)p & (a - 1)) == 0; }
+static inline size_t fax_round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+static inline size_t fax_elem_size(int prec) { return prec == FAX_PREC_BF16 ? 2 : 4; }
+
+// Bump allocator over a caller-provided arena (256-byte aligned pieces).
+struct FaxArena {
+  char* base; size_t off; size_t cap;
+  FaxArena(void* b, size_t c) : base((char*)b), off(0), cap(c) {}
+  void* take(size_t bytes) {
+    size_t o = fax_round_up(off, 256);
+    off = o + bytes;
+    return base ? (void*)(base + o) : (void*)0;
+  }
+  size_t used() const { return fax_round_up(off, 256); }
+};
+
+// ---- device numeric helpers -------------------------------------------------
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(bf16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ bf16 from_f32<bf16>(float v) { return __float2bfloat16_rn(v); }
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// tanh-form GELU and its derivative, float32.
+__device__ __forceinline__ float gelu_tanh_f(float h) {
+  const float c = 0.7978845608028654f, a = 0.044715f;
+  float t = tanhf(c * (h + a * h * h * h));
+  return 0.5f * h * (1.0f + t);
+}
+__device__ __forceinline__ float gelu_tanh_grad_f(float h) {
+  const float c = 0.7978845608028654f, a = 0.044715f;
+  float t = tanhf(c * (h + a * h * h * h));
+  return 0.5f * (1.0f + t) + 0.5f * h * (1.0f - t * t) * c * (1.0f + 3.0f * a * h * h);
+}
+
+// ---- internal operator interfaces (host functions that enqueue kernels) ------
+enum FaxEpilogue {
+  EPI_NONE = 0,        // C = acc
+  EPI_BIAS = 1,        // C = acc + bias[n]
+  EPI_BIAS_GELU = 2,   // C = acc + bias (pre-activation), aux = GELU(C)
+  EPI_BIAS_RESID = 3,  // C = acc + bias + resid
+  EPI_DGELU = 4        // C = acc * GELU'(aux)          (aux read-only, [M,N])
+};
+
+struct FaxGemm {
+  int M, N, K;
+  const void* A; int64_t lda; bool a_mn_major;  // false: A is [M,K] row-major; true: A is [K,M] row-major
+  const void* B; int64_t ldb; bool b_mn_major;  // false: B is [N,K] row-major; true: B is [K,N] row-major
+  void* C; int64_t ldc; bool c_f32;             // C is [M,N] row-major, type T or float
+  bool accumulate;                              // C += result (float output only)
+  int epi;
+  const void* bias;                             // [N] type T
+  const void* resid; int64_t ldr;               // [M,N] type T
+  void* aux; int64_t ldaux;                     // [M,N] type T
+  float alpha;                                  // scales acc before the epilogue
+};
+
+fax_status fax_gemm_simt(fax_ctx* ctx, int prec, const FaxGemm& g);
+fax_status fax_gemm_tc(fax_ctx* ctx, const FaxGemm& g);       // bf16 tcgen05 path
+bool fax_gemm_tc_supported(const FaxGemm& g);
+fax_status fax_gemm(fax_ctx* ctx, int prec, const FaxGemm& g); // dispatch
+
+fax_status fax_layernorm_fwd(fax_ctx* ctx, int prec, int rows, int d, const void* x, const void* gamma,
+                             const void* beta, float eps, void* out, float* mu, float* rstd, void* x_copy);
+// dx = (add ? add : 0) + LNbwd(da); partial: float scratch [2 * slabs * d]
+fax_status fax_layernorm_bwd(fax_ctx* ctx, int prec, int rows, int d, const void* da, const void* x,
+                             const float* mu, const float* rstd, const void* gamma, const void* add,
+                             void* dx, float* dgamma, float* dbeta, bool accumulate, float* partial,
+                             size_t partial_floats);
+size_t fax_layernorm_bwd_partial_floats(int rows, int d);
+
+// out[c] (+)= sum_r in[r, c]
+fax_status fax_colsum(fax_ctx* ctx, int prec, int rows, int cols, const void* in, int64_t ld, float* out,
+                      bool accumulate, float* partial, size_t partial_floats);
+size_t fax_colsum_partial_floats(int rows, int cols);
+
+fax_status fax_attention_fwd(fax_ctx* ctx, int prec, int B, int T, int H, int hd, const void* qkv,
+                             void* o, float* lse);
+fax_status fax_attention_bwd(fax_ctx* ctx, int prec, int B, int T, int H, int hd, const void* qkv,
+                             const void* o, const float* lse, const void* d_o, void* dqkv,
+                             void* scratch, size_t scratch_bytes);
+size_t fax_attention_bwd_scratch_bytes(int prec, int B, int T, int H, int hd);
+
+fax_status fax_adamw_launch(fax_ctx* ctx, const fax_adamw_tensor* tensors, int n, const fax_adamw_hparams* hp);
+
+fax_status fax_block_validate(const fax_block_cfg* cfg);
+
+fax_status fax_attention_fwd_simt(fax_ctx* ctx, int prec, int B, int T, int H, int hd, const void* qkv,
+                                  void* o, float* lse);
+fax_status fax_attention_bwd_simt(fax_ctx* ctx, int prec, int B, int T, int H, int hd, const void* qkv,
+                                  const void* o, const float* lse, const void* d_o, void* dqkv, float* Dv);
+fax_status fax_embed_fwd(fax_ctx* ctx, int prec, int B, int T, int d, int vocab, const int32_t* ids,
+                         const void* wte, const void* wpe, void* x0);
+fax_status fax_embed_bwd(fax_ctx* ctx, int prec, int B, int T, int max_seq, int d, int vocab,
+                         const int32_t* ids, const void* dx0, float* dwte, float* dwpe);
+fax_status fax_xent(fax_ctx* ctx, int prec, int rows, int vocab, void* logits, int64_t ld,
+                    const int32_t* targets, float inv_n, float* row_loss);
+fax_status fax_loss_mean(fax_ctx* ctx, int n, const float* row_loss, float* loss);

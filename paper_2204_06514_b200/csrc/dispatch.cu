@@ -1,0 +1,24 @@
+// Operator dispatch between the tensor-core kernels and the SIMT kernels.
+#include "common.cuh"
+
+fax_status fax_gemm(fax_ctx* ctx, int prec, const FaxGemm& g) {
+  if (prec == FAX_PREC_BF16 && fax_gemm_tc_supported(g)) return fax_gemm_tc(ctx, g);
+  return fax_gemm_simt(ctx, prec, g);
+}
+
+size_t fax_attention_bwd_scratch_bytes(int prec, int B, int T, int H, int hd) {
+  (void)prec; (void)hd;
+  return (size_t)B * H * T * sizeof(float);      // D = rowsum(dO * O)
+}
+
+fax_status fax_attention_fwd(fax_ctx* ctx, int prec, int B, int T, int H, int hd, const void* qkv,
+                             void* o, float* lse) {
+  return fax_attention_fwd_simt(ctx, prec, B, T, H, hd, qkv, o, lse);
+}
+
+fax_status fax_attention_bwd(fax_ctx* ctx, int prec, int B, int T, int H, int hd, const void* qkv,
+                             const void* o, const float* lse, const void* d_o, void* dqkv,
+                             void* scratch, size_t scratch_bytes) {
+  if (scratch_bytes < (size_t)B * H * T * sizeof(float)) return FAX_ERR_WORKSPACE_TOO_SMALL;
+  return fax_attention_bwd_simt(ctx, prec, B, T, H, hd, qkv, o, lse, d_o, dqkv, (float*)scratch);
+}

@@ -1,0 +1,146 @@
+// Embedding lookup / scatter and softmax cross-entropy of the LM step
+// (steps LM-E, LM-H loss part, LM-B).  All HBM-bound.
+#include "common.cuh"
+
+namespace {
+
+template <typename T>
+__global__ void embed_fwd_kernel(int n_tok, int Tn, int d, int vocab, const int32_t* __restrict__ ids,
+                                 const T* __restrict__ wte, const T* __restrict__ wpe, T* __restrict__ x0) {
+  int n = blockIdx.x;
+  int id = ids[n];
+  id = id < 0 ? 0 : (id >= vocab ? vocab - 1 : id);     // ids are validated upstream; clamp keeps reads in bounds
+  const T* e = wte + (size_t)id * d;
+  const T* p = wpe + (size_t)(n % Tn) * d;
+  for (int c = threadIdx.x; c < d; c += blockDim.x)
+    x0[(size_t)n * d + c] = from_f32<T>(to_f32(e[c]) + to_f32(p[c]));
+}
+
+// dwte[ids[n]] += dx0[n]   (float atomics on top of the head gradient)
+template <typename T>
+__global__ void embed_bwd_wte_kernel(int n_tok, int d, int vocab, const int32_t* __restrict__ ids,
+                                     const T* __restrict__ dx0, float* __restrict__ dwte) {
+  int n = blockIdx.x;
+  int id = ids[n];
+  if (id < 0 || id >= vocab) return;
+  for (int c = threadIdx.x; c < d; c += blockDim.x)
+    atomicAdd(dwte + (size_t)id * d + c, to_f32(dx0[(size_t)n * d + c]));
+}
+
+// dwpe[t] = sum_b dx0[b, t]   (fixed order: deterministic); rows t >= Tn are zeroed
+template <typename T>
+__global__ void embed_bwd_wpe_kernel(int Bn, int Tn, int max_seq, int d, const T* __restrict__ dx0,
+                                     float* __restrict__ dwpe) {
+  int t = blockIdx.x;
+  for (int c = threadIdx.x; c < d; c += blockDim.x) {
+    float s = 0.f;
+    if (t < Tn)
+      for (int b = 0; b < Bn; ++b) s += to_f32(dx0[((size_t)b * Tn + t) * d + c]);
+    dwpe[(size_t)t * d + c] = s;
+  }
+}
+
+__device__ __forceinline__ float block_reduce_max(float v, float* red) {
+  v = warp_max(v);
+  int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+  __syncthreads();
+  if (lane == 0) red[warp] = v;
+  __syncthreads();
+  float t = lane < nw ? red[lane] : -INFINITY;
+  return warp_max(t);
+}
+__device__ __forceinline__ float block_reduce_sum(float v, float* red) {
+  v = warp_sum(v);
+  int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+  __syncthreads();
+  if (lane == 0) red[warp] = v;
+  __syncthreads();
+  float t = lane < nw ? red[lane] : 0.f;
+  return warp_sum(t);
+}
+
+// One block per row of a logits chunk.  In place: logits -> (softmax - onehot) * inv_n.
+// row_loss[row0 + r] = logsumexp - logit[target].
+template <typename T>
+__global__ void __launch_bounds__(512)
+xent_kernel(int rows, int vocab, T* __restrict__ logits, int64_t ld, const int32_t* __restrict__ targets,
+            float inv_n, float* __restrict__ row_loss) {
+  __shared__ float red[32];
+  int r = blockIdx.x;
+  T* row = logits + (size_t)r * ld;
+  float mx = -INFINITY;
+  for (int c = threadIdx.x; c < vocab; c += blockDim.x) mx = fmaxf(mx, to_f32(row[c]));
+  mx = block_reduce_max(mx, red);
+  float s = 0.f;
+  for (int c = threadIdx.x; c < vocab; c += blockDim.x) s += __expf(to_f32(row[c]) - mx);
+  s = block_reduce_sum(s, red);
+  int tg = targets[r];
+  float lse = mx + logf(s);
+  if (threadIdx.x == 0) {
+    float lt = (tg >= 0 && tg < vocab) ? to_f32(row[tg]) : lse;
+    row_loss[r] = lse - lt;
+  }
+  __syncthreads();
+  float inv_s = 1.f / s;
+  for (int c = threadIdx.x; c < vocab; c += blockDim.x) {
+    float p = __expf(to_f32(row[c]) - mx) * inv_s;
+    if (c == tg) p -= 1.f;
+    row[c] = from_f32<T>(p * inv_n);
+  }
+}
+
+__global__ void loss_mean_kernel(int n, const float* __restrict__ row_loss, float* __restrict__ loss) {
+  __shared__ double red[32];
+  double s = 0.0;
+  for (int i = threadIdx.x; i < n; i += blockDim.x) s += (double)row_loss[i];
+  for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+  int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+  if (lane == 0) red[warp] = s;
+  __syncthreads();
+  if (warp == 0) {
+    double t = lane < nw ? red[lane] : 0.0;
+    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+    if (lane == 0) *loss = (float)(t / (double)n);
+  }
+}
+
+}  // namespace
+
+fax_status fax_embed_fwd(fax_ctx* ctx, int prec, int B, int T, int d, int vocab, const int32_t* ids,
+                         const void* wte, const void* wpe, void* x0) {
+  int n = B * T;
+  if (prec == FAX_PREC_BF16)
+    embed_fwd_kernel<bf16><<<n, 128, 0, ctx->stream>>>(n, T, d, vocab, ids, (const bf16*)wte, (const bf16*)wpe, (bf16*)x0);
+  else
+    embed_fwd_kernel<float><<<n, 128, 0, ctx->stream>>>(n, T, d, vocab, ids, (const float*)wte, (const float*)wpe, (float*)x0);
+  return fax_after_launch(ctx);
+}
+
+fax_status fax_embed_bwd(fax_ctx* ctx, int prec, int B, int T, int max_seq, int d, int vocab,
+                         const int32_t* ids, const void* dx0, float* dwte, float* dwpe) {
+  int n = B * T;
+  if (prec == FAX_PREC_BF16) {
+    embed_bwd_wte_kernel<bf16><<<n, 128, 0, ctx->stream>>>(n, d, vocab, ids, (const bf16*)dx0, dwte);
+    FAX_TRY(fax_after_launch(ctx));
+    embed_bwd_wpe_kernel<bf16><<<max_seq, 128, 0, ctx->stream>>>(B, T, max_seq, d, (const bf16*)dx0, dwpe);
+  } else {
+    embed_bwd_wte_kernel<float><<<n, 128, 0, ctx->stream>>>(n, d, vocab, ids, (const float*)dx0, dwte);
+    FAX_TRY(fax_after_launch(ctx));
+    embed_bwd_wpe_kernel<float><<<max_seq, 128, 0, ctx->stream>>>(B, T, max_seq, d, (const float*)dx0, dwpe);
+  }
+  return fax_after_launch(ctx);
+}
+
+fax_status fax_xent(fax_ctx* ctx, int prec, int rows, int vocab, void* logits, int64_t ld,
+                    const int32_t* targets, float inv_n, float* row_loss) {
+  if (prec == FAX_PREC_BF16)
+    xent_kernel<bf16><<<rows, 512, 0, ctx->stream>>>(rows, vocab, (bf16*)logits, ld, targets, inv_n, row_loss);
+  else
+    xent_kernel<float><<<rows, 512, 0, ctx->stream>>>(rows, vocab, (float*)logits, ld, targets, inv_n, row_loss);
+  return fax_after_launch(ctx);
+}
+
+fax_status fax_loss_mean(fax_ctx* ctx, int n, const float* row_loss, float* loss) {
+  loss_mean_kernel<<<1, 1024, 0, ctx->stream>>>(n, row_loss, loss);
+  return fax_after_launch(ctx);
+}

@@ -165,10 +165,12 @@ def lm_tokens(cfg: Config):
 
 
 def warm_state(seed: int, tensor_id: int, shape, scale: float):
-    """Non-zero optimizer state: m ~ N(0, scale^2), v = m^2 + positive noise."""
+    """Non-zero optimizer state: m ~ N(0, scale^2), v = m^2 + positive noise with a
+    floor of (scale/2)^2, so that the update stays Lipschitz in the gradient."""
     m = normal(seed, TID_STATE_M + 1000 * tensor_id, shape, scale)
     n = normal(seed, TID_STATE_V + 1000 * tensor_id, shape, scale)
-    return m, (m.astype(np.float64) ** 2 + n.astype(np.float64) ** 2).astype(np.float32)
+    v = m.astype(np.float64) ** 2 + n.astype(np.float64) ** 2 + (0.5 * scale) ** 2
+    return m, v.astype(np.float32)
 
 
 def scaled(cfg: Config, **kw) -> Config:

@@ -1,0 +1,195 @@
+"""GPU parity of the block and LM entry points against the fp64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+from parity_util import *  # noqa: F401,F403
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def sess():
+    s = Session(0)
+    yield s
+    s.close()
+
+
+def run_block_case(sess, cfg, prec, params, check_update=True):
+    x, dy = synth.block_inputs(cfg)
+    if prec == fx.FAX_PREC_FP32_VALIDATE:       # un-rounded inputs in validation mode
+        x = synth.normal(cfg.seed, synth.TID_X, x.shape)
+        dy = synth.normal(cfg.seed, synth.TID_DY, dy.shape)
+    pc = compute_params(params, prec)
+    B, T, H, hd = cfg.batch, cfg.seq, cfg.n_heads, cfg.head_dim
+    ry, saved = O.block_forward(x, pc, B, T, H, hd, cfg.ln_eps)
+    rdx, rg, _ = O.block_backward(dy, saved, pc, B, T, H, hd)
+    r = BlockRunner(sess, cfg, params, prec)
+    tx, tdy = r.to_device(x), r.to_device(dy)
+    tol_f = TOL_FWD_BF16 if prec == 0 else TOL_FP32
+    tol_g = TOL_GRAD_BF16 if prec == 0 else TOL_FP32
+    y = host(r.forward(tx))
+    assert relerr(y, ry) <= tol_f, "y"
+    dx = host(r.backward(tdy))
+    assert relerr(dx, rdx) <= tol_g, "dx"
+    grads = {k: host(r.p[k].g).reshape(rg[k].shape) for k in O.PARAM_NAMES}
+    for k in O.PARAM_NAMES:
+        assert relerr(grads[k], rg[k]) <= tol_g, k
+    # accumulate = 1 adds a second copy
+    r.backward(tdy, accumulate=True)
+    for k in ("w_fc1", "b_qkv", "ln1_g"):
+        assert relerr(host(r.p[k].g).reshape(rg[k].shape), 2 * rg[k]) <= tol_g, k + " (accumulate)"
+    if not check_update:
+        return
+    # fresh state, whole step through fax_block_step
+    hp = dict(synth.ADAMW)
+    wd = hp.pop("weight_decay")
+    r2 = BlockRunner(sess, cfg, params, prec, weight_decay=wd)
+    r2.step(tx, tdy, hparams(step=1, **hp))
+    assert relerr(host(r2.y), ry) <= tol_f and relerr(host(r2.dx), rdx) <= tol_g
+    for k in O.PARAM_NAMES:
+        g_gpu = host(r2.p[k].g).reshape(rg[k].shape)
+        w_gpu = host(r2.p[k].w).reshape(rg[k].shape)
+        w0 = params[k].astype(np.float64)
+        # composition: the oracle's AdamW applied to the GPU's own gradients
+        cw, cm, cv = O.adamw(w0, 0 * w0, 0 * w0, g_gpu, weight_decay=wd, step=1, **hp)
+        assert relerr(w_gpu, cw) <= TOL_ADAMW, k
+        assert relerr(host(r2.p[k].m).reshape(w0.shape), cm) <= TOL_ADAMW, k
+        # direct: oracle gradients all the way, sign-ambiguous elements bounded separately
+        rw, _, _ = O.adamw(w0, 0 * w0, 0 * w0, rg[k], weight_decay=wd, step=1, **hp)
+        check_adamw_update(k, w_gpu, w0, rg[k], rw, hp["lr"], wd, tol_g, tol_g)
+        if prec == 0:
+            assert torch.equal(r2.p[k].wc, r2.p[k].w.to(torch.bfloat16)), k
+    # warm state at t = 10: the update is Lipschitz in g, plain bound on every tensor
+    r3 = BlockRunner(sess, cfg, params, prec, weight_decay=wd)
+    ref_state = {}
+    for i, k in enumerate(O.PARAM_NAMES):
+        gs = max(np.abs(rg[k]).max(), 1e-12)
+        m0, v0 = synth.warm_state(cfg.seed, i, params[k].shape, gs)
+        r3.p[k].m.copy_(torch.as_tensor(m0)); r3.p[k].v.copy_(torch.as_tensor(v0))
+        ref_state[k] = (m0, v0)
+    r3.step(tx, tdy, hparams(step=10, **hp))
+    for k in O.PARAM_NAMES:
+        m0, v0 = ref_state[k]
+        w0 = params[k].astype(np.float64)
+        rw, _, _ = O.adamw(w0, m0, v0, rg[k], weight_decay=wd, step=10, **hp)
+        # compare the step taken, relative to the largest step
+        step_ref = rw - w0
+        step_gpu = host(r3.p[k].w).reshape(w0.shape) - w0
+        assert np.abs(step_gpu - step_ref).max() <= tol_g * max(np.abs(step_ref).max(), 1e-30) + 1e-7, k
+    st, _ = fx.fax_check_device_status(sess.ctx)
+    assert st == fx.FAX_OK
+
+
+def test_block_fp32_validate_tiny_ragged(sess):
+    cfg = synth.Config("tiny", 7, batch=2, seq=5, d_model=8, n_heads=2, head_dim=4, d_ff=16)
+    run_block_case(sess, cfg, fx.FAX_PREC_FP32_VALIDATE, perturbed_block_params(cfg))
+    cfg = synth.Config("odd", 8, batch=3, seq=37, d_model=96, n_heads=3, head_dim=32, d_ff=200)
+    run_block_case(sess, cfg, fx.FAX_PREC_FP32_VALIDATE, perturbed_block_params(cfg))
+
+
+def test_block_fp32_validate_c1(sess):
+    cfg = synth.CONFIGS["C1"]
+    run_block_case(sess, cfg, fx.FAX_PREC_FP32_VALIDATE, synth.block_params(cfg))
+
+
+def test_block_bf16_c1(sess):
+    cfg = synth.CONFIGS["C1"]
+    run_block_case(sess, cfg, fx.FAX_PREC_BF16, synth.block_params(cfg))
+    run_block_case(sess, cfg, fx.FAX_PREC_BF16, perturbed_block_params(cfg), check_update=False)
+
+
+def test_block_bf16_c2(sess):
+    cfg = synth.CONFIGS["C2"]
+    run_block_case(sess, cfg, fx.FAX_PREC_BF16, synth.block_params(cfg))
+
+
+def test_block_bf16_c3_width_reduced_tokens(sess):
+    # C3's widths (d 4096, 32 heads x 128, FFN 16384) on one 384-token sequence and
+    # a ragged 3 x 128 batch: spans many tiles, finishes in seconds on the CPU side
+    cfg = synth.scaled(synth.CONFIGS["C3"], batch=3, seq=128)
+    run_block_case(sess, cfg, fx.FAX_PREC_BF16, perturbed_block_params(cfg), check_update=False)
+
+
+def test_block_causal_invariance_on_gpu(sess):
+    cfg = synth.CONFIGS["C1"]
+    params = synth.block_params(cfg)
+    x, _ = synth.block_inputs(cfg)
+    r = BlockRunner(sess, cfg, params, fx.FAX_PREC_BF16)
+    y0 = r.forward(r.to_device(x)).clone()
+    t = 70
+    x2 = x.reshape(cfg.batch, cfg.seq, -1).copy()
+    x2[:, t + 1:] = synth.round_to_bf16(5 * np.random.default_rng(0).standard_normal(x2[:, t + 1:].shape).astype(np.float32))
+    y1 = r.forward(r.to_device(x2.reshape(x.shape)))
+    a = y0.view(cfg.batch, cfg.seq, -1)[:, :t + 1]
+    b = y1.view(cfg.batch, cfg.seq, -1)[:, :t + 1]
+    assert torch.equal(a, b)
+
+
+def test_block_error_paths(sess):
+    cfg = synth.CONFIGS["C1"]
+    r = BlockRunner(sess, cfg, synth.block_params(cfg), fx.FAX_PREC_BF16)
+    x = r.to_device(synth.block_inputs(cfg)[0])
+    with pytest.raises(fx.FaxError) as e:
+        fx.fax_block_forward(sess.ctx, r.bcfg, r.params_struct, ptr(x), ptr(r.y), ptr(r.saved), 1024,
+                             ptr(r.scratch), r.scratch_bytes)
+    assert e.value.status == fx.FAX_ERR_WORKSPACE_TOO_SMALL
+    with pytest.raises(fx.FaxError) as e:
+        fx.fax_block_forward(sess.ctx, r.bcfg, r.params_struct, ptr(x), ptr(x), ptr(r.saved), r.saved_bytes,
+                             ptr(r.scratch), r.scratch_bytes)
+    assert e.value.status == fx.FAX_ERR_INVALID_ARG
+
+
+def lm_case(sess, cfg, prec, lm):
+    ids, tg = synth.lm_tokens(cfg)
+    B, T, H, hd = cfg.batch, cfg.seq, cfg.n_heads, cfg.head_dim
+    rnd = (lambda a: synth.round_to_bf16(a).astype(np.float64)) if prec == 0 else (lambda a: a.astype(np.float64))
+    lmc = dict(wte=rnd(lm["wte"]), wpe=rnd(lm["wpe"]), lnf_g=rnd(lm["lnf_g"]), lnf_b=rnd(lm["lnf_b"]),
+               blocks=[{k: rnd(v) for k, v in p.items()} for p in lm["blocks"]])
+    hp = dict(synth.ADAMW)
+    wd = hp.pop("weight_decay")
+    zeros = {n: np.zeros_like(a, dtype=np.float64) for n, a in O.lm_tensors(lm)}
+    rloss, rg, rw, rm, rv = O.lm_step(ids, tg, lmc, zeros, zeros, B, T, H, hd,
+                                      dict(weight_decay=wd, step=1, **hp), cfg.ln_eps, lm_master=lm)
+    r = LmRunner(sess, cfg, lm, prec, weight_decay=wd)
+    tids = torch.as_tensor(ids).to(sess.device)
+    ttg = torch.as_tensor(tg).to(sess.device)
+    tol_f = TOL_FWD_BF16 if prec == 0 else TOL_FP32
+    tol_g = TOL_GRAD_BF16 if prec == 0 else TOL_FP32
+    r.forward_backward(tids, ttg)
+    loss = float(r.loss.item())
+    assert abs(loss - rloss) <= tol_f * abs(rloss)
+    for name, ps in r.named_params():
+        assert relerr(host(ps.g).reshape(rg[name].shape), rg[name]) <= tol_g, name
+    # full step on fresh state, host loss readback
+    r2 = LmRunner(sess, cfg, lm, prec, weight_decay=wd)
+    l2 = r2.step(tids, ttg, hparams(step=1, **hp), want_host_loss=True)
+    assert abs(l2 - rloss) <= tol_f * abs(rloss)
+    for name, ps in r2.named_params():
+        w0 = dict(O.lm_tensors(lm))[name].astype(np.float64)
+        g_gpu = host(ps.g).reshape(w0.shape)
+        cw, _, _ = O.adamw(w0, 0 * w0, 0 * w0, g_gpu, weight_decay=wd, step=1, **hp)
+        assert relerr(host(ps.w).reshape(w0.shape), cw) <= TOL_ADAMW, name
+        check_adamw_update(name, host(ps.w).reshape(w0.shape), w0, rg[name], rw[name], hp["lr"], wd, tol_g, tol_g)
+    # host-buffer entry point gives the same loss
+    r3 = LmRunner(sess, cfg, lm, prec, weight_decay=wd)
+    l3 = r3.step_host(torch.as_tensor(ids).pin_memory(), torch.as_tensor(tg).pin_memory(), hparams(step=1, **hp))
+    assert l3 == l2
+    st, _ = fx.fax_check_device_status(sess.ctx)
+    assert st == fx.FAX_OK
+
+
+def test_lm_fp32_validate_tiny(sess):
+    cfg = synth.Config("lm_tiny", 9, batch=2, seq=5, d_model=8, n_heads=2, head_dim=4, d_ff=16, n_layers=2, vocab=11)
+    lm = synth.lm_params(cfg)
+    for l in range(cfg.n_layers):
+        lm["blocks"][l] = perturbed_block_params(cfg, l)
+    lm["wte"] *= 10; lm["wpe"] *= 10
+    ids, _ = synth.lm_tokens(cfg)
+    lm_case(sess, cfg, fx.FAX_PREC_FP32_VALIDATE, lm)
+
+
+def test_lm_bf16_c4_shape_reduced(sess):
+    # C4's widths and full vocabulary (d 768, 12 x 64, FFN 3072, V 50304), 2 layers, 2 x 128 tokens
+    cfg = synth.scaled(synth.CONFIGS["C4"], batch=2, seq=128, n_layers=2)
+    lm_case(sess, cfg, fx.FAX_PREC_BF16, synth.lm_params(cfg))
