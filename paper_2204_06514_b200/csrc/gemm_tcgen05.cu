@@ -1,3 +1,411 @@
+// bf16 GEMM on the 5th-generation tensor cores: TMA-fed multi-stage shared
+// memory ring, tcgen05.mma issued by one thread with float accumulators in
+// tensor memory, double-buffered so the epilogue of one tile overlaps the main
+// loop of the next, persistent over output tiles.
+//
+//   warp 0      : TMA producer (one elected lane)
+//   warp 1      : tensor-memory allocation, MMA issue (one elected lane)
+//   warps 2..5  : epilogue; warp w reads TMEM lanes 32*(w%4) .. +31
+//
+// Operand layouts (both for A and B, chosen at run time):
+//   K-major  : [rows, K] row-major; one TMA box of 64 k x rows, 128-byte swizzle;
+//              8-row groups 1024 B apart (SBO); a K step of 16 elements is +32 B.
+//   MN-major : [K, rows] row-major; TMA boxes of 64 rows x 64 k (one per 64 rows,
+//              8192 B apart = LBO); 8-k groups 1024 B apart (SBO); a K step of 16
+//              is +2048 B.
+// Every device-side wait is bounded; on expiry the kernel records an error in
+// the context's status word, drains and returns.
 #include "common.cuh"
-bool fax_gemm_tc_supported(const FaxGemm&) { return false; }
-fax_status fax_gemm_tc(fax_ctx*, const FaxGemm&) { return FAX_ERR_UNSUPPORTED_SHAPE; }
+
+#include <cuda.h>
+
+namespace {
+
+constexpr int BM = 128;
+constexpr int BK = 64;
+constexpr int NUM_EPI_WARPS = 4;
+constexpr int NUM_THREADS = 32 * (2 + NUM_EPI_WARPS);
+constexpr long long WAIT_CYCLES = 4000000000LL;     // about two seconds
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when the abort flag is (or gets) set.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          int32_t* status, int code) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  int spins = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++spins & 255) == 0) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > WAIT_CYCLES) {
+        *abort_flag = 1;
+        if (atomicCAS(status, 0, 1) == 0) status[1] = code;
+        return false;
+      }
+    }
+  }
+  return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor (128-byte swizzle).  Addresses and offsets in
+// 16-byte units; bit 46 = descriptor version of this architecture; layout type
+// 2 (bits 61..63) = 128-byte swizzle.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFF) >> 4);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+
+struct GemmParams {
+  int M, N, K;
+  int a_mn, b_mn;
+  void* C; long long ldc; int c_f32; int accumulate;
+  int epi;
+  const bf16* bias;
+  const bf16* resid; long long ldr;
+  bf16* aux; long long ldaux;
+  float alpha;
+  int32_t* status;
+};
+
+template <int BN> struct Cfg {
+  static constexpr int A_BYTES = BM * BK * 2;
+  static constexpr int B_BYTES = BN * BK * 2;
+  static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  static constexpr int STAGES = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
+  static constexpr int TMEM_COLS = 2 * BN < 32 ? 32 : 2 * BN;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+template <int BN>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                    const GemmParams p) {
+  using C_ = Cfg<BN>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t tiles_base = (raw + 1023u) & ~1023u;
+  uint8_t* gen_base = smem_raw + (tiles_base - raw);
+  uint8_t* bar_mem = gen_base + C_::STAGES * C_::STAGE_BYTES;
+  const uint32_t bars = tiles_base + C_::STAGES * C_::STAGE_BYTES;
+  // barrier layout: full[S], empty[S], tmem_full[2], tmem_empty[2], then tmem base word + abort flag
+  auto full_bar = [&](int s) { return bars + 8u * s; };
+  auto empty_bar = [&](int s) { return bars + 8u * (C_::STAGES + s); };
+  auto tfull_bar = [&](int a) { return bars + 8u * (2 * C_::STAGES + a); };
+  auto tempty_bar = [&](int a) { return bars + 8u * (2 * C_::STAGES + 2 + a); };
+  volatile uint32_t* tmem_base_slot = (volatile uint32_t*)(bar_mem + 8 * (2 * C_::STAGES + 4));
+  volatile int* abort_flag = (volatile int*)(bar_mem + 8 * (2 * C_::STAGES + 4) + 4);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tiles_m = p.M / BM, tiles_n = p.N / BN;
+  const int num_tiles = tiles_m * tiles_n;
+  const int kblocks = p.K / BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < C_::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(tfull_bar(a), 1); mbar_init(tempty_bar(a), NUM_EPI_WARPS); }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_b) : "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32((const void*)tmem_base_slot)), "r"((uint32_t)C_::TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_base_slot;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      int stage = 0; uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 101)) { ok = false; break; }
+          const uint32_t a_dst = tiles_base + stage * C_::STAGE_BYTES;
+          const uint32_t b_dst = a_dst + C_::A_BYTES;
+          mbar_expect_tx(full_bar(stage), C_::STAGE_BYTES);
+          const int k0 = kb * BK;
+          if (!p.a_mn) {
+            tma_load_2d(a_dst, &tmap_a, full_bar(stage), k0, m0);
+          } else {
+#pragma unroll
+            for (int i = 0; i < BM / 64; ++i) tma_load_2d(a_dst + i * 8192, &tmap_a, full_bar(stage), m0 + 64 * i, k0);
+          }
+          if (!p.b_mn) {
+            tma_load_2d(b_dst, &tmap_b, full_bar(stage), k0, n0);
+          } else {
+#pragma unroll
+            for (int i = 0; i < BN / 64; ++i) tma_load_2d(b_dst + i * 8192, &tmap_b, full_bar(stage), n0 + 64 * i, k0);
+          }
+          if (++stage == C_::STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        // let copies already in flight land before the block can exit
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) { }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      // instruction descriptor: D = f32, A = B = bf16, majors, N >> 3, M >> 4
+      const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.a_mn ? 1 : 0) << 15) |
+                             ((uint32_t)(p.b_mn ? 1 : 0) << 16) | ((uint32_t)(BN >> 3) << 17) |
+                             ((uint32_t)(BM >> 4) << 24);
+      const uint32_t a_kstep = p.a_mn ? 2048u : 32u, b_kstep = p.b_mn ? 2048u : 32u;
+      const uint32_t a_lbo = p.a_mn ? 8192u : 16u, b_lbo = p.b_mn ? 8192u : 16u;
+      int stage = 0; uint32_t phase = 0;
+      int acc = 0; uint32_t acc_phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status, 102)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status, 103)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t a_src = tiles_base + stage * C_::STAGE_BYTES;
+          const uint32_t b_src = a_src + C_::A_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k) {
+            const uint64_t ad = smem_desc(a_src + k * a_kstep, a_lbo, 1024u);
+            const uint64_t bd = smem_desc(b_src + k * b_kstep, b_lbo, 1024u);
+            tc_mma_bf16(d_tmem, ad, bd, idesc, (kb | k) ? 1u : 0u);
+          }
+          tc_commit(empty_bar(stage));          // frees the smem stage once these MMAs have read it
+          if (++stage == C_::STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (!ok) break;
+        tc_commit(tfull_bar(acc));              // accumulator complete
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else {
+    // ---------------- epilogue ----------------
+    const int q = warp & 3;                      // TMEM lane quarter this warp may read
+    int acc = 0; uint32_t acc_phase = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+      const int m0 = (tile % tiles_m) * BM, n0 = (tile / tiles_m) * BN;
+      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status, 104)) { ok = false; break; }
+      tc_fence_after();
+      const long long row = m0 + 32 * q + lane;
+#pragma unroll 1
+      for (int c0 = 0; c0 < BN; c0 += 32) {
+        uint32_t r[32];
+        tc_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(acc * BN + c0), r);
+        tc_wait_ld();
+        const int col = n0 + c0;
+        float v[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) * p.alpha;
+        if (p.epi == EPI_BIAS || p.epi == EPI_BIAS_GELU || p.epi == EPI_BIAS_RESID) {
+          const uint4* bp = reinterpret_cast<const uint4*>(p.bias + col);
+#pragma unroll
+          for (int j4 = 0; j4 < 4; ++j4) {
+            uint4 u = __ldg(bp + j4);
+            const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { float2 f = __bfloat1622float2(h[e]); v[8 * j4 + 2 * e] += f.x; v[8 * j4 + 2 * e + 1] += f.y; }
+          }
+        }
+        if (p.epi == EPI_BIAS_RESID) {
+          const uint4* rp = reinterpret_cast<const uint4*>(p.resid + row * p.ldr + col);
+#pragma unroll
+          for (int j4 = 0; j4 < 4; ++j4) {
+            uint4 u = rp[j4];
+            const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { float2 f = __bfloat1622float2(h[e]); v[8 * j4 + 2 * e] += f.x; v[8 * j4 + 2 * e + 1] += f.y; }
+          }
+        }
+        if (p.epi == EPI_DGELU) {
+          const uint4* ap = reinterpret_cast<const uint4*>(p.aux + row * p.ldaux + col);
+#pragma unroll
+          for (int j4 = 0; j4 < 4; ++j4) {
+            uint4 u = ap[j4];
+            const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              float2 f = __bfloat1622float2(h[e]);
+              v[8 * j4 + 2 * e] *= gelu_tanh_grad_f(f.x);
+              v[8 * j4 + 2 * e + 1] *= gelu_tanh_grad_f(f.y);
+            }
+          }
+        }
+        if (p.c_f32) {
+          float4* cp = reinterpret_cast<float4*>((float*)p.C + row * p.ldc + col);
+#pragma unroll
+          for (int j4 = 0; j4 < 8; ++j4) {
+            float4 o = make_float4(v[4 * j4], v[4 * j4 + 1], v[4 * j4 + 2], v[4 * j4 + 3]);
+            if (p.accumulate) { float4 c = cp[j4]; o.x += c.x; o.y += c.y; o.z += c.z; o.w += c.w; }
+            cp[j4] = o;
+          }
+        } else {
+          uint4* cp = reinterpret_cast<uint4*>((bf16*)p.C + row * p.ldc + col);
+          uint4* gp = (p.epi == EPI_BIAS_GELU) ? reinterpret_cast<uint4*>(p.aux + row * p.ldaux + col) : nullptr;
+#pragma unroll
+          for (int j4 = 0; j4 < 4; ++j4) {
+            uint4 u;
+            __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&u);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) h[e] = __floats2bfloat162_rn(v[8 * j4 + 2 * e], v[8 * j4 + 2 * e + 1]);
+            cp[j4] = u;
+            if (gp) {
+              // GELU of the stored (rounded) pre-activation, so backward sees the same h
+              uint4 g;
+              __nv_bfloat162* gh = reinterpret_cast<__nv_bfloat162*>(&g);
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                float2 f = __bfloat1622float2(h[e]);
+                gh[e] = __floats2bfloat162_rn(gelu_tanh_f(f.x), gelu_tanh_f(f.y));
+              }
+              gp[j4] = g;
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)C_::TMEM_COLS) : "memory");
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// 2-D bf16 tensor map: inner (contiguous) extent `inner`, `outer` rows of pitch ld elements.
+bool make_map(fax_ctx* ctx, CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint64_t ld,
+              uint32_t box_inner, uint32_t box_outer) {
+  cuuint64_t dims[2] = {inner, outer};
+  cuuint64_t strides[1] = {ld * 2};
+  cuuint32_t box[2] = {box_inner, box_outer};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = ((EncodeTiledFn)ctx->encode_tiled)(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void*)base, dims, strides,
+                                                 box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+int pick_bn(int N) { return (N % 256 == 0) ? 256 : (N % 128 == 0 ? 128 : (N % 64 == 0 ? 64 : 0)); }
+
+template <int BN>
+fax_status launch(fax_ctx* ctx, const FaxGemm& g) {
+  CUtensorMap ma, mb;
+  bool ok = g.a_mn_major ? make_map(ctx, &ma, g.A, g.M, g.K, g.lda, 64, BK)
+                         : make_map(ctx, &ma, g.A, g.K, g.M, g.lda, BK, BM);
+  ok = ok && (g.b_mn_major ? make_map(ctx, &mb, g.B, g.N, g.K, g.ldb, 64, BK)
+                           : make_map(ctx, &mb, g.B, g.K, g.N, g.ldb, BK, BN));
+  if (!ok) return FAX_ERR_INVALID_ARG;
+  GemmParams p;
+  p.M = g.M; p.N = g.N; p.K = g.K; p.a_mn = g.a_mn_major; p.b_mn = g.b_mn_major;
+  p.C = g.C; p.ldc = g.ldc; p.c_f32 = g.c_f32; p.accumulate = g.accumulate; p.epi = g.epi;
+  p.bias = (const bf16*)g.bias; p.resid = (const bf16*)g.resid; p.ldr = g.ldr; p.aux = (bf16*)g.aux; p.ldaux = g.ldaux;
+  p.alpha = g.alpha; p.status = ctx->dev_status;
+  static bool attr_set = false;
+  if (!attr_set) {
+    FAX_CUDA_TRY(ctx, cudaFuncSetAttribute(gemm_tcgen05_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           Cfg<BN>::SMEM_BYTES));
+    attr_set = true;
+  }
+  const int tiles = (g.M / BM) * (g.N / BN);
+  const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
+  gemm_tcgen05_kernel<BN><<<grid, NUM_THREADS, Cfg<BN>::SMEM_BYTES, ctx->stream>>>(ma, mb, p);
+  return fax_after_launch(ctx);
+}
+
+}  // namespace
+
+bool fax_gemm_tc_supported(const FaxGemm& g) {
+  if (g.M % BM || g.K % BK || pick_bn(g.N) == 0) return false;
+  if (g.lda % 8 || g.ldb % 8) return false;
+  if (!fax_aligned(g.A, 16) || !fax_aligned(g.B, 16) || !fax_aligned(g.C, 16)) return false;
+  if (g.ldc % (g.c_f32 ? 4 : 8)) return false;
+  if (g.bias && !fax_aligned(g.bias, 16)) return false;
+  if (g.resid && (!fax_aligned(g.resid, 16) || g.ldr % 8)) return false;
+  if (g.aux && (!fax_aligned(g.aux, 16) || g.ldaux % 8)) return false;
+  return true;
+}
+
+fax_status fax_gemm_tc(fax_ctx* ctx, const FaxGemm& g) {
+  if (!fax_gemm_tc_supported(g)) return FAX_ERR_UNSUPPORTED_SHAPE;
+  switch (pick_bn(g.N)) {
+    case 256: return launch<256>(ctx, g);
+    case 128: return launch<128>(ctx, g);
+    default: return launch<64>(ctx, g);
+  }
+}

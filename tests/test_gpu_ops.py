@@ -119,6 +119,8 @@ def test_gemm_layouts(sess, prec, a_mn, b_mn, shape, force_simt):
     desc = ops.GemmDesc(M, N, K, ptr(tA), M if a_mn else K, a_mn, ptr(tB), N if b_mn else K, b_mn,
                         ptr(tC), N, 0, 0, ops.FAX_EPI_NONE, None, None, 0, None, 0, 1.0, force_simt)
     ops.fax_op_gemm(sess.ctx, prec, desc)
+    st, detail = fx.fax_check_device_status(sess.ctx)
+    assert st == fx.FAX_OK, detail
     ref = A.astype(np.float64) @ B.astype(np.float64).T
     assert relerr(host(tC), ref) <= (TOL_FWD_BF16 if prec == 0 else TOL_FP32)
 
