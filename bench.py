@@ -1,0 +1,388 @@
+#!/usr/bin/env python
+"""Benchmark of the single-GPU training step (forward + backward + AdamW).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config C1..C5] [--impl ours|reference]
+
+Prints ONE JSON line.  `value` = training tokens/s of the whole job with the
+inputs resident in HBM; `e2e` = the same through the host-buffer entry point
+(host->device copies of the step's inputs and device->host read of its results
+inside the timed region).  N > 1 runs N independent replicas (one process per
+GPU, no data-path collective): the step has no exchange step on one device.
+`--impl reference` times the fp64 CPU oracle on a bounded sample instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "training tokens/sec, fwd+bwd+AdamW, 1 GPU (MFU reported beside it)"
+UNIT = "tokens/s"
+NOMINAL_BF16_TFLOPS = 2250.0        # B200 dense bf16, datasheet
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+        except Exception:
+            pass
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc, self.thread = index, [], None, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), [c.strip() for c in line.split(",")]))
+
+    def stop(self, t0: float, t1: float) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        rows = [r for t, r in self.rows if t0 <= t <= t1 + 0.2] or [r for _, r in self.rows]
+        sm, mx, reasons, pw = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1])); pw.append(float(r[2]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+_ORACLE_INPUTS = {}
+
+
+def oracle_sample(cfg, n_tokens: int):
+    """Time the fp64 oracle (as it stands) on a bounded sample of the workload and
+    extrapolate to tokens/s of the full step.  Block configs: forward + backward at
+    full widths on one sequence of n_tokens tokens (time scaled by tokens), plus the
+    oracle's AdamW on the leading 1/16 of every tensor (time scaled by 16).  The LM
+    config: lm_step on one n_tokens sequence with 2 layers, scaled by FLOPs per token."""
+    import numpy as np
+    import threadpoolctl
+    from oracle import fax_oracle as O
+    from paper_2204_06514_b200 import synth
+    seq = min(cfg.seq, n_tokens)
+    small = synth.scaled(cfg, batch=1, seq=seq, n_layers=min(cfg.n_layers, 2) if cfg.is_lm else 1)
+    hp = dict(synth.ADAMW, step=1)
+    info = threadpoolctl.threadpool_info()
+    cores = max((i.get("num_threads", 1) for i in info), default=1)
+    key = (cfg.name, seq)
+    if key not in _ORACLE_INPUTS:
+        rng = np.random.default_rng(0)
+        blocks = [{k: rng.standard_normal(s) * 0.02 for k, s in small.block_param_shapes().items()}
+                  for _ in range(small.n_layers)]
+        if small.is_lm:
+            _ORACLE_INPUTS[key] = dict(
+                lm=dict(wte=rng.standard_normal((small.vocab, small.d_model)) * 0.02,
+                        wpe=rng.standard_normal((seq, small.d_model)) * 0.02, blocks=blocks,
+                        lnf_g=np.ones(small.d_model), lnf_b=np.zeros(small.d_model)),
+                ids=rng.integers(0, small.vocab, (1, seq)))
+        else:
+            _ORACLE_INPUTS[key] = dict(p=blocks[0], x=rng.standard_normal((seq, small.d_model)),
+                                       dy=rng.standard_normal((seq, small.d_model)))
+    inp = _ORACLE_INPUTS[key]
+    if small.is_lm:
+        lm, ids = inp["lm"], inp["ids"]
+        zeros = {n: np.zeros(a.shape) for n, a in O.lm_tensors(lm)}
+        t0 = time.perf_counter()
+        O.lm_step(ids, ids, lm, zeros, zeros, 1, seq, small.n_heads, small.head_dim, hp, small.ln_eps)
+        dt = time.perf_counter() - t0
+        frac = (small.step_flops() / small.tokens) / (cfg.step_flops() / cfg.tokens)
+        full = dt / frac * (cfg.tokens / seq)
+        what = (f"oracle lm_step on 1 x {seq} tokens with {small.n_layers} of {cfg.n_layers} layers, "
+                f"time scaled by FLOPs per token and by tokens to the full step")
+    else:
+        p, x, dy = inp["p"], inp["x"], inp["dy"]
+        t0 = time.perf_counter()
+        y, sv = O.block_forward(x, p, 1, seq, small.n_heads, small.head_dim, small.ln_eps)
+        dx, gr, _ = O.block_backward(dy, sv, p, 1, seq, small.n_heads, small.head_dim)
+        t_fb = time.perf_counter() - t0
+        div = 16 if cfg.n_params > 10_000_000 else 1
+        t0 = time.perf_counter()
+        for k in O.PARAM_NAMES:
+            n = max(1, p[k].shape[0] // div)
+            w, g = p[k][:n], gr[k][:n]
+            O.adamw(w, np.zeros_like(w), np.zeros_like(w), g, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"],
+                    hp["weight_decay"], 1)
+        t_ad = (time.perf_counter() - t0) * div
+        full = t_fb * (cfg.tokens / seq) + t_ad
+        what = (f"oracle block forward+backward at full widths on 1 x {seq} tokens (time scaled by tokens) "
+                f"+ oracle AdamW on the leading 1/{div} of every tensor (time scaled by {div})")
+    return cfg.tokens / full, cores, what
+
+
+SAMPLE_TOKENS = {"C1": 128, "C2": 512, "C3": 128, "C4": 128, "C5": 32}
+
+
+def run_reference(args):
+    """Reference arm: the fp64 oracle on host cores, bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2204_06514_b200 import synth
+    cfg = synth.CONFIGS[args.config]
+    budget = SAMPLE_TOKENS[args.config]
+    vals, cores, what = [], 1, ""
+    for i in range(args.warmup + args.steps):
+        v, cores, what = oracle_sample(cfg, budget)
+        if i >= args.warmup:
+            vals.append(v)
+    tps = sum(vals) / len(vals)
+    line = {"impl": "reference", "metric": METRIC, "value": tps, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * cfg.tokens / tps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": {"workload": workload_name(cfg)},
+            "cpu_baseline": {"value": tps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what},
+            "e2e": {"value": tps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def workload_name(cfg):
+    if cfg.is_lm:
+        return (f"{cfg.name}: {cfg.n_layers}-layer LM step d{cfg.d_model} {cfg.n_heads}x{cfg.head_dim} "
+                f"ffn{cfg.d_ff} vocab{cfg.vocab} batch{cfg.batch} seq{cfg.seq}")
+    return (f"{cfg.name}: pre-LN decoder block fwd+bwd+AdamW d{cfg.d_model} {cfg.n_heads}x{cfg.head_dim} "
+            f"ffn{cfg.d_ff} batch{cfg.batch} seq{cfg.seq}")
+
+
+def run_ours(args):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    from paper_2204_06514_b200 import binding as fx
+    from paper_2204_06514_b200 import build, synth
+    from paper_2204_06514_b200.state import BlockRunner, LmRunner, Session, hparams
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: there is no CPU fallback")
+    if rank == 0:
+        build.build()
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        dist.barrier()
+    torch.cuda.set_device(local)
+    fx.load_library()
+    cfg = synth.CONFIGS[args.config]
+    peaks, peaks_kind = load_peaks()
+    sess = Session(local)
+    dev = sess.device
+    hp0 = dict(synth.ADAMW)
+    wd = hp0.pop("weight_decay")
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(cfg.seed + rank)
+
+    def rand(shape, std):
+        return torch.randn(shape, generator=gen, device=dev, dtype=torch.float32) * std
+
+    # seeded synthetic state, generated on the device (same recipe as the parity inputs:
+    # N(0, 0.02) matrices, zero biases, unit LayerNorm gains; N(0,1) bf16 activations)
+    def block_params():
+        out = {}
+        for k, s in cfg.block_param_shapes().items():
+            out[k] = rand(s, 0.02) if k.startswith("w_") else (torch.ones(s) if k.endswith("_g") else torch.zeros(s))
+        return out
+
+    step_no = [0]
+    if cfg.is_lm:
+        lm = dict(wte=rand((cfg.vocab, cfg.d_model), 0.02), wpe=rand((cfg.seq, cfg.d_model), 0.02),
+                  blocks=[block_params() for _ in range(cfg.n_layers)],
+                  lnf_g=torch.ones(cfg.d_model), lnf_b=torch.zeros(cfg.d_model))
+        runner = LmRunner(sess, cfg, lm, fx.FAX_PREC_BF16, weight_decay=wd)
+        raw = torch.randint(0, cfg.vocab, (cfg.batch, cfg.seq + 1), generator=gen, device=dev, dtype=torch.int32)
+        ids, tg = raw[:, :-1].contiguous(), raw[:, 1:].contiguous()
+        ids_h, tg_h = ids.cpu().pin_memory(), tg.cpu().pin_memory()
+        h2d, d2h = 2 * ids_h.numel() * 4, 4
+
+        def step():
+            step_no[0] += 1
+            runner.step(ids, tg, hparams(step=step_no[0], **hp0))
+
+        def step_host():
+            step_no[0] += 1
+            runner.step_host(ids_h, tg_h, hparams(step=step_no[0], **hp0))
+    else:
+        runner = BlockRunner(sess, cfg, block_params(), fx.FAX_PREC_BF16, weight_decay=wd, host_io=True)
+        x = torch.randn((cfg.tokens, cfg.d_model), generator=gen, device=dev).to(torch.bfloat16)
+        dy = torch.randn((cfg.tokens, cfg.d_model), generator=gen, device=dev).to(torch.bfloat16)
+        x_h, dy_h = x.cpu().pin_memory(), dy.cpu().pin_memory()
+        y_h, dx_h = torch.empty_like(x_h).pin_memory(), torch.empty_like(x_h).pin_memory()
+        h2d = 2 * x_h.numel() * 2
+        d2h = 2 * x_h.numel() * 2
+
+        def step():
+            step_no[0] += 1
+            runner.step(x, dy, hparams(step=step_no[0], **hp0))
+
+        def step_host():
+            step_no[0] += 1
+            runner.step_host(x_h, dy_h, y_h, dx_h, hparams(step=step_no[0], **hp0))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        """K steps between two CUDA events on the launching stream; max over ranks."""
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(sess.stream)
+        for _ in range(steps):
+            fn()
+        e1.record(sess.stream)
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if world > 1:
+            t = torch.tensor([ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.25)
+    l0 = sess.launches()
+    t0 = time.time()
+    ms = timed(step, args.steps)
+    t1 = time.time()
+    launches = sess.launches() - l0
+    clocks = sampler.stop(t0, t1)
+    st, detail = fx.fax_check_device_status(sess.ctx)
+    if st != fx.FAX_OK:
+        raise RuntimeError(f"device status {st} detail {detail}")
+
+    # end to end through the host-buffer entry point
+    step_host()
+    e2e_steps = max(1, min(args.steps, 10))
+    ms_e2e = timed(step_host, e2e_steps)
+
+    # per-kernel profile over whole steps (events around every operator launch)
+    fx.fax_profile_begin(sess.ctx)
+    prof_steps = max(1, min(args.steps, 5))
+    for _ in range(prof_steps):
+        step()
+    prof = fx.fax_profile_end(sess.ctx)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    ms_step = ms / args.steps
+    tokens = cfg.tokens
+    tps = world * tokens / (ms_step * 1e-3)
+    flops = cfg.step_flops()
+    achieved_tf = flops / (ms_step * 1e-3) / 1e12
+    kernels = {}
+    total_ms = sum(v["ms"] for v in prof.values()) or 1.0
+    for name, v in prof.items():
+        per = v["ms"] / v["launches"]
+        ent = {"launches_per_step": v["launches"] / prof_steps, "ms_per_step": v["ms"] / prof_steps,
+               "share": v["ms"] / total_ms, "avg_launch_ms": per}
+        if v["flops"] > 0:
+            ent.update(bound="tensor", achieved=v["flops"] / (v["ms"] * 1e-3) / 1e12, unit="TFLOP/s")
+            ent["frac"] = ent["achieved"] / peaks["bf16_tflops_sustained"]
+        else:
+            ent.update(bound="hbm", achieved=v["bytes"] / (v["ms"] * 1e-3) / 1e9, unit="GB/s")
+            ent["frac"] = ent["achieved"] / peaks["hbm_gbs"]
+        kernels[name] = ent
+    top = max(kernels, key=lambda k: kernels[k]["ms_per_step"])
+    tk = kernels[top]
+    roofline = {"kernel": top, "bound": tk["bound"], "achieved": tk["achieved"],
+                "peak": peaks["bf16_tflops_sustained"] if tk["bound"] == "tensor" else peaks["hbm_gbs"],
+                "unit": tk["unit"], "frac": tk["frac"], "traffic": None,
+                "peak_source": f"{peaks_kind} ({'sustained bf16 GEMM' if tk['bound'] == 'tensor' else 'copy'})",
+                "per_launch": {"avg_ms": tk["avg_launch_ms"],
+                               "algorithmic": (prof[top]["flops"] or prof[top]["bytes"]) / prof[top]["launches"]}}
+
+    cpu_val, cores, what = oracle_sample(cfg, SAMPLE_TOKENS[cfg.name])
+
+    line = {
+        "metric": METRIC, "value": tps, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": workload_name(cfg), "tokens_per_step": tokens, "params": cfg.n_params,
+                   "replicas": world, "l2": "working set per step far exceeds the 126 MB L2"
+                   if cfg.n_params * 2 > 200e6 else "working set is L2-resident (small parity config)"},
+        "mfu": {"step_flops": flops, "achieved_tflops": achieved_tf,
+                "vs_nominal_2250": achieved_tf / NOMINAL_BF16_TFLOPS,
+                "vs_measured_sustained": achieved_tf / peaks["bf16_tflops_sustained"],
+                "flops_convention": "6*matmul_params*tokens + causal-halved attention (6*B*T^2*d per layer)"},
+        "roofline": roofline, "kernels": kernels,
+        "cpu_baseline": {"value": cpu_val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what},
+        "e2e": {"value": world * tokens / (ms_e2e / e2e_steps * 1e-3), "unit": UNIT,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": launches, "clocks": clocks,
+    }
+    print(json.dumps(line), flush=True)
+    sess.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", default="C3", choices=["C1", "C2", "C3", "C4", "C5"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

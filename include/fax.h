@@ -74,6 +74,21 @@ fax_status fax_check_device_status(fax_ctx* ctx, int32_t* detail_host);
 /* Number of kernel launches this context has enqueued since creation. */
 uint64_t fax_launch_count(const fax_ctx* ctx);
 
+/* Per-kernel profile.  Between fax_profile_begin and fax_profile_end every
+ * operator launch on this context is bracketed by a pair of CUDA events on the
+ * context's stream.  fax_profile_end synchronises the stream and fills `out`
+ * (HOST array of n_out >= FAX_KERNEL_CLASSES entries, indexed by kernel class)
+ * with, per class: operator launches, summed device milliseconds, summed
+ * algorithmic FLOPs (2 per multiply-add) and summed algorithmic bytes (what the
+ * operator must read and write once).  Profiling costs two event records per
+ * launch, so timed runs keep it off. */
+#define FAX_KERNEL_CLASSES 10
+typedef struct { int64_t launches; double ms, flops, bytes; } fax_profile_entry;
+fax_status fax_profile_begin(fax_ctx* ctx);
+fax_status fax_profile_end(fax_ctx* ctx, fax_profile_entry* out, int32_t n_out);
+/* Name of a kernel class ("gemm_tcgen05", "attention_fwd", "layernorm_fwd", "adamw", ...). */
+const char* fax_kernel_class_name(int32_t cls);
+
 typedef enum { FAX_PREC_BF16 = 0, FAX_PREC_FP32_VALIDATE = 1 } fax_precision;
 
 /* One pre-LayerNorm decoder block with a causal mask (always causal). */

@@ -29,6 +29,13 @@ class FaxError(RuntimeError):
         super().__init__(f"{where}: {status_string(status)} ({status})")
 
 
+FAX_KERNEL_CLASSES = 10
+
+
+class ProfileEntry(C.Structure):
+    _fields_ = [("launches", C.c_int64), ("ms", C.c_double), ("flops", C.c_double), ("bytes", C.c_double)]
+
+
 class BlockCfg(C.Structure):
     _fields_ = [("batch", C.c_int32), ("seq", C.c_int32), ("d_model", C.c_int32), ("n_heads", C.c_int32),
                 ("head_dim", C.c_int32), ("d_ff", C.c_int32), ("ln_eps", C.c_float), ("prec", C.c_int32)]
@@ -84,6 +91,9 @@ _SIGNATURES = {
     "fax_last_cuda_error": (C.c_int32, [_P]),
     "fax_check_device_status": (C.c_int32, [_P, C.POINTER(C.c_int32)]),
     "fax_launch_count": (C.c_uint64, [_P]),
+    "fax_profile_begin": (C.c_int32, [_P]),
+    "fax_profile_end": (C.c_int32, [_P, C.POINTER(ProfileEntry), C.c_int32]),
+    "fax_kernel_class_name": (C.c_char_p, [C.c_int32]),
     "fax_block_sizes": (C.c_int32, [C.POINTER(BlockCfg), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]),
     "fax_block_forward": (C.c_int32, [_P, C.POINTER(BlockCfg), C.POINTER(BlockParams), _P, _P, _P,
                                       C.c_size_t, _P, C.c_size_t]),
@@ -164,6 +174,26 @@ def fax_check_device_status(ctx) -> tuple[int, int]:
     if s not in (FAX_OK, FAX_ERR_TIMEOUT):
         raise FaxError(s, "fax_check_device_status")
     return s, d.value
+
+
+def fax_profile_begin(ctx):
+    _check(load_library().fax_profile_begin(ctx), "fax_profile_begin")
+
+
+def fax_profile_end(ctx) -> dict:
+    """Per kernel class: dict(launches, ms, flops, bytes); classes never launched are left out."""
+    arr = (ProfileEntry * FAX_KERNEL_CLASSES)()
+    _check(load_library().fax_profile_end(ctx, arr, FAX_KERNEL_CLASSES), "fax_profile_end")
+    out = {}
+    for i in range(FAX_KERNEL_CLASSES):
+        if arr[i].launches:
+            out[fax_kernel_class_name(i)] = dict(launches=arr[i].launches, ms=arr[i].ms, flops=arr[i].flops,
+                                                 bytes=arr[i].bytes)
+    return out
+
+
+def fax_kernel_class_name(cls: int) -> str:
+    return load_library().fax_kernel_class_name(cls).decode()
 
 
 def fax_block_sizes(cfg: BlockCfg) -> tuple[int, int]:

@@ -105,6 +105,10 @@ fax_status fax_adamw_launch(fax_ctx* ctx, const fax_adamw_tensor* tensors, int n
         (t.w_compute && !fax_aligned(t.w_compute, 8)))
       return FAX_ERR_INVALID_ARG;
   }
+  double total = 0;
+  for (int j = 0; j < n; ++j) total += (double)tensors[j].n;
+  // read w, m, v, g; write w, m, v and the bf16 copy
+  FaxProfScope prof(ctx, KC_ADAMW, 0.0, total * (hp->grad_is_bf16 ? 28.0 : 30.0));
   int i = 0;
   while (i < n) {
     AdamBatch batch;

@@ -34,6 +34,7 @@ extern "C" fax_status fax_create(fax_ctx** out, int32_t device_ordinal, void* cu
   c->sm_count = prop.multiProcessorCount;
   c->dev_status = nullptr;
   c->encode_tiled = nullptr;
+  c->prof_on = false;
   if (cudaMalloc((void**)&c->dev_status, 64) != cudaSuccess ||
       cudaMemset(c->dev_status, 0, 64) != cudaSuccess) {
     delete c;
@@ -58,6 +59,7 @@ extern "C" fax_status fax_destroy(fax_ctx* ctx) {
   cudaSetDevice(ctx->device);
   cudaStreamSynchronize(ctx->stream);
   if (ctx->dev_status) cudaFree(ctx->dev_status);
+  for (FaxProfRec& r : ctx->prof) { cudaEventDestroy(r.e0); cudaEventDestroy(r.e1); }
   delete ctx;
   return FAX_OK;
 }
@@ -76,4 +78,34 @@ extern "C" fax_status fax_check_device_status(fax_ctx* ctx, int32_t* detail_host
     return FAX_ERR_TIMEOUT;
   }
   return FAX_OK;
+}
+
+extern "C" fax_status fax_profile_begin(fax_ctx* ctx) {
+  if (!ctx) return FAX_ERR_INVALID_ARG;
+  for (FaxProfRec& r : ctx->prof) { cudaEventDestroy(r.e0); cudaEventDestroy(r.e1); }
+  ctx->prof.clear();
+  ctx->prof_on = true;
+  return FAX_OK;
+}
+
+extern "C" fax_status fax_profile_end(fax_ctx* ctx, fax_profile_entry* out, int32_t n_out) {
+  if (!ctx || !out || n_out < FAX_KERNEL_CLASSES) return FAX_ERR_INVALID_ARG;
+  ctx->prof_on = false;
+  FAX_CUDA_TRY(ctx, cudaStreamSynchronize(ctx->stream));
+  for (int i = 0; i < FAX_KERNEL_CLASSES; ++i) { out[i].launches = 0; out[i].ms = 0; out[i].flops = 0; out[i].bytes = 0; }
+  for (FaxProfRec& r : ctx->prof) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, r.e0, r.e1) == cudaSuccess && r.cls >= 0 && r.cls < FAX_KERNEL_CLASSES) {
+      out[r.cls].launches += 1; out[r.cls].ms += ms; out[r.cls].flops += r.flops; out[r.cls].bytes += r.bytes;
+    }
+    cudaEventDestroy(r.e0); cudaEventDestroy(r.e1);
+  }
+  ctx->prof.clear();
+  return FAX_OK;
+}
+
+extern "C" const char* fax_kernel_class_name(int32_t cls) {
+  static const char* names[FAX_KERNEL_CLASSES] = {"gemm_tcgen05", "gemm_simt", "attention_fwd", "attention_bwd",
+                                                  "layernorm_fwd", "layernorm_bwd", "adamw", "colsum", "embed", "xent"};
+  return (cls >= 0 && cls < FAX_KERNEL_CLASSES) ? names[cls] : "unknown";
 }

@@ -7,9 +7,18 @@
 #include <stdint.h>
 #include <stddef.h>
 
+#include <vector>
+
 #include "../../include/fax.h"
 
 typedef __nv_bfloat16 bf16;
+
+// Kernel classes of the per-kernel profile (order fixed by fax.h).
+enum FaxKernelClass {
+  KC_GEMM_TC = 0, KC_GEMM_SIMT, KC_ATTN_FWD, KC_ATTN_BWD, KC_LN_FWD, KC_LN_BWD, KC_ADAMW, KC_COLSUM,
+  KC_EMBED, KC_XENT, KC_COUNT
+};
+struct FaxProfRec { int cls; cudaEvent_t e0, e1; double flops, bytes; };
 
 // Device status block owned by the context: word 0 = error flag, word 1 = detail.
 struct fax_ctx {
@@ -20,6 +29,22 @@ struct fax_ctx {
   uint64_t launches;
   int sm_count;
   void* encode_tiled;        // cuTensorMapEncodeTiled, resolved at create
+  bool prof_on;
+  std::vector<FaxProfRec> prof;
+};
+
+// Brackets the launches of one operator with CUDA events while profiling is on.
+struct FaxProfScope {
+  fax_ctx* c; int idx;
+  FaxProfScope(fax_ctx* ctx, int cls, double flops, double bytes) : c(ctx), idx(-1) {
+    if (!ctx->prof_on) return;
+    FaxProfRec r; r.cls = cls; r.flops = flops; r.bytes = bytes; r.e0 = nullptr; r.e1 = nullptr;
+    if (cudaEventCreate(&r.e0) != cudaSuccess || cudaEventCreate(&r.e1) != cudaSuccess) return;
+    cudaEventRecord(r.e0, ctx->stream);
+    ctx->prof.push_back(r);
+    idx = (int)ctx->prof.size() - 1;
+  }
+  ~FaxProfScope() { if (idx >= 0) cudaEventRecord(c->prof[idx].e1, c->stream); }
 };
 
 #define FAX_CUDA_TRY(ctx, expr)                                   \

@@ -13,6 +13,8 @@ size_t fax_attention_bwd_scratch_bytes(int prec, int B, int T, int H, int hd) {
 
 fax_status fax_attention_fwd(fax_ctx* ctx, int prec, int B, int T, int H, int hd, const void* qkv,
                              void* o, float* lse) {
+  // causal half of QK^T and PV
+  FaxProfScope prof(ctx, KC_ATTN_FWD, 2.0 * B * H * (double)T * T * hd, 0.0);
   return fax_attention_fwd_simt(ctx, prec, B, T, H, hd, qkv, o, lse);
 }
 
@@ -20,5 +22,7 @@ fax_status fax_attention_bwd(fax_ctx* ctx, int prec, int B, int T, int H, int hd
                              const void* o, const float* lse, const void* d_o, void* dqkv,
                              void* scratch, size_t scratch_bytes) {
   if (scratch_bytes < (size_t)B * H * T * sizeof(float)) return FAX_ERR_WORKSPACE_TOO_SMALL;
+  // causal half of dV, dP, dQ, dK (the recomputed QK^T is not counted)
+  FaxProfScope prof(ctx, KC_ATTN_BWD, 4.0 * B * H * (double)T * T * hd, 0.0);
   return fax_attention_bwd_simt(ctx, prec, B, T, H, hd, qkv, o, lse, d_o, dqkv, (float*)scratch);
 }

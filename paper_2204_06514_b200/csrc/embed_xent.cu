@@ -109,6 +109,7 @@ __global__ void loss_mean_kernel(int n, const float* __restrict__ row_loss, floa
 fax_status fax_embed_fwd(fax_ctx* ctx, int prec, int B, int T, int d, int vocab, const int32_t* ids,
                          const void* wte, const void* wpe, void* x0) {
   int n = B * T;
+  FaxProfScope prof(ctx, KC_EMBED, 0.0, 3.0 * n * d * fax_elem_size(prec));
   if (prec == FAX_PREC_BF16)
     embed_fwd_kernel<bf16><<<n, 128, 0, ctx->stream>>>(n, T, d, vocab, ids, (const bf16*)wte, (const bf16*)wpe, (bf16*)x0);
   else
@@ -119,6 +120,7 @@ fax_status fax_embed_fwd(fax_ctx* ctx, int prec, int B, int T, int d, int vocab,
 fax_status fax_embed_bwd(fax_ctx* ctx, int prec, int B, int T, int max_seq, int d, int vocab,
                          const int32_t* ids, const void* dx0, float* dwte, float* dwpe) {
   int n = B * T;
+  FaxProfScope prof(ctx, KC_EMBED, 0.0, (double)n * d * (2.0 * fax_elem_size(prec) + 8.0));
   if (prec == FAX_PREC_BF16) {
     embed_bwd_wte_kernel<bf16><<<n, 128, 0, ctx->stream>>>(n, d, vocab, ids, (const bf16*)dx0, dwte);
     FAX_TRY(fax_after_launch(ctx));
@@ -133,6 +135,8 @@ fax_status fax_embed_bwd(fax_ctx* ctx, int prec, int B, int T, int max_seq, int 
 
 fax_status fax_xent(fax_ctx* ctx, int prec, int rows, int vocab, void* logits, int64_t ld,
                     const int32_t* targets, float inv_n, float* row_loss) {
+  // read the logits once, write dlogits once
+  FaxProfScope prof(ctx, KC_XENT, 0.0, 2.0 * rows * (double)vocab * fax_elem_size(prec));
   if (prec == FAX_PREC_BF16)
     xent_kernel<bf16><<<rows, 512, 0, ctx->stream>>>(rows, vocab, (bf16*)logits, ld, targets, inv_n, row_loss);
   else

@@ -98,5 +98,6 @@ fax_status launch(fax_ctx* ctx, const FaxGemm& g) {
 
 fax_status fax_gemm_simt(fax_ctx* ctx, int prec, const FaxGemm& g) {
   if (g.M <= 0 || g.N <= 0 || g.K <= 0) return FAX_ERR_INVALID_ARG;
+  FaxProfScope prof(ctx, KC_GEMM_SIMT, 2.0 * g.M * g.N * g.K, 0.0);
   return prec == FAX_PREC_BF16 ? launch<bf16>(ctx, g) : launch<float>(ctx, g);
 }

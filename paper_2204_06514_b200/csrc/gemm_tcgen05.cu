@@ -403,6 +403,7 @@ bool fax_gemm_tc_supported(const FaxGemm& g) {
 
 fax_status fax_gemm_tc(fax_ctx* ctx, const FaxGemm& g) {
   if (!fax_gemm_tc_supported(g)) return FAX_ERR_UNSUPPORTED_SHAPE;
+  FaxProfScope prof(ctx, KC_GEMM_TC, 2.0 * g.M * g.N * g.K, 0.0);
   switch (pick_bn(g.N)) {
     case 256: return launch<256>(ctx, g);
     case 128: return launch<128>(ctx, g);

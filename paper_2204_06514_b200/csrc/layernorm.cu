@@ -280,6 +280,8 @@ size_t fax_layernorm_bwd_partial_floats(int rows, int d) {
 
 fax_status fax_layernorm_fwd(fax_ctx* ctx, int prec, int rows, int d, const void* x, const void* gamma,
                              const void* beta, float eps, void* out, float* mu, float* rstd, void* x_copy) {
+  // read x, write out (and the optional copy of x)
+  FaxProfScope prof(ctx, KC_LN_FWD, 0.0, (double)rows * d * fax_elem_size(prec) * (x_copy ? 3 : 2));
   if (prec == FAX_PREC_BF16) {
     if (d % 8) return FAX_ERR_UNSUPPORTED_SHAPE;
     return ln_fwd_t<bf16>(ctx, rows, d, x, gamma, beta, eps, out, mu, rstd, x_copy);
@@ -294,6 +296,8 @@ fax_status fax_layernorm_bwd(fax_ctx* ctx, int prec, int rows, int d, const void
                              size_t partial_floats) {
   if (ctx->sm_count > 256) return FAX_ERR_ARCH;
   if (partial_floats < (size_t)2 * ln_bwd_slabs(ctx, rows) * d) return FAX_ERR_WORKSPACE_TOO_SMALL;
+  // read da, x (and add), write dx
+  FaxProfScope prof(ctx, KC_LN_BWD, 0.0, (double)rows * d * fax_elem_size(prec) * (add ? 4 : 3));
   if (prec == FAX_PREC_BF16) {
     if (d % 8) return FAX_ERR_UNSUPPORTED_SHAPE;
     return ln_bwd_t<bf16>(ctx, rows, d, da, x, mu, rstd, gamma, add, dx, dgamma, dbeta, accumulate, partial);
@@ -320,6 +324,7 @@ fax_status fax_colsum(fax_ctx* ctx, int prec, int rows, int cols, const void* in
   if (slabs > 256) slabs = 256;
   if (slabs < 1) slabs = 1;
   if (partial_floats < (size_t)slabs * cols) return FAX_ERR_WORKSPACE_TOO_SMALL;
+  FaxProfScope prof(ctx, KC_COLSUM, 0.0, (double)rows * cols * fax_elem_size(prec));
   dim3 grid(gx, slabs);
   if (prec == FAX_PREC_BF16)
     colsum_partial_kernel<bf16><<<grid, threads, 0, ctx->stream>>>(rows, cols, (const bf16*)in, ld, partial);
