@@ -183,3 +183,6 @@ fax_status fax_embed_bwd(fax_ctx* ctx, int prec, int B, int T, int max_seq, int 
 fax_status fax_xent(fax_ctx* ctx, int prec, int rows, int vocab, void* logits, int64_t ld,
                     const int32_t* targets, float inv_n, float* row_loss);
 fax_status fax_loss_mean(fax_ctx* ctx, int n, const float* row_loss, float* loss);
+
+bool fax_attention_tc_supported(int B, int T, int H, int hd);
+fax_status fax_attention_fwd_tc(fax_ctx* ctx, int B, int T, int H, int hd, const void* qkv, void* o, float* lse);

@@ -15,6 +15,8 @@ fax_status fax_attention_fwd(fax_ctx* ctx, int prec, int B, int T, int H, int hd
                              void* o, float* lse) {
   // causal half of QK^T and PV
   FaxProfScope prof(ctx, KC_ATTN_FWD, 2.0 * B * H * (double)T * T * hd, 0.0);
+  if (prec == FAX_PREC_BF16 && fax_attention_tc_supported(B, T, H, hd))
+    return fax_attention_fwd_tc(ctx, B, T, H, hd, qkv, o, lse);
   return fax_attention_fwd_simt(ctx, prec, B, T, H, hd, qkv, o, lse);
 }
 
