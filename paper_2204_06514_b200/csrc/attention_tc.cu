@@ -249,6 +249,303 @@ fax_status launch_fwd(fax_ctx* ctx, int B, int T, int H, const void* qkv, void* 
   return fax_after_launch(ctx);
 }
 
+
+// ---------------------------------------------------------------------------
+// Backward.  One CTA per (batch, head, 128-key tile j); it keeps K_j and V_j in
+// shared memory and walks the query tiles i >= j.  Per step the elected thread
+// issues S = Q_i K_j^T and dP = dO_i V_j^T; the row threads (one query row
+// each) form P = exp(S/sqrt(hd) - LSE) and dS = P * (dP - D) and write both as
+// bf16 operand tiles; the elected thread then issues dV_j += P^T dO_i and
+// dK_j += dS^T Q_i (accumulating in tensor memory over the whole walk) and
+// dQ_i = dS K_j, which the row threads add into a float32 dQ buffer with vector
+// atomics.  The P / dS / Q / dO / K tiles are each used both as a K-major and as
+// an MN-major operand: the bytes are the same, only the descriptor differs.
+// Tensor memory: [0,128) S then dQ, [128,256) dP, [256,256+HD) dV, [384,384+HD) dK.
+// ---------------------------------------------------------------------------
+constexpr int BWD_THREADS = 160;
+
+struct AttnBwdParams {
+  int B, T, H;
+  const float* lse; const float* Dv;
+  float* dq_acc; bf16* dqkv;
+  float scale, scale_log2;
+  int32_t* status;
+};
+
+template <int HD> struct BwdCfg {
+  static constexpr int TILE_BYTES = 128 * HD * 2;
+  static constexpr int PS_BYTES = 128 * 128 * 2;
+  static constexpr int K_OFF = 0, V_OFF = TILE_BYTES, Q_OFF = 2 * TILE_BYTES, DO_OFF = 3 * TILE_BYTES;
+  static constexpr int P_OFF = 4 * TILE_BYTES, DS_OFF = P_OFF + PS_BYTES;
+  static constexpr int BAR_OFF = DS_OFF + PS_BYTES;
+  static constexpr int SMEM_BYTES = BAR_OFF + 128 + 1024;
+  static constexpr int TMEM_COLS = 512;
+};
+
+template <int HD>
+__global__ void __launch_bounds__(BWD_THREADS, 1)
+attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_constant__ CUtensorMap tmap_do,
+                   const AttnBwdParams p) {
+  using C_ = BwdCfg<HD>;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  uint8_t* gbase = smem_raw + (base - raw);
+  const uint32_t bars = base + C_::BAR_OFF;
+  // barriers: 0 K/V, 1 Q/dO, 2 S+dP, 3 P+dS (4 arrivals), 4 dV/dK/dQ issued and done, 5 dQ read out (4 arrivals)
+  auto bar = [&](int i) { return bars + 8u * i; };
+  volatile uint32_t* tmem_slot = (volatile uint32_t*)(gbase + C_::BAR_OFF + 64);
+  volatile int* abort_flag = (volatile int*)(gbase + C_::BAR_OFF + 68);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nq = p.T / 128;
+  const int bh_count = p.B * p.H;
+  const int kj = (int)(blockIdx.x / bh_count);             // heaviest key tiles (small j) first
+  const int bh = blockIdx.x % bh_count;
+  const int b = bh / p.H, h = bh % p.H;
+  const int d = p.H * HD;
+  const int row0 = b * p.T;
+  const int qcol = h * HD, kcol = d + h * HD, vcol = 2 * d + h * HD;
+  const int nsteps = nq - kj;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < 6; ++i) mbar_init(bar(i), (i == 3 || i == 5) ? 4u : 1u);
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_qkv) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_do) : "memory");
+  }
+  if (warp == 4) tmem_alloc(smem_u32((const void*)tmem_slot), C_::TMEM_COLS);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t tm_s = tmem, tm_dp = tmem + 128, tm_dv = tmem + 256, tm_dk = tmem + 384;
+
+  if (warp == 4) {
+    if (lane == 0) {
+      const uint32_t k_s = base + C_::K_OFF, v_s = base + C_::V_OFF, q_s = base + C_::Q_OFF, do_s = base + C_::DO_OFF;
+      const uint32_t p_s = base + C_::P_OFF, ds_s = base + C_::DS_OFF;
+      const uint32_t idesc_s = idesc_bf16(128, false, false);
+      const uint32_t idesc_kv = idesc_bf16(HD, true, true);
+      const uint32_t idesc_q = idesc_bf16(HD, false, true);
+      auto koff = [](int s) { return (uint32_t)((s / 4) * 16384 + (s % 4) * 32); };   // K-major k-step
+      // K_j, V_j once
+      mbar_expect_tx(bar(0), 2 * C_::TILE_BYTES);
+#pragma unroll
+      for (int i = 0; i < HD / 64; ++i) {
+        tma_load_2d(k_s + i * 16384, &tmap_qkv, bar(0), kcol + 64 * i, row0 + kj * 128);
+        tma_load_2d(v_s + i * 16384, &tmap_qkv, bar(0), vcol + 64 * i, row0 + kj * 128);
+      }
+      auto load_q_do = [&](int qi) {
+        mbar_expect_tx(bar(1), 2 * C_::TILE_BYTES);
+#pragma unroll
+        for (int i = 0; i < HD / 64; ++i) {
+          tma_load_2d(q_s + i * 16384, &tmap_qkv, bar(1), qcol + 64 * i, row0 + qi * 128);
+          tma_load_2d(do_s + i * 16384, &tmap_do, bar(1), qcol + 64 * i, row0 + qi * 128);
+        }
+      };
+      load_q_do(kj);
+      bool ok = mbar_wait(bar(0), 0, abort_flag, p.status, 301);
+      for (int it = 0; it < nsteps && ok; ++it) {
+        const uint32_t ph = (uint32_t)(it & 1);
+        if (!mbar_wait(bar(1), ph, abort_flag, p.status, 302)) { ok = false; break; }
+        if (it > 0 && !mbar_wait(bar(5), ph ^ 1u, abort_flag, p.status, 303)) { ok = false; break; }  // dQ of it-1 read
+        tc_fence_after();
+#pragma unroll
+        for (int s = 0; s < HD / 16; ++s)
+          tc_mma_bf16(tm_s, smem_desc(q_s + koff(s), 16, 1024), smem_desc(k_s + koff(s), 16, 1024), idesc_s, s ? 1u : 0u);
+#pragma unroll
+        for (int s = 0; s < HD / 16; ++s)
+          tc_mma_bf16(tm_dp, smem_desc(do_s + koff(s), 16, 1024), smem_desc(v_s + koff(s), 16, 1024), idesc_s, s ? 1u : 0u);
+        tc_commit(bar(2));
+        if (!mbar_wait(bar(3), ph, abort_flag, p.status, 304)) { ok = false; break; }
+        tc_fence_after();
+#pragma unroll
+        for (int s = 0; s < 8; ++s)      // dV += P^T dO   (contraction over the 128 queries)
+          tc_mma_bf16(tm_dv, smem_desc(p_s + s * 2048, 16384, 1024), smem_desc(do_s + s * 2048, 16384, 1024),
+                      idesc_kv, (it | s) ? 1u : 0u);
+#pragma unroll
+        for (int s = 0; s < 8; ++s)      // dK += dS^T Q
+          tc_mma_bf16(tm_dk, smem_desc(ds_s + s * 2048, 16384, 1024), smem_desc(q_s + s * 2048, 16384, 1024),
+                      idesc_kv, (it | s) ? 1u : 0u);
+#pragma unroll
+        for (int s = 0; s < 8; ++s)      // dQ = dS K   (contraction over the 128 keys)
+          tc_mma_bf16(tm_s, smem_desc(ds_s + koff(s), 16, 1024), smem_desc(k_s + s * 2048, 16384, 1024),
+                      idesc_q, s ? 1u : 0u);
+        tc_commit(bar(4));
+        if (it + 1 < nsteps) {
+          if (!mbar_wait(bar(4), ph, abort_flag, p.status, 305)) { ok = false; break; }   // Q, dO tiles free
+          load_q_do(kj + it + 1);
+        }
+      }
+      if (!ok) { const long long t0 = clock64(); while (clock64() - t0 < 2000000LL) { } }
+    }
+  } else {
+    const int r = 32 * warp + lane;
+    const uint32_t lane_base = (uint32_t)(32 * warp) << 16;
+    uint8_t* p_row = gbase + C_::P_OFF + r * 128;
+    uint8_t* ds_row = gbase + C_::DS_OFF + r * 128;
+    bool ok = true;
+    for (int it = 0; it < nsteps; ++it) {
+      const uint32_t ph = (uint32_t)(it & 1);
+      const int qi = kj + it;
+      const long long tok = (long long)row0 + qi * 128 + r;
+      const long long stat = ((long long)b * p.H + h) * p.T + qi * 128 + r;
+      const float lse2 = p.lse[stat] * 1.4426950408889634f;
+      const float Dr = p.Dv[stat];
+      if (!mbar_wait(bar(2), ph, abort_flag, p.status, 306)) { ok = false; break; }
+      tc_fence_after();
+      const bool diag = (it == 0);
+#pragma unroll 1
+      for (int c0 = 0; c0 < 128; c0 += 32) {
+        uint32_t sv[32], dv[32];
+        tc_ld32(tm_s + lane_base + c0, sv);
+        tc_ld32(tm_dp + lane_base + c0, dv);
+        tc_wait_ld();
+        uint32_t pp[16], dd[16];
+#pragma unroll
+        for (int c = 0; c < 32; c += 2) {
+          float p0 = exp2f(__uint_as_float(sv[c]) * p.scale_log2 - lse2);
+          float p1 = exp2f(__uint_as_float(sv[c + 1]) * p.scale_log2 - lse2);
+          if (diag) { if (c0 + c > r) p0 = 0.f; if (c0 + c + 1 > r) p1 = 0.f; }
+          float d0 = p0 * (__uint_as_float(dv[c]) - Dr);
+          float d1 = p1 * (__uint_as_float(dv[c + 1]) - Dr);
+          __nv_bfloat162 hp = __floats2bfloat162_rn(p0, p1), hd2 = __floats2bfloat162_rn(d0, d1);
+          pp[c >> 1] = *reinterpret_cast<uint32_t*>(&hp);
+          dd[c >> 1] = *reinterpret_cast<uint32_t*>(&hd2);
+        }
+        const int blk = (c0 >> 6) * 16384;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int off = blk + ((((c0 & 63) >> 3) + k) ^ (r & 7)) * 16;
+          *reinterpret_cast<uint4*>(p_row + off) = make_uint4(pp[4 * k], pp[4 * k + 1], pp[4 * k + 2], pp[4 * k + 3]);
+          *reinterpret_cast<uint4*>(ds_row + off) = make_uint4(dd[4 * k], dd[4 * k + 1], dd[4 * k + 2], dd[4 * k + 3]);
+        }
+      }
+      fence_proxy_async();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(3));
+      if (!mbar_wait(bar(4), ph, abort_flag, p.status, 307)) { ok = false; break; }
+      tc_fence_after();
+      float* dq_row = p.dq_acc + tok * d + h * HD;
+#pragma unroll 1
+      for (int c0 = 0; c0 < HD; c0 += 32) {
+        uint32_t v[32];
+        tc_ld32(tm_s + lane_base + c0, v);
+        tc_wait_ld();
+#pragma unroll
+        for (int c = 0; c < 32; c += 4)
+          atomicAdd(reinterpret_cast<float4*>(dq_row + c0 + c),
+                    make_float4(__uint_as_float(v[c]), __uint_as_float(v[c + 1]), __uint_as_float(v[c + 2]),
+                                __uint_as_float(v[c + 3])));
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(5));
+    }
+    if (ok) {
+      // the last wait on barrier 4 covered every MMA: dV and dK of this key tile are final
+      const long long tok = (long long)row0 + kj * 128 + r;
+      bf16* dk_row = p.dqkv + tok * 3 * d + d + h * HD;
+      bf16* dv_row = p.dqkv + tok * 3 * d + 2 * d + h * HD;
+#pragma unroll 1
+      for (int c0 = 0; c0 < HD; c0 += 32) {
+        uint32_t kv[32], vv[32];
+        tc_ld32(tm_dk + lane_base + c0, kv);
+        tc_ld32(tm_dv + lane_base + c0, vv);
+        tc_wait_ld();
+#pragma unroll
+        for (int c = 0; c < 32; c += 8) {
+          uint4 uk, uv;
+          __nv_bfloat162* hk = reinterpret_cast<__nv_bfloat162*>(&uk);
+          __nv_bfloat162* hv = reinterpret_cast<__nv_bfloat162*>(&uv);
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            hk[e] = __floats2bfloat162_rn(__uint_as_float(kv[c + 2 * e]) * p.scale, __uint_as_float(kv[c + 2 * e + 1]) * p.scale);
+            hv[e] = __floats2bfloat162_rn(__uint_as_float(vv[c + 2 * e]), __uint_as_float(vv[c + 2 * e + 1]));
+          }
+          *reinterpret_cast<uint4*>(dk_row + c0 + c) = uk;
+          *reinterpret_cast<uint4*>(dv_row + c0 + c) = uv;
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 4) { tc_fence_after(); tmem_dealloc(tmem, C_::TMEM_COLS); }
+}
+
+// D[b,h,t] = sum_c dO[t,c] * O[t,c] over the head's columns; one warp per (token, head)
+__global__ void attn_rowdot_bf16_kernel(int n_tok, int T, int H, int hd, const bf16* __restrict__ d_o,
+                                        const bf16* __restrict__ o, float* __restrict__ Dv) {
+  const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (gw >= n_tok * H) return;
+  const int tok = gw / H, h = gw % H;
+  const long long off = (long long)tok * H * hd + h * hd;
+  float s = 0.f;
+  for (int c = lane * 2; c < hd; c += 64) {
+    float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(d_o + off + c));
+    float2 bq = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(o + off + c));
+    s += a.x * bq.x + a.y * bq.y;
+  }
+  s = warp_sum(s);
+  if (lane == 0) Dv[((long long)(tok / T) * H + h) * T + (tok % T)] = s;
+}
+
+// dqkv[n, 0:d] = bf16(dq_acc[n, :] * scale)
+__global__ void attn_dq_convert_kernel(long long n_tok, int d, const float* __restrict__ dq_acc, float scale,
+                                       bf16* __restrict__ dqkv) {
+  const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;     // one per 4 elements
+  const long long total = n_tok * d / 4;
+  if (idx >= total) return;
+  const long long e = idx * 4;
+  const long long n = e / d; const int c = (int)(e % d);
+  float4 v = *reinterpret_cast<const float4*>(dq_acc + e);
+  uint2 u;
+  *reinterpret_cast<__nv_bfloat162*>(&u.x) = __floats2bfloat162_rn(v.x * scale, v.y * scale);
+  *reinterpret_cast<__nv_bfloat162*>(&u.y) = __floats2bfloat162_rn(v.z * scale, v.w * scale);
+  *reinterpret_cast<uint2*>(dqkv + n * 3 * d + c) = u;
+}
+
+template <int HD>
+fax_status launch_bwd(fax_ctx* ctx, int B, int T, int H, const void* qkv, const void* o, const float* lse,
+                      const void* d_o, void* dqkv, float* Dv, float* dq_acc) {
+  CUtensorMap mq, md;
+  const uint64_t d = (uint64_t)H * HD;
+  const long long n_tok = (long long)B * T;
+  if (!make_map(ctx, &mq, qkv, 3 * d, (uint64_t)n_tok, 3 * d, 64, 128)) return FAX_ERR_INVALID_ARG;
+  if (!make_map(ctx, &md, d_o, d, (uint64_t)n_tok, d, 64, 128)) return FAX_ERR_INVALID_ARG;
+  FAX_CUDA_TRY(ctx, cudaMemsetAsync(dq_acc, 0, (size_t)n_tok * d * sizeof(float), ctx->stream));
+  {
+    const long long warps = n_tok * H;
+    const int threads = 256;
+    const long long blocks = (warps * 32 + threads - 1) / threads;
+    attn_rowdot_bf16_kernel<<<(unsigned)blocks, threads, 0, ctx->stream>>>((int)n_tok, T, H, HD, (const bf16*)d_o,
+                                                                          (const bf16*)o, Dv);
+    FAX_TRY(fax_after_launch(ctx));
+  }
+  AttnBwdParams p;
+  p.B = B; p.T = T; p.H = H; p.lse = lse; p.Dv = Dv; p.dq_acc = dq_acc; p.dqkv = (bf16*)dqkv;
+  p.scale = 1.0f / sqrtf((float)HD);
+  p.scale_log2 = 1.4426950408889634f * p.scale;
+  p.status = ctx->dev_status;
+  static bool attr_set = false;
+  if (!attr_set) {
+    FAX_CUDA_TRY(ctx, cudaFuncSetAttribute(attn_bwd_tc_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           BwdCfg<HD>::SMEM_BYTES));
+    attr_set = true;
+  }
+  const int grid = B * H * (T / 128);
+  attn_bwd_tc_kernel<HD><<<grid, BWD_THREADS, BwdCfg<HD>::SMEM_BYTES, ctx->stream>>>(mq, md, p);
+  FAX_TRY(fax_after_launch(ctx));
+  const long long quads = n_tok * (long long)d / 4;
+  attn_dq_convert_kernel<<<(unsigned)((quads + 255) / 256), 256, 0, ctx->stream>>>(n_tok, (int)d, dq_acc, p.scale,
+                                                                                  (bf16*)dqkv);
+  return fax_after_launch(ctx);
+}
+
 }  // namespace
 
 bool fax_attention_tc_supported(int B, int T, int H, int hd) {
@@ -259,4 +556,20 @@ fax_status fax_attention_fwd_tc(fax_ctx* ctx, int B, int T, int H, int hd, const
   if (!fax_attention_tc_supported(B, T, H, hd) || !fax_aligned(qkv, 16) || !fax_aligned(o, 16))
     return FAX_ERR_UNSUPPORTED_SHAPE;
   return hd == 64 ? launch_fwd<64>(ctx, B, T, H, qkv, o, lse) : launch_fwd<128>(ctx, B, T, H, qkv, o, lse);
+}
+
+size_t fax_attention_bwd_tc_scratch_bytes(int B, int T, int H, int hd) {
+  return fax_round_up((size_t)B * H * T * sizeof(float), 256) + (size_t)B * T * H * hd * sizeof(float);
+}
+
+fax_status fax_attention_bwd_tc(fax_ctx* ctx, int B, int T, int H, int hd, const void* qkv, const void* o,
+                                const float* lse, const void* d_o, void* dqkv, void* scratch, size_t scratch_bytes) {
+  if (!fax_attention_tc_supported(B, T, H, hd) || !fax_aligned(qkv, 16) || !fax_aligned(o, 16) ||
+      !fax_aligned(d_o, 16) || !fax_aligned(dqkv, 16) || !fax_aligned(scratch, 256))
+    return FAX_ERR_UNSUPPORTED_SHAPE;
+  if (scratch_bytes < fax_attention_bwd_tc_scratch_bytes(B, T, H, hd)) return FAX_ERR_WORKSPACE_TOO_SMALL;
+  float* Dv = (float*)scratch;
+  float* dq_acc = (float*)((char*)scratch + fax_round_up((size_t)B * H * T * sizeof(float), 256));
+  return hd == 64 ? launch_bwd<64>(ctx, B, T, H, qkv, o, lse, d_o, dqkv, Dv, dq_acc)
+                  : launch_bwd<128>(ctx, B, T, H, qkv, o, lse, d_o, dqkv, Dv, dq_acc);
 }

@@ -7,8 +7,12 @@ fax_status fax_gemm(fax_ctx* ctx, int prec, const FaxGemm& g) {
 }
 
 size_t fax_attention_bwd_scratch_bytes(int prec, int B, int T, int H, int hd) {
-  (void)prec; (void)hd;
-  return (size_t)B * H * T * sizeof(float);      // D = rowsum(dO * O)
+  size_t simt = (size_t)B * H * T * sizeof(float);      // D = rowsum(dO * O)
+  if (prec == FAX_PREC_BF16 && fax_attention_tc_supported(B, T, H, hd)) {
+    size_t t = fax_attention_bwd_tc_scratch_bytes(B, T, H, hd);
+    return t > simt ? t : simt;
+  }
+  return simt;
 }
 
 fax_status fax_attention_fwd(fax_ctx* ctx, int prec, int B, int T, int H, int hd, const void* qkv,
@@ -26,5 +30,7 @@ fax_status fax_attention_bwd(fax_ctx* ctx, int prec, int B, int T, int H, int hd
   if (scratch_bytes < (size_t)B * H * T * sizeof(float)) return FAX_ERR_WORKSPACE_TOO_SMALL;
   // causal half of dV, dP, dQ, dK (the recomputed QK^T is not counted)
   FaxProfScope prof(ctx, KC_ATTN_BWD, 4.0 * B * H * (double)T * T * hd, 0.0);
+  if (prec == FAX_PREC_BF16 && fax_attention_tc_supported(B, T, H, hd))
+    return fax_attention_bwd_tc(ctx, B, T, H, hd, qkv, o, lse, d_o, dqkv, scratch, scratch_bytes);
   return fax_attention_bwd_simt(ctx, prec, B, T, H, hd, qkv, o, lse, d_o, dqkv, (float*)scratch);
 }
