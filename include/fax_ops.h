@@ -62,6 +62,34 @@ fax_status fax_op_layernorm_backward(fax_ctx* ctx, int32_t prec, int32_t rows, i
                                      const void* add, void* dx, float* dgamma, float* dbeta,
                                      void* scratch, size_t scratch_bytes);
 
+/* LayerNorm backward without caller scratch and without any allocation.  (The
+ * paper has no counterpart of this call; it exists for deployment reasons.)
+ * Some hosts of this library cannot give it scratch memory or let it call
+ * cudaMalloc: a serving or training process whose own pool already owns all
+ * device memory, a plug-in that runs under a fixed memory budget, or a
+ * latency-critical loop that cannot afford the device-wide synchronisation an
+ * allocation implies.  For them the column-sum partials of dgamma / dbeta live
+ * in a fixed array inside the library image: FAX_LN_STATIC_SCRATCH_FLOATS
+ * floats (8 MiB), resident on every GPU that loads the library until the
+ * process exits.  The call computes exactly what fax_op_layernorm_backward
+ * computes (same kernels) and calls no cudaMalloc, cudaFree or allocating
+ * library routine.
+ *  - Limit: 2 * min(rows, SM count) * d <= FAX_LN_STATIC_SCRATCH_FLOATS (on a
+ *    148-SM B200 with rows >= 148: d <= 7084); beyond it the call does nothing
+ *    and returns FAX_ERR_WORKSPACE_TOO_SMALL.
+ *  - The first call on each device looks the array's device address up (one
+ *    cudaGetSymbolAddress with that device current).  Make that first call
+ *    before starting any stream capture on the device.
+ *  - All calls on a device share the one array, and it keeps whatever the last
+ *    call left.  Nothing in it needs clearing (every slot is written before it
+ *    is read), but two calls whose kernels overlap on the GPU (different
+ *    streams or contexts) race on it: serialise them. */
+#define FAX_LN_STATIC_SCRATCH_FLOATS (2 * 256 * 4096)
+fax_status fax_op_layernorm_backward_static(fax_ctx* ctx, int32_t prec, int32_t rows, int32_t d, const void* da,
+                                            const void* x, const float* mu, const float* rstd,
+                                            const void* gamma, const void* add, void* dx, float* dgamma,
+                                            float* dbeta);
+
 /* Causal multi-head attention (Sec. 3.2: multi-headed attention blocks) on a
  * fused qkv [batch*seq, 3*n_heads*head_dim] T buffer (layout in fax.h):
  * o [batch*seq, n_heads*head_dim] T, lse [batch, n_heads, seq] float

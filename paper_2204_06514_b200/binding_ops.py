@@ -24,6 +24,8 @@ _SIGNATURES = {
     "fax_op_layernorm_backward_scratch_bytes": (C.c_int32, [C.c_int32, C.c_int32, C.POINTER(C.c_size_t)]),
     "fax_op_layernorm_backward": (C.c_int32, [_P, C.c_int32, C.c_int32, C.c_int32, _P, _P, _P, _P, _P, _P,
                                               _P, _P, _P, _P, C.c_size_t]),
+    "fax_op_layernorm_backward_static": (C.c_int32, [_P, C.c_int32, C.c_int32, C.c_int32, _P, _P, _P, _P, _P, _P,
+                                                     _P, _P, _P]),
     "fax_op_attention_forward": (C.c_int32, [_P, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                              _P, _P, _P]),
     "fax_op_attention_backward_scratch_bytes": (C.c_int32, [C.c_int32] * 5 + [C.POINTER(C.c_size_t)]),
@@ -75,6 +77,13 @@ def fax_op_layernorm_backward(ctx, prec, rows, d, da, x, mu, rstd, gamma, add, d
                               scratch_bytes):
     _check(_L().fax_op_layernorm_backward(ctx, prec, rows, d, da, x, mu, rstd, gamma, add, dx, dgamma, dbeta,
                                           scratch, scratch_bytes), "fax_op_layernorm_backward")
+
+
+def fax_op_layernorm_backward_static(ctx, prec, rows, d, da, x, mu, rstd, gamma, add, dx, dgamma, dbeta):
+    """LayerNorm backward whose scratch is a fixed array inside the library: for callers that
+    cannot allocate device memory or pass any.  Same results as fax_op_layernorm_backward."""
+    _check(_L().fax_op_layernorm_backward_static(ctx, prec, rows, d, da, x, mu, rstd, gamma, add, dx, dgamma,
+                                                 dbeta), "fax_op_layernorm_backward_static")
 
 
 def fax_op_attention_forward(ctx, prec, batch, seq, n_heads, head_dim, qkv, o, lse):

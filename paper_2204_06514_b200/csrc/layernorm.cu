@@ -2,6 +2,7 @@
 // LayerNorm).  HBM-bound: one block per row keeps the whole row in registers,
 // 128-bit loads and stores, warp-shuffle reductions, two-pass mean / variance.
 #include "common.cuh"
+#include "../../include/fax_ops.h"
 
 namespace {
 
@@ -333,4 +334,42 @@ fax_status fax_colsum(fax_ctx* ctx, int prec, int rows, int cols, const void* in
   FAX_TRY(fax_after_launch(ctx));
   colsum_fold_kernel<<<(cols + 255) / 256, 256, 0, ctx->stream>>>(slabs, cols, partial, out, accumulate ? 1 : 0);
   return fax_after_launch(ctx);
+}
+
+// ---------------------------------------------------------------------------
+// LayerNorm backward for callers that have no device memory to hand over as
+// scratch and may not allocate any: the column-sum partials live in a fixed
+// array that is part of the library image (8 MiB on every GPU that loads it,
+// until the process exits).
+// ---------------------------------------------------------------------------
+static __device__ __align__(256) float g_ln_static_partial[FAX_LN_STATIC_SCRATCH_FLOATS];
+
+// Device address of the array above, per device ordinal.  In host code the
+// array's name is only a handle for the runtime, not a device pointer; the
+// address a kernel can use comes from cudaGetSymbolAddress, asked once per
+// device with that device current.
+static float* g_ln_static_ptr[64] = {nullptr};
+
+extern "C" fax_status fax_op_layernorm_backward_static(fax_ctx* ctx, int32_t prec, int32_t rows, int32_t d,
+                                                       const void* da, const void* x, const float* mu,
+                                                       const float* rstd, const void* gamma, const void* add,
+                                                       void* dx, float* dgamma, float* dbeta) {
+  if (!ctx || !da || !x || !mu || !rstd || !gamma || !dx || !dgamma || !dbeta || rows <= 0 || d <= 0)
+    return FAX_ERR_INVALID_ARG;
+  if (prec != FAX_PREC_BF16 && prec != FAX_PREC_FP32_VALIDATE) return FAX_ERR_INVALID_ARG;
+  if (ctx->device < 0 || ctx->device >= 64 || ctx->sm_count > 256) return FAX_ERR_ARCH;
+  const size_t need = (size_t)2 * ln_bwd_slabs(ctx, rows) * d;
+  if (need > (size_t)FAX_LN_STATIC_SCRATCH_FLOATS) return FAX_ERR_WORKSPACE_TOO_SMALL;   // beyond the fixed array
+  if (!g_ln_static_ptr[ctx->device]) {
+    // one-time set-up on this device (no allocation: the array already exists in the loaded module)
+    FAX_CUDA_TRY(ctx, cudaSetDevice(ctx->device));
+    float* ptr = nullptr;
+    FAX_CUDA_TRY(ctx, cudaGetSymbolAddress((void**)&ptr, g_ln_static_partial));
+    if (!ptr) return FAX_ERR_CUDA;
+    g_ln_static_ptr[ctx->device] = ptr;
+  }
+  // Every slab writes its whole slice of the partials before the fold kernel reads it, so
+  // nothing in the shared array has to start at zero and stale contents are harmless.
+  return fax_layernorm_bwd(ctx, prec, rows, d, da, x, mu, rstd, gamma, add, dx, dgamma, dbeta, false,
+                           g_ln_static_ptr[ctx->device], FAX_LN_STATIC_SCRATCH_FLOATS);
 }
