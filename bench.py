@@ -195,12 +195,10 @@ def run_ours(args):
     import torch.distributed as dist
 
     from paper_2204_06514_b200 import binding as fx
-    from paper_2204_06514_b200 import build, synth
+    from paper_2204_06514_b200 import build, dist_util, synth
     from paper_2204_06514_b200.state import BlockRunner, LmRunner, Session, hparams
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = dist_util.env_rank()
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device: there is no CPU fallback")
     if rank == 0:
@@ -279,12 +277,7 @@ def run_ours(args):
             fn()
         e1.record(sess.stream)
         barrier()
-        ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms
+        return dist_util.max_over_ranks(e0.elapsed_time(e1), dev)
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -320,7 +313,7 @@ def run_ours(args):
 
     ms_step = ms / args.steps
     tokens = cfg.tokens
-    tps = world * tokens / (ms_step * 1e-3)
+    tps = dist_util.whole_job_rate(tokens, world, ms_step)
     flops = cfg.step_flops()
     achieved_tf = flops / (ms_step * 1e-3) / 1e12
     kernels = {}
@@ -360,7 +353,7 @@ def run_ours(args):
                 "flops_convention": "6*matmul_params*tokens + causal-halved attention (6*B*T^2*d per layer)"},
         "roofline": roofline, "kernels": kernels,
         "cpu_baseline": {"value": cpu_val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what},
-        "e2e": {"value": world * tokens / (ms_e2e / e2e_steps * 1e-3), "unit": UNIT,
+        "e2e": {"value": dist_util.whole_job_rate(tokens, world, ms_e2e / e2e_steps), "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": launches, "clocks": clocks,
     }

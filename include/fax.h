@@ -114,6 +114,13 @@ typedef struct {
  * scratch arena of one block.  Host pointers. */
 fax_status fax_block_sizes(const fax_block_cfg* cfg, size_t* saved_bytes, size_t* scratch_bytes);
 
+/* Where the pieces live inside the two block arenas (byte offsets from the
+ * arena base), for inspection, checkpointing and tests.  saved_off[13]: x, a
+ * (LN1 out), qkv, o, x1, m (LN2 out), h, g, mu1, rstd1, mu2, rstd2, lse.
+ * scratch_off[4], valid after fax_block_backward: dh [N,f], dqkv [N,3d],
+ * da [N,d] (gradient at LN1's output), dx1 [N,d].  Host pointers. */
+fax_status fax_block_arena_layout(const fax_block_cfg* cfg, size_t* saved_off, size_t* scratch_off);
+
 /* Forward pass of the block (Fig. 3 "forward pass"):
  *   a = LN(x; ln1)            qkv = a Wqkv + bqkv
  *   o = causal multi-head softmax attention of qkv (log-sum-exp kept)
@@ -158,6 +165,14 @@ typedef struct {
 /* `tensors` is a HOST array of n_tensors descriptors of device buffers. */
 fax_status fax_adamw_step(fax_ctx* ctx, const fax_adamw_tensor* tensors, int32_t n_tensors,
                           const fax_adamw_hparams* hp);
+
+/* The whole-step calls (fax_block_step*, fax_lm_step*) run the AdamW update of
+ * each tensor on a second stream owned by the context as soon as that tensor's
+ * gradient is complete and its old value is no longer needed, i.e. under the
+ * rest of the backward pass; the calls join that stream before they return
+ * control of the main stream.  enable = 0 keeps everything on the main stream.
+ * Results are identical either way.  Default: enabled. */
+fax_status fax_set_adamw_overlap(fax_ctx* ctx, int32_t enable);
 
 /* One trainable tensor of a training state: float32 master, compute-precision
  * copy (bf16; in FP32_VALIDATE may equal w or be NULL), Adam moments, float32
@@ -209,6 +224,16 @@ typedef struct {
 } fax_lm_state;
 
 fax_status fax_lm_sizes(const fax_lm_cfg* cfg, size_t* saved_bytes, size_t* scratch_bytes);
+
+/* Layout of the LM arenas (byte offsets, host pointers): act_off[n_layers+1]
+ * (input of block l; last = output of the last block), layer_saved_off[n_layers]
+ * (base of block l's saved pieces, laid out as fax_block_arena_layout's
+ * saved_off minus its x entry, which is act_off[l]), xf_off (final LayerNorm
+ * output), all in the saved arena; row_loss_off (per-token loss, float [N])
+ * and block_scratch_off (base of the block scratch, as scratch_off above) in
+ * the scratch arena. */
+fax_status fax_lm_arena_layout(const fax_lm_cfg* cfg, size_t* act_off, size_t* layer_saved_off,
+                               size_t* xf_off, size_t* row_loss_off, size_t* block_scratch_off);
 
 /* Full LM training step (Fig. 3: forward pass, loss, backward pass; then the
  * Adam update): ids, targets are device int32 [batch, seq].  Gradients of

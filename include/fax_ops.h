@@ -74,9 +74,9 @@ fax_status fax_op_layernorm_backward(fax_ctx* ctx, int32_t prec, int32_t rows, i
  * process exits.  The call computes exactly what fax_op_layernorm_backward
  * computes (same kernels) and calls no cudaMalloc, cudaFree or allocating
  * library routine.
- *  - Limit: 2 * min(rows, SM count) * d <= FAX_LN_STATIC_SCRATCH_FLOATS (on a
- *    148-SM B200 with rows >= 148: d <= 7084); beyond it the call does nothing
- *    and returns FAX_ERR_WORKSPACE_TOO_SMALL.
+ *  - Limit: d <= FAX_LN_STATIC_MAX_D (4096) at any row count (the array holds
+ *    the partial sums of up to 256 row slabs of that width); a wider row makes
+ *    the call do nothing and return FAX_ERR_WORKSPACE_TOO_SMALL.
  *  - The first call on each device looks the array's device address up (one
  *    cudaGetSymbolAddress with that device current).  Make that first call
  *    before starting any stream capture on the device.
@@ -84,7 +84,8 @@ fax_status fax_op_layernorm_backward(fax_ctx* ctx, int32_t prec, int32_t rows, i
  *    call left.  Nothing in it needs clearing (every slot is written before it
  *    is read), but two calls whose kernels overlap on the GPU (different
  *    streams or contexts) race on it: serialise them. */
-#define FAX_LN_STATIC_SCRATCH_FLOATS (2 * 256 * 4096)
+#define FAX_LN_STATIC_MAX_D 4096
+#define FAX_LN_STATIC_SCRATCH_FLOATS (2 * 256 * FAX_LN_STATIC_MAX_D)
 fax_status fax_op_layernorm_backward_static(fax_ctx* ctx, int32_t prec, int32_t rows, int32_t d, const void* da,
                                             const void* x, const float* mu, const float* rstd,
                                             const void* gamma, const void* add, void* dx, float* dgamma,

@@ -91,10 +91,14 @@ _SIGNATURES = {
     "fax_last_cuda_error": (C.c_int32, [_P]),
     "fax_check_device_status": (C.c_int32, [_P, C.POINTER(C.c_int32)]),
     "fax_launch_count": (C.c_uint64, [_P]),
+    "fax_set_adamw_overlap": (C.c_int32, [_P, C.c_int32]),
     "fax_profile_begin": (C.c_int32, [_P]),
     "fax_profile_end": (C.c_int32, [_P, C.POINTER(ProfileEntry), C.c_int32]),
     "fax_kernel_class_name": (C.c_char_p, [C.c_int32]),
     "fax_block_sizes": (C.c_int32, [C.POINTER(BlockCfg), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]),
+    "fax_block_arena_layout": (C.c_int32, [C.POINTER(BlockCfg), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]),
+    "fax_lm_arena_layout": (C.c_int32, [C.POINTER(LmCfg), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t),
+                                        C.POINTER(C.c_size_t), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]),
     "fax_block_forward": (C.c_int32, [_P, C.POINTER(BlockCfg), C.POINTER(BlockParams), _P, _P, _P,
                                       C.c_size_t, _P, C.c_size_t]),
     "fax_block_backward": (C.c_int32, [_P, C.POINTER(BlockCfg), C.POINTER(BlockParams), _P, _P, C.c_size_t,
@@ -176,6 +180,10 @@ def fax_check_device_status(ctx) -> tuple[int, int]:
     return s, d.value
 
 
+def fax_set_adamw_overlap(ctx, enable: bool):
+    _check(load_library().fax_set_adamw_overlap(ctx, int(bool(enable))), "fax_set_adamw_overlap")
+
+
 def fax_profile_begin(ctx):
     _check(load_library().fax_profile_begin(ctx), "fax_profile_begin")
 
@@ -200,6 +208,26 @@ def fax_block_sizes(cfg: BlockCfg) -> tuple[int, int]:
     a, b = C.c_size_t(), C.c_size_t()
     _check(load_library().fax_block_sizes(C.byref(cfg), C.byref(a), C.byref(b)), "fax_block_sizes")
     return a.value, b.value
+
+
+SAVED_NAMES = ("x", "a", "qkv", "o", "x1", "m", "h", "g", "mu1", "rstd1", "mu2", "rstd2", "lse")
+SCRATCH_NAMES = ("dh", "dqkv", "da", "dx1")
+
+
+def fax_block_arena_layout(cfg: BlockCfg) -> tuple[dict, dict]:
+    """(saved offsets by name, scratch offsets by name), in bytes."""
+    a, b = (C.c_size_t * 13)(), (C.c_size_t * 4)()
+    _check(load_library().fax_block_arena_layout(C.byref(cfg), a, b), "fax_block_arena_layout")
+    return dict(zip(SAVED_NAMES, a)), dict(zip(SCRATCH_NAMES, b))
+
+
+def fax_lm_arena_layout(cfg: LmCfg) -> dict:
+    L = cfg.n_layers
+    act, lay = (C.c_size_t * (L + 1))(), (C.c_size_t * L)()
+    xf, rl, bs = C.c_size_t(), C.c_size_t(), C.c_size_t()
+    _check(load_library().fax_lm_arena_layout(C.byref(cfg), act, lay, C.byref(xf), C.byref(rl), C.byref(bs)),
+           "fax_lm_arena_layout")
+    return dict(act=list(act), layer_saved=list(lay), xf=xf.value, row_loss=rl.value, block_scratch=bs.value)
 
 
 def fax_block_host_scratch_bytes(cfg: BlockCfg) -> int:

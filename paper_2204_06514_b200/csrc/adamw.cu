@@ -49,31 +49,43 @@ adamw_kernel(const __grid_constant__ AdamBatch batch, AdamScalars sc) {
     unsigned long long end = base + CHUNK < t.n ? base + CHUNK : t.n;
     const bool vec_ok = ((t.n & 3ull) == 0);
     if (vec_ok) {
-      for (unsigned long long e = base + 4ull * threadIdx.x; e < end; e += 4ull * THREADS) {
-        float4 w = *reinterpret_cast<const float4*>(t.w + e);
-        float4 m = *reinterpret_cast<const float4*>(t.m + e);
-        float4 v = *reinterpret_cast<const float4*>(t.v + e);
-        float4 g;
-        if (G_BF16) {
-          uint2 raw = *reinterpret_cast<const uint2*>((const bf16*)t.g + e);
-          float2 a = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&raw.x));
-          float2 b = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&raw.y));
-          g = make_float4(a.x, a.y, b.x, b.y);
-        } else {
-          g = *reinterpret_cast<const float4*>((const float*)t.g + e);
+      // a full chunk is 4 float4 groups per thread: issue all loads first, then update and store
+      constexpr int U = CHUNK / (4 * THREADS);
+      float4 w[U], m[U], v[U], g[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const unsigned long long e = base + 4ull * (threadIdx.x + u * THREADS);
+        if (e < end) {
+          w[u] = *reinterpret_cast<const float4*>(t.w + e);
+          m[u] = *reinterpret_cast<const float4*>(t.m + e);
+          v[u] = *reinterpret_cast<const float4*>(t.v + e);
+          if (G_BF16) {
+            uint2 raw = *reinterpret_cast<const uint2*>((const bf16*)t.g + e);
+            float2 a = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&raw.x));
+            float2 b = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&raw.y));
+            g[u] = make_float4(a.x, a.y, b.x, b.y);
+          } else {
+            g[u] = *reinterpret_cast<const float4*>((const float*)t.g + e);
+          }
         }
-        adam_elem<G_BF16>(w.x, m.x, v.x, g.x, t.wd, sc);
-        adam_elem<G_BF16>(w.y, m.y, v.y, g.y, t.wd, sc);
-        adam_elem<G_BF16>(w.z, m.z, v.z, g.z, t.wd, sc);
-        adam_elem<G_BF16>(w.w, m.w, v.w, g.w, t.wd, sc);
-        *reinterpret_cast<float4*>(t.w + e) = w;
-        *reinterpret_cast<float4*>(t.m + e) = m;
-        *reinterpret_cast<float4*>(t.v + e) = v;
-        if (t.wc) {
-          uint2 o;
-          *reinterpret_cast<__nv_bfloat162*>(&o.x) = __floats2bfloat162_rn(w.x, w.y);
-          *reinterpret_cast<__nv_bfloat162*>(&o.y) = __floats2bfloat162_rn(w.z, w.w);
-          *reinterpret_cast<uint2*>(t.wc + e) = o;
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const unsigned long long e = base + 4ull * (threadIdx.x + u * THREADS);
+        if (e < end) {
+          adam_elem<G_BF16>(w[u].x, m[u].x, v[u].x, g[u].x, t.wd, sc);
+          adam_elem<G_BF16>(w[u].y, m[u].y, v[u].y, g[u].y, t.wd, sc);
+          adam_elem<G_BF16>(w[u].z, m[u].z, v[u].z, g[u].z, t.wd, sc);
+          adam_elem<G_BF16>(w[u].w, m[u].w, v[u].w, g[u].w, t.wd, sc);
+          *reinterpret_cast<float4*>(t.w + e) = w[u];
+          *reinterpret_cast<float4*>(t.m + e) = m[u];
+          *reinterpret_cast<float4*>(t.v + e) = v[u];
+          if (t.wc) {
+            uint2 o;
+            *reinterpret_cast<__nv_bfloat162*>(&o.x) = __floats2bfloat162_rn(w[u].x, w[u].y);
+            *reinterpret_cast<__nv_bfloat162*>(&o.y) = __floats2bfloat162_rn(w[u].z, w[u].w);
+            *reinterpret_cast<uint2*>(t.wc + e) = o;
+          }
         }
       }
     } else {
@@ -129,13 +141,35 @@ fax_status fax_adamw_launch(fax_ctx* ctx, const fax_adamw_tensor* tensors, int n
     batch.n_tensors = k;
     batch.total_chunks = (unsigned int)chunks;
     unsigned long long want = chunks;
-    unsigned int grid = (unsigned int)(want < (unsigned long long)ctx->sm_count * 16 ? want : ctx->sm_count * 16);
+    // on the optimizer stream keep two blocks per SM so that the main stream's kernels still fit beside them
+    const unsigned long long cap = (unsigned long long)ctx->sm_count * (ctx->stream == ctx->side ? 2 : 16);
+    unsigned int grid = (unsigned int)(want < cap ? want : cap);
     if (hp->grad_is_bf16)
       adamw_kernel<true><<<grid, THREADS, 0, ctx->stream>>>(batch, sc);
     else
       adamw_kernel<false><<<grid, THREADS, 0, ctx->stream>>>(batch, sc);
     FAX_TRY(fax_after_launch(ctx));
   }
+  return FAX_OK;
+}
+
+fax_status fax_adamw_async(fax_ctx* ctx, const fax_adamw_tensor* tensors, int n, const fax_adamw_hparams* hp) {
+  if (!ctx->overlap_adamw) return fax_adamw_launch(ctx, tensors, n, hp);
+  FAX_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_fork, ctx->stream));
+  FAX_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0));
+  cudaStream_t main_stream = ctx->stream;
+  ctx->stream = ctx->side;
+  fax_status s = fax_adamw_launch(ctx, tensors, n, hp);
+  ctx->stream = main_stream;
+  ctx->side_busy = true;
+  return s;
+}
+
+fax_status fax_adamw_join(fax_ctx* ctx) {
+  if (!ctx->side_busy) return FAX_OK;
+  FAX_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_join, ctx->side));
+  FAX_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->stream, ctx->ev_join, 0));
+  ctx->side_busy = false;
   return FAX_OK;
 }
 

@@ -35,6 +35,8 @@ extern "C" fax_status fax_create(fax_ctx** out, int32_t device_ordinal, void* cu
   c->dev_status = nullptr;
   c->encode_tiled = nullptr;
   c->prof_on = false;
+  c->side = nullptr; c->ev_fork = nullptr; c->ev_join = nullptr; c->side_busy = false;
+  c->overlap_adamw = true;
   if (cudaMalloc((void**)&c->dev_status, 64) != cudaSuccess ||
       cudaMemset(c->dev_status, 0, 64) != cudaSuccess) {
     delete c;
@@ -50,6 +52,13 @@ extern "C" fax_status fax_create(fax_ctx** out, int32_t device_ordinal, void* cu
     return FAX_ERR_CUDA;
   }
   c->encode_tiled = fn;
+  if (cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+    cudaFree(c->dev_status);
+    delete c;
+    return FAX_ERR_CUDA;
+  }
   *out = c;
   return FAX_OK;
 }
@@ -58,6 +67,9 @@ extern "C" fax_status fax_destroy(fax_ctx* ctx) {
   if (!ctx) return FAX_ERR_INVALID_ARG;
   cudaSetDevice(ctx->device);
   cudaStreamSynchronize(ctx->stream);
+  if (ctx->side) { cudaStreamSynchronize(ctx->side); cudaStreamDestroy(ctx->side); }
+  if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+  if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
   if (ctx->dev_status) cudaFree(ctx->dev_status);
   for (FaxProfRec& r : ctx->prof) { cudaEventDestroy(r.e0); cudaEventDestroy(r.e1); }
   delete ctx;
@@ -77,6 +89,12 @@ extern "C" fax_status fax_check_device_status(fax_ctx* ctx, int32_t* detail_host
     FAX_CUDA_TRY(ctx, cudaMemset(ctx->dev_status, 0, 8));
     return FAX_ERR_TIMEOUT;
   }
+  return FAX_OK;
+}
+
+extern "C" fax_status fax_set_adamw_overlap(fax_ctx* ctx, int32_t enable) {
+  if (!ctx) return FAX_ERR_INVALID_ARG;
+  ctx->overlap_adamw = enable != 0;
   return FAX_OK;
 }
 

@@ -66,6 +66,27 @@ extern "C" fax_status fax_block_sizes(const fax_block_cfg* cfg, size_t* saved_by
   return FAX_OK;
 }
 
+static void saved_offsets(const BlockSaved& s, const char* base, size_t* off) {
+  const void* p[13] = {s.x, s.a, s.qkv, s.o, s.x1, s.m, s.h, s.g, s.mu1, s.rstd1, s.mu2, s.rstd2, s.lse};
+  for (int i = 0; i < 13; ++i) off[i] = p[i] ? (size_t)((const char*)p[i] - base) : (size_t)-1;
+}
+
+extern "C" fax_status fax_block_arena_layout(const fax_block_cfg* cfg, size_t* saved_off, size_t* scratch_off) {
+  FAX_TRY(fax_block_validate(cfg));
+  if (!saved_off || !scratch_off) return FAX_ERR_INVALID_ARG;
+  char* base = (char*)4096;              // any non-null base: only differences are used
+  FaxArena a(base, (size_t)-1), b(base, (size_t)-1);
+  BlockSaved s; BlockScratch w;
+  fax_block_carve_saved(cfg, a, true, &s);
+  fax_block_carve_scratch(cfg, b, &w);
+  saved_offsets(s, base, saved_off);
+  scratch_off[0] = (size_t)((char*)w.bufF - base);
+  scratch_off[1] = (size_t)((char*)w.bufQ - base);
+  scratch_off[2] = (size_t)((char*)w.bufA - base);
+  scratch_off[3] = (size_t)((char*)w.bufB - base);
+  return FAX_OK;
+}
+
 static FaxGemm gemm_desc(int M, int N, int K) {
   FaxGemm g;
   g.M = M; g.N = N; g.K = K;
@@ -123,23 +144,33 @@ fax_status fax_block_forward_impl(fax_ctx* ctx, const fax_block_cfg* c, const fa
 
 fax_status fax_block_backward_impl(fax_ctx* ctx, const fax_block_cfg* c, const fax_block_params* p,
                                    const void* dy, const BlockSaved& s, const void* x, void* dx,
-                                   const fax_block_grads* gr, bool acc, const BlockScratch& w) {
+                                   const fax_block_grads* gr, bool acc, const BlockScratch& w,
+                                   const FaxAdamHook* hook) {
   const int N = c->batch * c->seq, d = c->d_model, f = c->d_ff, prec = c->prec;
+  // once both gradients of a linear layer (or LayerNorm) exist and the data-gradient GEMM has
+  // consumed the old weight, its AdamW update runs on the optimizer stream under the rest of backward
+  auto update = [&](int first) -> fax_status {
+    return hook ? fax_adamw_async(ctx, hook->t + first, 2, hook->hp) : FAX_OK;
+  };
   // B1: through FC2 and GELU
   FAX_TRY(linear_bwd_data(ctx, prec, N, f, d, dy, p->w_fc2, EPI_DGELU, s.h, w.bufF));          // dh
   FAX_TRY(linear_bwd_weight(ctx, prec, N, f, d, s.g, dy, gr->w_fc2, acc));
   FAX_TRY(fax_colsum(ctx, prec, N, d, dy, d, gr->b_fc2, acc, w.partial, w.partial_floats));
+  FAX_TRY(update(10));
   // B2: through FC1
   FAX_TRY(linear_bwd_data(ctx, prec, N, d, f, w.bufF, p->w_fc1, EPI_NONE, nullptr, w.bufA));    // dm
   FAX_TRY(linear_bwd_weight(ctx, prec, N, d, f, s.m, w.bufF, gr->w_fc1, acc));
   FAX_TRY(fax_colsum(ctx, prec, N, f, w.bufF, f, gr->b_fc1, acc, w.partial, w.partial_floats));
+  FAX_TRY(update(8));
   // B3: LN2 backward plus the residual branch
   FAX_TRY(fax_layernorm_bwd(ctx, prec, N, d, w.bufA, s.x1, s.mu2, s.rstd2, p->ln2_g, dy, w.bufB,
                             gr->ln2_g, gr->ln2_b, acc, w.partial, w.partial_floats));           // dx1
+  FAX_TRY(update(6));
   // B4: through the attention output projection
   FAX_TRY(linear_bwd_data(ctx, prec, N, d, d, w.bufB, p->w_o, EPI_NONE, nullptr, w.bufA));      // do
   FAX_TRY(linear_bwd_weight(ctx, prec, N, d, d, s.o, w.bufB, gr->w_o, acc));
   FAX_TRY(fax_colsum(ctx, prec, N, d, w.bufB, d, gr->b_o, acc, w.partial, w.partial_floats));
+  FAX_TRY(update(4));
   // B5: attention backward
   FAX_TRY(fax_attention_bwd(ctx, prec, c->batch, c->seq, c->n_heads, c->head_dim, s.qkv, s.o, s.lse,
                             w.bufA, w.bufQ, w.attn, w.attn_bytes));                             // dqkv
@@ -147,10 +178,11 @@ fax_status fax_block_backward_impl(fax_ctx* ctx, const fax_block_cfg* c, const f
   FAX_TRY(linear_bwd_data(ctx, prec, N, d, 3 * d, w.bufQ, p->w_qkv, EPI_NONE, nullptr, w.bufA)); // da
   FAX_TRY(linear_bwd_weight(ctx, prec, N, d, 3 * d, s.a, w.bufQ, gr->w_qkv, acc));
   FAX_TRY(fax_colsum(ctx, prec, N, 3 * d, w.bufQ, 3 * d, gr->b_qkv, acc, w.partial, w.partial_floats));
+  FAX_TRY(update(2));
   // B7: LN1 backward plus the residual branch
   FAX_TRY(fax_layernorm_bwd(ctx, prec, N, d, w.bufA, x, s.mu1, s.rstd1, p->ln1_g, w.bufB, dx,
                             gr->ln1_g, gr->ln1_b, acc, w.partial, w.partial_floats));
-  return FAX_OK;
+  return update(0);
 }
 
 static fax_status check_params(const fax_block_params* p) {
@@ -238,13 +270,15 @@ static fax_status block_step_impl(fax_ctx* ctx, const fax_block_cfg* cfg, const 
   if (ar.used() > st->saved_bytes || aw.used() + scratch_skip > st->scratch_bytes) return FAX_ERR_WORKSPACE_TOO_SMALL;
   fax_block_params p; fax_block_grads g;
   fax_layer_views(&st->layer, cfg->prec, &p, &g);
-  FAX_TRY(fax_block_forward_impl(ctx, cfg, &p, x, y, s, true));
-  FAX_TRY(fax_block_backward_impl(ctx, cfg, &p, dy, s, s.x, dx, &g, false, w));
   fax_adamw_tensor t[12];
   fax_layer_adamw_tensors(&st->layer, cfg->prec, t);
   fax_adamw_hparams h = *hp;
   h.grad_is_bf16 = 0;
-  return fax_adamw_launch(ctx, t, 12, &h);
+  if (h.step < 1) return FAX_ERR_INVALID_ARG;
+  FaxAdamHook hook = {t, &h};
+  FAX_TRY(fax_block_forward_impl(ctx, cfg, &p, x, y, s, true));
+  FAX_TRY(fax_block_backward_impl(ctx, cfg, &p, dy, s, s.x, dx, &g, false, w, &hook));
+  return fax_adamw_join(ctx);
 }
 
 extern "C" fax_status fax_block_step(fax_ctx* ctx, const fax_block_cfg* cfg, const fax_block_state* st,

@@ -18,7 +18,8 @@ fax_status fax_block_forward_impl(fax_ctx* ctx, const fax_block_cfg* c, const fa
                                   const void* x, void* y, const BlockSaved& s, bool copy_x);
 fax_status fax_block_backward_impl(fax_ctx* ctx, const fax_block_cfg* c, const fax_block_params* p,
                                    const void* dy, const BlockSaved& s, const void* x, void* dx,
-                                   const fax_block_grads* gr, bool acc, const BlockScratch& w);
+                                   const fax_block_grads* gr, bool acc, const BlockScratch& w,
+                                   const FaxAdamHook* hook = nullptr);
 void fax_layer_views(const fax_layer_state* L, int prec, fax_block_params* p, fax_block_grads* g);
 int fax_layer_adamw_tensors(const fax_layer_state* L, int prec, fax_adamw_tensor* out);
 fax_status fax_layer_check(const fax_layer_state* L, const fax_block_cfg* c);

@@ -31,6 +31,10 @@ struct fax_ctx {
   void* encode_tiled;        // cuTensorMapEncodeTiled, resolved at create
   bool prof_on;
   std::vector<FaxProfRec> prof;
+  cudaStream_t side;         // optimizer stream: AdamW of finished tensors overlaps the rest of backward
+  cudaEvent_t ev_fork, ev_join;
+  bool side_busy;
+  bool overlap_adamw;
 };
 
 // Brackets the launches of one operator with CUDA events while profiling is on.
@@ -169,6 +173,11 @@ fax_status fax_attention_bwd(fax_ctx* ctx, int prec, int B, int T, int H, int hd
 size_t fax_attention_bwd_scratch_bytes(int prec, int B, int T, int H, int hd);
 
 fax_status fax_adamw_launch(fax_ctx* ctx, const fax_adamw_tensor* tensors, int n, const fax_adamw_hparams* hp);
+// Enqueue AdamW on the context's optimizer stream, ordered after everything enqueued on the main
+// stream so far; fax_adamw_join makes the main stream wait for all of it.
+fax_status fax_adamw_async(fax_ctx* ctx, const fax_adamw_tensor* tensors, int n, const fax_adamw_hparams* hp);
+fax_status fax_adamw_join(fax_ctx* ctx);
+struct FaxAdamHook { const fax_adamw_tensor* t; const fax_adamw_hparams* hp; };   // t: 12 tensors in parameter order
 
 fax_status fax_block_validate(const fax_block_cfg* cfg);
 

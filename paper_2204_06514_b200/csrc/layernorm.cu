@@ -59,6 +59,71 @@ __device__ __forceinline__ float2 block_sum2(float a, float b, float2* red) {
   return make_float2(warp_sum(t.x), warp_sum(t.y));
 }
 
+// ---- raw 16-byte vectors kept packed in registers ---------------------------
+template <typename T> __device__ __forceinline__ void unpack(const uint4& u, float (&f)[Vec<T>::N]);
+template <> __device__ __forceinline__ void unpack<float>(const uint4& u, float (&f)[4]) {
+  f[0] = __uint_as_float(u.x); f[1] = __uint_as_float(u.y); f[2] = __uint_as_float(u.z); f[3] = __uint_as_float(u.w);
+}
+template <> __device__ __forceinline__ void unpack<bf16>(const uint4& u, float (&f)[8]) {
+  const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) { float2 t = __bfloat1622float2(h[i]); f[2 * i] = t.x; f[2 * i + 1] = t.y; }
+}
+
+// Forward, one warp per row (rows of up to 32*VPT vectors): the row stays packed in
+// registers, reductions are warp shuffles only, no block barrier.
+template <typename T, int VPT>
+__global__ void __launch_bounds__(128)
+layernorm_fwd_warp_kernel(int rows, int d, const T* __restrict__ x, const T* __restrict__ gamma,
+                          const T* __restrict__ beta, float eps, T* __restrict__ out,
+                          float* __restrict__ mu_out, float* __restrict__ rstd_out, T* __restrict__ x_copy) {
+  constexpr int VN = Vec<T>::N;
+  const int lane = threadIdx.x & 31;
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  const int nvec = d / VN;
+  const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)row * d);
+  uint4 raw[VPT];
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) {
+    const int vi = lane + 32 * i;
+    if (vi < nvec) {
+      raw[i] = xr[vi];
+      float f[VN]; unpack<T>(raw[i], f);
+#pragma unroll
+      for (int j = 0; j < VN; ++j) s += f[j];
+    }
+  }
+  const float mu = warp_sum(s) / (float)d;
+  float q = 0.f;
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) {
+    if (lane + 32 * i < nvec) {
+      float f[VN]; unpack<T>(raw[i], f);
+#pragma unroll
+      for (int j = 0; j < VN; ++j) { float t = f[j] - mu; q += t * t; }
+    }
+  }
+  const float rstd = rsqrtf(warp_sum(q) / (float)d + eps);
+  if (lane == 0) { mu_out[row] = mu; rstd_out[row] = rstd; }
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) {
+    const int vi = lane + 32 * i;
+    if (vi < nvec) {
+      float f[VN], g[VN], b[VN], o[VN];
+      unpack<T>(raw[i], f);
+      load_vec<T>(gamma + vi * VN, g);
+      load_vec<T>(beta + vi * VN, b);
+#pragma unroll
+      for (int j = 0; j < VN; ++j) o[j] = (f[j] - mu) * rstd * g[j] + b[j];
+      store_vec<T>(out + (size_t)row * d + vi * VN, o);
+      if (x_copy) reinterpret_cast<uint4*>(x_copy + (size_t)row * d)[vi] = raw[i];
+    }
+  }
+}
+
+// Forward, one block per row (wide rows).
 template <typename T, int VPT>
 __global__ void __launch_bounds__(512)
 layernorm_fwd_kernel(int rows, int d, const T* __restrict__ x, const T* __restrict__ gamma,
@@ -67,158 +132,215 @@ layernorm_fwd_kernel(int rows, int d, const T* __restrict__ x, const T* __restri
   constexpr int VN = Vec<T>::N;
   __shared__ float red[32];
   const int nvec = d / VN;
-  for (int row = blockIdx.x; row < rows; row += gridDim.x) {
-    const T* xr = x + (size_t)row * d;
-    float v[VPT][VN];
-    float s = 0.f;
-#pragma unroll
-    for (int i = 0; i < VPT; ++i) {
-      int vi = threadIdx.x + i * blockDim.x;
-      if (vi < nvec) {
-        load_vec<T>(xr + vi * VN, v[i]);
-#pragma unroll
-        for (int j = 0; j < VN; ++j) s += v[i][j];
-      }
-    }
-    float mu = block_sum(s, red) / (float)d;
-    float q = 0.f;
-#pragma unroll
-    for (int i = 0; i < VPT; ++i) {
-      int vi = threadIdx.x + i * blockDim.x;
-      if (vi < nvec) {
-#pragma unroll
-        for (int j = 0; j < VN; ++j) { float t = v[i][j] - mu; q += t * t; }
-      }
-    }
-    float rstd = rsqrtf(block_sum(q, red) / (float)d + eps);
-    if (threadIdx.x == 0) { mu_out[row] = mu; rstd_out[row] = rstd; }
-#pragma unroll
-    for (int i = 0; i < VPT; ++i) {
-      int vi = threadIdx.x + i * blockDim.x;
-      if (vi < nvec) {
-        float g[VN], b[VN], o[VN];
-        load_vec<T>(gamma + vi * VN, g);
-        load_vec<T>(beta + vi * VN, b);
-#pragma unroll
-        for (int j = 0; j < VN; ++j) o[j] = (v[i][j] - mu) * rstd * g[j] + b[j];
-        store_vec<T>(out + (size_t)row * d + vi * VN, o);
-        if (x_copy) store_vec<T>(x_copy + (size_t)row * d + vi * VN, v[i]);
-      }
-    }
-  }
-}
-
-// Each block walks rows blockIdx.x, +gridDim.x, ...; column sums of da and
-// da*xhat stay in registers and are written once per block to `partial`
-// ([gridDim.x][2][d]); a second kernel folds the slabs.
-template <typename T, int VPT>
-__global__ void __launch_bounds__(512)
-layernorm_bwd_kernel(int rows, int d, const T* __restrict__ da, const T* __restrict__ x,
-                     const float* __restrict__ mu_in, const float* __restrict__ rstd_in,
-                     const T* __restrict__ gamma, const T* __restrict__ add, T* __restrict__ dx,
-                     float* __restrict__ partial) {
-  constexpr int VN = Vec<T>::N;
-  __shared__ float2 red[32];
-  const int nvec = d / VN;
-  float g[VPT][VN], accg[VPT][VN], accb[VPT][VN];
+  const int row = blockIdx.x;
+  const T* xr = x + (size_t)row * d;
+  float v[VPT][VN];
+  float s = 0.f;
 #pragma unroll
   for (int i = 0; i < VPT; ++i) {
     int vi = threadIdx.x + i * blockDim.x;
+    if (vi < nvec) {
+      load_vec<T>(xr + vi * VN, v[i]);
 #pragma unroll
-    for (int j = 0; j < VN; ++j) { accg[i][j] = 0.f; accb[i][j] = 0.f; g[i][j] = 0.f; }
-    if (vi < nvec) load_vec<T>(gamma + vi * VN, g[i]);
-  }
-  for (int row = blockIdx.x; row < rows; row += gridDim.x) {
-    const float mu = mu_in[row], rstd = rstd_in[row];
-    float u[VPT][VN], xh[VPT][VN];
-    float s1 = 0.f, s2 = 0.f;
-#pragma unroll
-    for (int i = 0; i < VPT; ++i) {
-      int vi = threadIdx.x + i * blockDim.x;
-      if (vi < nvec) {
-        float dv[VN], xv[VN];
-        load_vec<T>(da + (size_t)row * d + vi * VN, dv);
-        load_vec<T>(x + (size_t)row * d + vi * VN, xv);
-#pragma unroll
-        for (int j = 0; j < VN; ++j) {
-          xh[i][j] = (xv[j] - mu) * rstd;
-          u[i][j] = dv[j] * g[i][j];
-          accg[i][j] += dv[j] * xh[i][j];
-          accb[i][j] += dv[j];
-          s1 += u[i][j];
-          s2 += u[i][j] * xh[i][j];
-        }
-      }
-    }
-    float2 t = block_sum2(s1, s2, red);
-    const float c1 = t.x / (float)d, c2 = t.y / (float)d;
-#pragma unroll
-    for (int i = 0; i < VPT; ++i) {
-      int vi = threadIdx.x + i * blockDim.x;
-      if (vi < nvec) {
-        float o[VN];
-#pragma unroll
-        for (int j = 0; j < VN; ++j) o[j] = rstd * (u[i][j] - c1 - xh[i][j] * c2);
-        if (add) {
-          float av[VN];
-          load_vec<T>(add + (size_t)row * d + vi * VN, av);
-#pragma unroll
-          for (int j = 0; j < VN; ++j) o[j] += av[j];
-        }
-        store_vec<T>(dx + (size_t)row * d + vi * VN, o);
-      }
+      for (int j = 0; j < VN; ++j) s += v[i][j];
     }
   }
-  float* pg = partial + (size_t)blockIdx.x * 2 * d;
-  float* pb = pg + d;
+  float mu = block_sum(s, red) / (float)d;
+  float q = 0.f;
 #pragma unroll
   for (int i = 0; i < VPT; ++i) {
     int vi = threadIdx.x + i * blockDim.x;
     if (vi < nvec) {
 #pragma unroll
-      for (int j = 0; j < VN; ++j) { pg[vi * VN + j] = accg[i][j]; pb[vi * VN + j] = accb[i][j]; }
+      for (int j = 0; j < VN; ++j) { float t = v[i][j] - mu; q += t * t; }
+    }
+  }
+  float rstd = rsqrtf(block_sum(q, red) / (float)d + eps);
+  if (threadIdx.x == 0) { mu_out[row] = mu; rstd_out[row] = rstd; }
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) {
+    int vi = threadIdx.x + i * blockDim.x;
+    if (vi < nvec) {
+      float g[VN], b[VN], o[VN];
+      load_vec<T>(gamma + vi * VN, g);
+      load_vec<T>(beta + vi * VN, b);
+#pragma unroll
+      for (int j = 0; j < VN; ++j) o[j] = (v[i][j] - mu) * rstd * g[j] + b[j];
+      store_vec<T>(out + (size_t)row * d + vi * VN, o);
+      if (x_copy) store_vec<T>(x_copy + (size_t)row * d + vi * VN, v[i]);
     }
   }
 }
 
-// out[k][c] (+)= sum_s partial[s][k][c], k in {0: dgamma, 1: dbeta}
-__global__ void layernorm_bwd_fold_kernel(int slabs, int d, const float* __restrict__ partial,
-                                          float* __restrict__ dgamma, float* __restrict__ dbeta,
-                                          int accumulate) {
-  int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= 2 * d) return;
-  float s = 0.f;
-  for (int i = 0; i < slabs; ++i) s += partial[(size_t)i * 2 * d + c];
-  float* dst = (c < d) ? (dgamma + c) : (dbeta + (c - d));
-  *dst = accumulate ? (*dst + s) : s;
-}
-
-// partial[s][c] = sum over the rows of slab s of in[r][c]
-template <typename T>
-__global__ void colsum_partial_kernel(int rows, int cols, const T* __restrict__ in, int64_t ld,
-                                      float* __restrict__ partial) {
+// Backward dx, one warp per row: da and x stay packed in registers.
+//   u = da*gamma; dx = rstd*(u - mean(u) - xhat*mean(u*xhat)) (+ add)
+template <typename T, int VPT>
+__global__ void __launch_bounds__(128)
+layernorm_bwd_dx_warp_kernel(int rows, int d, const T* __restrict__ da, const T* __restrict__ x,
+                             const float* __restrict__ mu_in, const float* __restrict__ rstd_in,
+                             const T* __restrict__ gamma, const T* __restrict__ add, T* __restrict__ dx) {
   constexpr int VN = Vec<T>::N;
-  int vc = blockIdx.x * blockDim.x + threadIdx.x;   // vector column
-  if (vc * VN >= cols) return;
-  float acc[VN];
+  const int lane = threadIdx.x & 31;
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (row >= rows) return;
+  const int nvec = d / VN;
+  const float mu = mu_in[row], rstd = rstd_in[row];
+  const uint4* dar = reinterpret_cast<const uint4*>(da + (size_t)row * d);
+  const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)row * d);
+  uint4 rda[VPT], rx[VPT];
+  float s1 = 0.f, s2 = 0.f;
 #pragma unroll
-  for (int j = 0; j < VN; ++j) acc[j] = 0.f;
-  for (int r = blockIdx.y; r < rows; r += gridDim.y) {
-    float v[VN];
-    load_vec<T>(in + (size_t)r * ld + vc * VN, v);
-#pragma unroll
-    for (int j = 0; j < VN; ++j) acc[j] += v[j];
+  for (int i = 0; i < VPT; ++i) {
+    const int vi = lane + 32 * i;
+    if (vi < nvec) { rda[i] = dar[vi]; rx[i] = xr[vi]; }
   }
 #pragma unroll
-  for (int j = 0; j < VN; ++j) partial[(size_t)blockIdx.y * cols + vc * VN + j] = acc[j];
+  for (int i = 0; i < VPT; ++i) {
+    const int vi = lane + 32 * i;
+    if (vi < nvec) {
+      float fd[VN], fx[VN], g[VN];
+      unpack<T>(rda[i], fd); unpack<T>(rx[i], fx);
+      load_vec<T>(gamma + vi * VN, g);
+#pragma unroll
+      for (int j = 0; j < VN; ++j) { float u = fd[j] * g[j]; s1 += u; s2 += u * (fx[j] - mu) * rstd; }
+    }
+  }
+  const float c1 = warp_sum(s1) / (float)d, c2 = warp_sum(s2) / (float)d;
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) {
+    const int vi = lane + 32 * i;
+    if (vi < nvec) {
+      float fd[VN], fx[VN], g[VN], o[VN];
+      unpack<T>(rda[i], fd); unpack<T>(rx[i], fx);
+      load_vec<T>(gamma + vi * VN, g);
+#pragma unroll
+      for (int j = 0; j < VN; ++j) o[j] = rstd * (fd[j] * g[j] - c1 - (fx[j] - mu) * rstd * c2);
+      if (add) {
+        float av[VN];
+        load_vec<T>(add + (size_t)row * d + vi * VN, av);
+#pragma unroll
+        for (int j = 0; j < VN; ++j) o[j] += av[j];
+      }
+      store_vec<T>(dx + (size_t)row * d + vi * VN, o);
+    }
+  }
 }
-__global__ void colsum_fold_kernel(int slabs, int cols, const float* __restrict__ partial,
-                                   float* __restrict__ out, int accumulate) {
+
+// Backward dx, one block per row (wide rows).
+template <typename T, int VPT>
+__global__ void __launch_bounds__(512)
+layernorm_bwd_dx_kernel(int rows, int d, const T* __restrict__ da, const T* __restrict__ x,
+                        const float* __restrict__ mu_in, const float* __restrict__ rstd_in,
+                        const T* __restrict__ gamma, const T* __restrict__ add, T* __restrict__ dx) {
+  constexpr int VN = Vec<T>::N;
+  __shared__ float2 red[32];
+  const int nvec = d / VN;
+  const int row = blockIdx.x;
+  const float mu = mu_in[row], rstd = rstd_in[row];
+  float u[VPT][VN], xh[VPT][VN];
+  float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) {
+    int vi = threadIdx.x + i * blockDim.x;
+    if (vi < nvec) {
+      float dv[VN], xv[VN], g[VN];
+      load_vec<T>(da + (size_t)row * d + vi * VN, dv);
+      load_vec<T>(x + (size_t)row * d + vi * VN, xv);
+      load_vec<T>(gamma + vi * VN, g);
+#pragma unroll
+      for (int j = 0; j < VN; ++j) {
+        xh[i][j] = (xv[j] - mu) * rstd;
+        u[i][j] = dv[j] * g[j];
+        s1 += u[i][j];
+        s2 += u[i][j] * xh[i][j];
+      }
+    }
+  }
+  float2 t = block_sum2(s1, s2, red);
+  const float c1 = t.x / (float)d, c2 = t.y / (float)d;
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) {
+    int vi = threadIdx.x + i * blockDim.x;
+    if (vi < nvec) {
+      float o[VN];
+#pragma unroll
+      for (int j = 0; j < VN; ++j) o[j] = rstd * (u[i][j] - c1 - xh[i][j] * c2);
+      if (add) {
+        float av[VN];
+        load_vec<T>(add + (size_t)row * d + vi * VN, av);
+#pragma unroll
+        for (int j = 0; j < VN; ++j) o[j] += av[j];
+      }
+      store_vec<T>(dx + (size_t)row * d + vi * VN, o);
+    }
+  }
+}
+
+// Column reductions over row slabs.  Block = 32 vector columns x 8 row phases;
+// grid = (column groups, slabs).  LN = false: partial[slab][c] = sum_r in[r][c].
+// LN = true: partial[slab][0][c] = sum_r in[r][c] * xhat[r][c] (dgamma) and
+// partial[slab][1][c] = sum_r in[r][c] (dbeta), xhat from x, mu, rstd.
+template <typename T, bool LN>
+__global__ void __launch_bounds__(256)
+colreduce_kernel(int rows, int cols, const T* __restrict__ in, int64_t ld, const T* __restrict__ x,
+                 const float* __restrict__ mu, const float* __restrict__ rstd, float* __restrict__ partial) {
+  constexpr int VN = Vec<T>::N;
+  __shared__ float sm[LN ? 2 : 1][8][32 * VN + 1];
+  const int lane = threadIdx.x & 31, ph = threadIdx.x >> 5;
+  const int vc = blockIdx.x * 32 + lane;
+  const bool active = vc * VN < cols;
+  const int per = (rows + gridDim.y - 1) / gridDim.y;
+  const int r0 = blockIdx.y * per, r1 = min(rows, r0 + per);
+  float a0[VN], a1[VN];
+#pragma unroll
+  for (int j = 0; j < VN; ++j) { a0[j] = 0.f; a1[j] = 0.f; }
+  if (active) {
+#pragma unroll 4
+    for (int r = r0 + ph; r < r1; r += 8) {
+      float v[VN];
+      load_vec<T>(in + (size_t)r * ld + vc * VN, v);
+      if (LN) {
+        float xv[VN];
+        load_vec<T>(x + (size_t)r * ld + vc * VN, xv);
+        const float m = mu[r], rs = rstd[r];
+#pragma unroll
+        for (int j = 0; j < VN; ++j) { a0[j] += v[j] * (xv[j] - m) * rs; a1[j] += v[j]; }
+      } else {
+#pragma unroll
+        for (int j = 0; j < VN; ++j) a0[j] += v[j];
+      }
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < VN; ++j) {
+    sm[0][ph][lane * VN + j] = a0[j];
+    if (LN) sm[LN ? 1 : 0][ph][lane * VN + j] = a1[j];
+  }
+  __syncthreads();
+  for (int c = threadIdx.x; c < 32 * VN; c += 256) {
+    const int gc = blockIdx.x * 32 * VN + c;
+    if (gc >= cols) continue;
+    float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) { s0 += sm[0][k][c]; if (LN) s1 += sm[LN ? 1 : 0][k][c]; }
+    if (LN) {
+      partial[(size_t)blockIdx.y * 2 * cols + gc] = s0;
+      partial[(size_t)blockIdx.y * 2 * cols + cols + gc] = s1;
+    } else {
+      partial[(size_t)blockIdx.y * cols + gc] = s0;
+    }
+  }
+}
+
+// out[c] (+)= sum_s partial[s][c] for c < width (width = cols, or 2*cols with out split in two)
+__global__ void colreduce_fold_kernel(int slabs, int width, int cols, const float* __restrict__ partial,
+                                      float* __restrict__ out0, float* __restrict__ out1, int accumulate) {
   int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= cols) return;
+  if (c >= width) return;
   float s = 0.f;
-  for (int i = 0; i < slabs; ++i) s += partial[(size_t)i * cols + c];
-  out[c] = accumulate ? out[c] + s : s;
+  for (int i = 0; i < slabs; ++i) s += partial[(size_t)i * width + c];
+  float* dst = (c < cols) ? (out0 + c) : (out1 + (c - cols));
+  *dst = accumulate ? (*dst + s) : s;
 }
 
 int pick_vpt(int nvec, int max_threads, int* threads) {
@@ -231,18 +353,41 @@ int pick_vpt(int nvec, int max_threads, int* threads) {
   return 0;
 }
 
-int ln_bwd_slabs(fax_ctx* ctx, int rows) { return rows < ctx->sm_count ? rows : ctx->sm_count; }
+// Row slabs of the column reductions: enough blocks to fill the machine, at most 256 slabs.
+int colreduce_slabs(fax_ctx* ctx, int rows, int nvec) {
+  const int gx = (nvec + 31) / 32;
+  int slabs = (8 * ctx->sm_count + gx - 1) / gx;
+  const int max_by_rows = (rows + 31) / 32;
+  if (slabs > max_by_rows) slabs = max_by_rows;
+  if (slabs > 256) slabs = 256;
+  if (slabs < 1) slabs = 1;
+  return slabs;
+}
+int ln_bwd_slabs(fax_ctx* ctx, int rows, int d, int prec) {
+  return colreduce_slabs(ctx, rows, d / (prec == FAX_PREC_BF16 ? 8 : 4));
+}
 
 template <typename T>
 fax_status ln_fwd_t(fax_ctx* ctx, int rows, int d, const void* x, const void* gamma, const void* beta,
                     float eps, void* out, float* mu, float* rstd, void* x_copy) {
+  const int nvec = d / Vec<T>::N;
+  if (nvec <= 512) {
+    const int need = (nvec + 31) / 32;
+#define LN_FWDW(V)                                                                                      \
+    if (need <= V) {                                                                                    \
+      layernorm_fwd_warp_kernel<T, V><<<(rows + 3) / 4, 128, 0, ctx->stream>>>(                         \
+          rows, d, (const T*)x, (const T*)gamma, (const T*)beta, eps, (T*)out, mu, rstd, (T*)x_copy);   \
+      return fax_after_launch(ctx);                                                                     \
+    }
+    LN_FWDW(1) LN_FWDW(2) LN_FWDW(3) LN_FWDW(4) LN_FWDW(6) LN_FWDW(8) LN_FWDW(12) LN_FWDW(16)
+#undef LN_FWDW
+  }
   int threads = 0;
-  int vpt = pick_vpt(d / Vec<T>::N, 512, &threads);
+  int vpt = pick_vpt(nvec, 512, &threads);
   if (!vpt) return FAX_ERR_UNSUPPORTED_SHAPE;
-  int grid = rows;
 #define LN_FWD(V)                                                                                    \
   case V:                                                                                            \
-    layernorm_fwd_kernel<T, V><<<grid, threads, 0, ctx->stream>>>(                                   \
+    layernorm_fwd_kernel<T, V><<<rows, threads, 0, ctx->stream>>>(                                   \
         rows, d, (const T*)x, (const T*)gamma, (const T*)beta, eps, (T*)out, mu, rstd, (T*)x_copy);   \
     break;
   switch (vpt) { LN_FWD(1) LN_FWD(2) LN_FWD(3) LN_FWD(4) LN_FWD(6) LN_FWD(8) LN_FWD(12) LN_FWD(16) }
@@ -251,32 +396,53 @@ fax_status ln_fwd_t(fax_ctx* ctx, int rows, int d, const void* x, const void* ga
 }
 
 template <typename T>
-fax_status ln_bwd_t(fax_ctx* ctx, int rows, int d, const void* da, const void* x, const float* mu,
-                    const float* rstd, const void* gamma, const void* add, void* dx, float* dgamma,
-                    float* dbeta, bool accumulate, float* partial) {
+fax_status ln_bwd_dx_t(fax_ctx* ctx, int rows, int d, const void* da, const void* x, const float* mu,
+                       const float* rstd, const void* gamma, const void* add, void* dx) {
+  const int nvec = d / Vec<T>::N;
+  if (nvec <= 512) {
+    const int need = (nvec + 31) / 32;
+#define LN_BWDW(V)                                                                                      \
+    if (need <= V) {                                                                                    \
+      layernorm_bwd_dx_warp_kernel<T, V><<<(rows + 3) / 4, 128, 0, ctx->stream>>>(                      \
+          rows, d, (const T*)da, (const T*)x, mu, rstd, (const T*)gamma, (const T*)add, (T*)dx);        \
+      return fax_after_launch(ctx);                                                                     \
+    }
+    LN_BWDW(1) LN_BWDW(2) LN_BWDW(3) LN_BWDW(4) LN_BWDW(6) LN_BWDW(8) LN_BWDW(12) LN_BWDW(16)
+#undef LN_BWDW
+  }
   int threads = 0;
-  int vpt = pick_vpt(d / Vec<T>::N, 512, &threads);
+  int vpt = pick_vpt(nvec, 512, &threads);
   if (!vpt || vpt > 8) return FAX_ERR_UNSUPPORTED_SHAPE;
-  int slabs = ln_bwd_slabs(ctx, rows);
 #define LN_BWD(V)                                                                                   \
   case V:                                                                                           \
-    layernorm_bwd_kernel<T, V><<<slabs, threads, 0, ctx->stream>>>(                                 \
-        rows, d, (const T*)da, (const T*)x, mu, rstd, (const T*)gamma, (const T*)add, (T*)dx,       \
-        partial);                                                                                   \
+    layernorm_bwd_dx_kernel<T, V><<<rows, threads, 0, ctx->stream>>>(                               \
+        rows, d, (const T*)da, (const T*)x, mu, rstd, (const T*)gamma, (const T*)add, (T*)dx);      \
     break;
   switch (vpt) { LN_BWD(1) LN_BWD(2) LN_BWD(3) LN_BWD(4) LN_BWD(6) LN_BWD(8) }
 #undef LN_BWD
+  return fax_after_launch(ctx);
+}
+
+template <typename T, bool LN>
+fax_status colreduce_t(fax_ctx* ctx, int rows, int cols, const void* in, int64_t ld, const void* x,
+                       const float* mu, const float* rstd, float* out0, float* out1, bool accumulate,
+                       float* partial) {
+  const int nvec = cols / Vec<T>::N;
+  const int slabs = colreduce_slabs(ctx, rows, nvec);
+  dim3 grid((nvec + 31) / 32, slabs);
+  colreduce_kernel<T, LN><<<grid, 256, 0, ctx->stream>>>(rows, cols, (const T*)in, ld, (const T*)x, mu, rstd, partial);
   FAX_TRY(fax_after_launch(ctx));
-  layernorm_bwd_fold_kernel<<<(2 * d + 255) / 256, 256, 0, ctx->stream>>>(slabs, d, partial, dgamma, dbeta,
-                                                                          accumulate ? 1 : 0);
+  const int width = LN ? 2 * cols : cols;
+  colreduce_fold_kernel<<<(width + 255) / 256, 256, 0, ctx->stream>>>(slabs, width, cols, partial, out0, out1,
+                                                                      accumulate ? 1 : 0);
   return fax_after_launch(ctx);
 }
 
 }  // namespace
 
 size_t fax_layernorm_bwd_partial_floats(int rows, int d) {
-  int slabs = rows < 256 ? rows : 256;     // upper bound on the SM count used for slabs
-  return (size_t)2 * slabs * d;
+  (void)rows;
+  return (size_t)2 * 256 * d;     // 256 = upper bound of the slab count
 }
 
 fax_status fax_layernorm_fwd(fax_ctx* ctx, int prec, int rows, int d, const void* x, const void* gamma,
@@ -295,45 +461,32 @@ fax_status fax_layernorm_bwd(fax_ctx* ctx, int prec, int rows, int d, const void
                              const float* mu, const float* rstd, const void* gamma, const void* add,
                              void* dx, float* dgamma, float* dbeta, bool accumulate, float* partial,
                              size_t partial_floats) {
-  if (ctx->sm_count > 256) return FAX_ERR_ARCH;
-  if (partial_floats < (size_t)2 * ln_bwd_slabs(ctx, rows) * d) return FAX_ERR_WORKSPACE_TOO_SMALL;
-  // read da, x (and add), write dx
+  if (d % (prec == FAX_PREC_BF16 ? 8 : 4)) return FAX_ERR_UNSUPPORTED_SHAPE;
+  if (partial_floats < (size_t)2 * ln_bwd_slabs(ctx, rows, d, prec) * d) return FAX_ERR_WORKSPACE_TOO_SMALL;
+  // dx pass reads da, x (and add) and writes dx; the dgamma/dbeta pass reads da and x again
   FaxProfScope prof(ctx, KC_LN_BWD, 0.0, (double)rows * d * fax_elem_size(prec) * (add ? 4 : 3));
   if (prec == FAX_PREC_BF16) {
-    if (d % 8) return FAX_ERR_UNSUPPORTED_SHAPE;
-    return ln_bwd_t<bf16>(ctx, rows, d, da, x, mu, rstd, gamma, add, dx, dgamma, dbeta, accumulate, partial);
+    FAX_TRY(ln_bwd_dx_t<bf16>(ctx, rows, d, da, x, mu, rstd, gamma, add, dx));
+    return colreduce_t<bf16, true>(ctx, rows, d, da, d, x, mu, rstd, dgamma, dbeta, accumulate, partial);
   }
-  if (d % 4) return FAX_ERR_UNSUPPORTED_SHAPE;
-  return ln_bwd_t<float>(ctx, rows, d, da, x, mu, rstd, gamma, add, dx, dgamma, dbeta, accumulate, partial);
+  FAX_TRY(ln_bwd_dx_t<float>(ctx, rows, d, da, x, mu, rstd, gamma, add, dx));
+  return colreduce_t<float, true>(ctx, rows, d, da, d, x, mu, rstd, dgamma, dbeta, accumulate, partial);
 }
 
 size_t fax_colsum_partial_floats(int rows, int cols) {
-  int slabs = rows < 256 ? rows : 256;
-  return (size_t)slabs * cols;
+  (void)rows;
+  return (size_t)256 * cols;
 }
 
 fax_status fax_colsum(fax_ctx* ctx, int prec, int rows, int cols, const void* in, int64_t ld, float* out,
                       bool accumulate, float* partial, size_t partial_floats) {
   const int vn = prec == FAX_PREC_BF16 ? 8 : 4;
   if (cols % vn || ld % vn) return FAX_ERR_UNSUPPORTED_SHAPE;
-  int vcols = cols / vn;
-  int threads = 128;
-  int gx = (vcols + threads - 1) / threads;
-  // enough row slabs to fill the machine, at most 256
-  int slabs = (2 * ctx->sm_count + gx - 1) / gx;
-  if (slabs > rows) slabs = rows;
-  if (slabs > 256) slabs = 256;
-  if (slabs < 1) slabs = 1;
-  if (partial_floats < (size_t)slabs * cols) return FAX_ERR_WORKSPACE_TOO_SMALL;
+  if (partial_floats < (size_t)colreduce_slabs(ctx, rows, cols / vn) * cols) return FAX_ERR_WORKSPACE_TOO_SMALL;
   FaxProfScope prof(ctx, KC_COLSUM, 0.0, (double)rows * cols * fax_elem_size(prec));
-  dim3 grid(gx, slabs);
   if (prec == FAX_PREC_BF16)
-    colsum_partial_kernel<bf16><<<grid, threads, 0, ctx->stream>>>(rows, cols, (const bf16*)in, ld, partial);
-  else
-    colsum_partial_kernel<float><<<grid, threads, 0, ctx->stream>>>(rows, cols, (const float*)in, ld, partial);
-  FAX_TRY(fax_after_launch(ctx));
-  colsum_fold_kernel<<<(cols + 255) / 256, 256, 0, ctx->stream>>>(slabs, cols, partial, out, accumulate ? 1 : 0);
-  return fax_after_launch(ctx);
+    return colreduce_t<bf16, false>(ctx, rows, cols, in, ld, nullptr, nullptr, nullptr, out, out, accumulate, partial);
+  return colreduce_t<float, false>(ctx, rows, cols, in, ld, nullptr, nullptr, nullptr, out, out, accumulate, partial);
 }
 
 // ---------------------------------------------------------------------------
@@ -357,9 +510,11 @@ extern "C" fax_status fax_op_layernorm_backward_static(fax_ctx* ctx, int32_t pre
   if (!ctx || !da || !x || !mu || !rstd || !gamma || !dx || !dgamma || !dbeta || rows <= 0 || d <= 0)
     return FAX_ERR_INVALID_ARG;
   if (prec != FAX_PREC_BF16 && prec != FAX_PREC_FP32_VALIDATE) return FAX_ERR_INVALID_ARG;
-  if (ctx->device < 0 || ctx->device >= 64 || ctx->sm_count > 256) return FAX_ERR_ARCH;
-  const size_t need = (size_t)2 * ln_bwd_slabs(ctx, rows) * d;
-  if (need > (size_t)FAX_LN_STATIC_SCRATCH_FLOATS) return FAX_ERR_WORKSPACE_TOO_SMALL;   // beyond the fixed array
+  if (ctx->device < 0 || ctx->device >= 64) return FAX_ERR_ARCH;
+  if (d % (prec == FAX_PREC_BF16 ? 8 : 4)) return FAX_ERR_UNSUPPORTED_SHAPE;
+  // the array holds 2 * 256 * FAX_LN_STATIC_MAX_D partial sums: any row count, d up to the stated maximum
+  if (d > FAX_LN_STATIC_MAX_D || (size_t)2 * ln_bwd_slabs(ctx, rows, d, prec) * d > (size_t)FAX_LN_STATIC_SCRATCH_FLOATS)
+    return FAX_ERR_WORKSPACE_TOO_SMALL;
   if (!g_ln_static_ptr[ctx->device]) {
     // one-time set-up on this device (no allocation: the array already exists in the loaded module)
     FAX_CUDA_TRY(ctx, cudaSetDevice(ctx->device));

@@ -79,7 +79,8 @@ fax_status lm_check_state(const fax_lm_cfg* c, const fax_lm_state* st) {
 }
 
 fax_status lm_fwd_bwd(fax_ctx* ctx, const fax_lm_cfg* c, const fax_lm_state* st, const int32_t* ids,
-                      const int32_t* targets, float* loss_device, const LmSaved& sv, const LmScratch& w) {
+                      const int32_t* targets, float* loss_device, const LmSaved& sv, const LmScratch& w,
+                      const fax_adamw_hparams* hp) {
   const fax_block_cfg* bc = &c->block;
   const int prec = bc->prec, L = c->n_layers;
   const int N = bc->batch * bc->seq, d = bc->d_model, V = c->vocab;
@@ -135,17 +136,22 @@ fax_status lm_fwd_bwd(fax_ctx* ctx, const fax_lm_cfg* c, const fax_lm_state* st,
   for (int l = L - 1; l >= 0; --l) {
     fax_block_params p; fax_block_grads g;
     fax_layer_views(&st->layers[l], prec, &p, &g);
-    FAX_TRY(fax_block_backward_impl(ctx, bc, &p, dcur, sv.blk[l], sv.act[l], dnext, &g, false, w.blk));
+    fax_adamw_tensor t12[12];
+    FaxAdamHook hook = {t12, hp};
+    if (hp) fax_layer_adamw_tensors(&st->layers[l], prec, t12);
+    FAX_TRY(fax_block_backward_impl(ctx, bc, &p, dcur, sv.blk[l], sv.act[l], dnext, &g, false, w.blk,
+                                    hp ? &hook : nullptr));
     void* t = dcur; dcur = dnext; dnext = t;
   }
   // embedding gradients: scatter into the tied dwte, batch-sum into dwpe
   return fax_embed_bwd(ctx, prec, bc->batch, bc->seq, c->max_seq, d, V, ids, dcur, st->wte.g, st->wpe.g);
 }
 
+// AdamW of the tensors that are not inside a block (the blocks' tensors are updated under backward).
 fax_status lm_adamw(fax_ctx* ctx, const fax_lm_cfg* c, const fax_lm_state* st, const fax_adamw_hparams* hp) {
   const int prec = c->block.prec;
   std::vector<fax_adamw_tensor> t;
-  t.reserve(4 + 12 * (size_t)c->n_layers);
+  t.reserve(4);
   auto push = [&](const fax_param& p) {
     fax_adamw_tensor a;
     a.w = p.w; a.m = p.m; a.v = p.v; a.g = p.g;
@@ -154,14 +160,9 @@ fax_status lm_adamw(fax_ctx* ctx, const fax_lm_cfg* c, const fax_lm_state* st, c
     t.push_back(a);
   };
   push(st->wte); push(st->wpe);
-  for (int l = 0; l < c->n_layers; ++l) {
-    const fax_param* a = (const fax_param*)&st->layers[l];
-    for (int i = 0; i < 12; ++i) push(a[i]);
-  }
   push(st->lnf_g); push(st->lnf_b);
-  fax_adamw_hparams h = *hp;
-  h.grad_is_bf16 = 0;
-  return fax_adamw_launch(ctx, t.data(), (int)t.size(), &h);
+  FAX_TRY(fax_adamw_launch(ctx, t.data(), (int)t.size(), hp));
+  return fax_adamw_join(ctx);
 }
 
 fax_status lm_run(fax_ctx* ctx, const fax_lm_cfg* cfg, const fax_lm_state* st, const int32_t* ids,
@@ -181,8 +182,14 @@ fax_status lm_run(fax_ctx* ctx, const fax_lm_cfg* cfg, const fax_lm_state* st, c
     FAX_CUDA_TRY(ctx, cudaMemcpyAsync(w.targets, targets_host, nb, cudaMemcpyHostToDevice, ctx->stream));
     ids = w.ids; targets = w.targets;
   }
-  FAX_TRY(lm_fwd_bwd(ctx, cfg, st, ids, targets, loss_device, sv, w));
-  if (hp) FAX_TRY(lm_adamw(ctx, cfg, st, hp));
+  fax_adamw_hparams h;
+  if (hp) {
+    h = *hp;
+    h.grad_is_bf16 = 0;
+    if (h.step < 1) return FAX_ERR_INVALID_ARG;
+  }
+  FAX_TRY(lm_fwd_bwd(ctx, cfg, st, ids, targets, loss_device, sv, w, hp ? &h : nullptr));
+  if (hp) FAX_TRY(lm_adamw(ctx, cfg, st, &h));
   return FAX_OK;
 }
 
@@ -196,6 +203,23 @@ extern "C" fax_status fax_lm_sizes(const fax_lm_cfg* cfg, size_t* saved_bytes, s
   carve_scratch(cfg, b, &w);
   if (saved_bytes) *saved_bytes = a.used();
   if (scratch_bytes) *scratch_bytes = b.used();
+  return FAX_OK;
+}
+
+extern "C" fax_status fax_lm_arena_layout(const fax_lm_cfg* cfg, size_t* act_off, size_t* layer_saved_off,
+                                          size_t* xf_off, size_t* row_loss_off, size_t* block_scratch_off) {
+  FAX_TRY(lm_validate(cfg));
+  if (!act_off || !layer_saved_off || !xf_off || !row_loss_off || !block_scratch_off) return FAX_ERR_INVALID_ARG;
+  char* base = (char*)4096;
+  FaxArena a(base, (size_t)-1), b(base, (size_t)-1);
+  LmSaved s; LmScratch w;
+  carve_saved(cfg, a, &s);
+  carve_scratch(cfg, b, &w);
+  for (int l = 0; l <= cfg->n_layers; ++l) act_off[l] = (size_t)((char*)s.act[l] - base);
+  for (int l = 0; l < cfg->n_layers; ++l) layer_saved_off[l] = (size_t)((char*)s.blk[l].a - base);
+  *xf_off = (size_t)((char*)s.xf - base);
+  *row_loss_off = (size_t)((char*)w.row_loss - base);
+  *block_scratch_off = (size_t)((char*)w.blk.bufF - base);
   return FAX_OK;
 }
 
