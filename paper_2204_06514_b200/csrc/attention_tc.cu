@@ -20,7 +20,7 @@ using namespace tc;
 
 constexpr int TQ = 128;            // queries per CTA
 constexpr int TK = 128;            // keys per tile
-constexpr int FWD_THREADS = 160;   // 4 row warps + 1 driver warp
+constexpr int FWD_THREADS = 192;   // 4 row warps + MMA warp + TMA warp
 
 struct AttnFwdParams {
   int B, T, H;
@@ -37,8 +37,8 @@ template <int HD> struct FwdCfg {
   static constexpr int V_OFF = 3 * TILE_BYTES;          // 2 buffers
   static constexpr int P_OFF = 5 * TILE_BYTES;
   static constexpr int BAR_OFF = P_OFF + P_BYTES;
-  static constexpr int SMEM_BYTES = BAR_OFF + 128 + 1024;
-  static constexpr int TMEM_COLS = 256;                 // S: 128 columns, O: HD columns
+  static constexpr int SMEM_BYTES = BAR_OFF + 256 + 1024;
+  static constexpr int TMEM_COLS = 512;                 // S0 [0,128), S1 [128,256), O [256, 256+HD)
 };
 
 // Load a 128-row x HD-column tile as HD/64 boxes of 64 columns (16 KB each).
@@ -49,6 +49,11 @@ __device__ __forceinline__ void load_tile(uint32_t dst, const CUtensorMap* map, 
   for (int i = 0; i < HD / 64; ++i) tma_load_2d(dst + i * 16384, map, bar, col + 64 * i, row);
 }
 
+// Forward.  S for tile j+1 and j+2 is issued ahead, so the row threads always find
+// their next scores ready while the tensor core runs P V of the tile before; O
+// accumulates in tensor memory and is rescaled only when a row maximum has grown by
+// more than 2^8 since the value the accumulator is expressed in (the decision is
+// taken per warp, because tensor-memory loads and stores are warp-collective).
 template <int HD>
 __global__ void __launch_bounds__(FWD_THREADS, 1)
 attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnFwdParams p) {
@@ -58,10 +63,10 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnFwdParams
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* gbase = smem_raw + (base - raw);
   const uint32_t bars = base + C_::BAR_OFF;
-  // barriers: 0 Q, 1-2 K[2], 3-4 V[2], 5 S, 6 P, 7 O
+  // barriers: 0 Q | 1,2 K full | 3,4 K empty | 5,6 V full | 7,8 V empty | 9,10 S full | 11 P ready | 12 O done
   auto bar = [&](int i) { return bars + 8u * i; };
-  volatile uint32_t* tmem_slot = (volatile uint32_t*)(gbase + C_::BAR_OFF + 64);
-  volatile int* abort_flag = (volatile int*)(gbase + C_::BAR_OFF + 68);
+  volatile uint32_t* tmem_slot = (volatile uint32_t*)(gbase + C_::BAR_OFF + 128);
+  volatile int* abort_flag = (volatile int*)(gbase + C_::BAR_OFF + 132);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nq = p.T / TQ;
@@ -75,7 +80,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnFwdParams
   const int qcol = h * HD, kcol = d + h * HD, vcol = 2 * d + h * HD;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < 8; ++i) mbar_init(bar(i), i == 6 ? 4u : 1u);
+    for (int i = 0; i < 13; ++i) mbar_init(bar(i), i == 11 ? 4u : 1u);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap) : "memory");
@@ -85,143 +90,164 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnFwdParams
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t tmem_s = tmem, tmem_o = tmem + 128;
+  const uint32_t tmem_o = tmem + 256;
+  const uint32_t q_s = base + C_::Q_OFF, p_s = base + C_::P_OFF;
+  auto k_s = [&](int i) { return base + C_::K_OFF + i * C_::TILE_BYTES; };
+  auto v_s = [&](int i) { return base + C_::V_OFF + i * C_::TILE_BYTES; };
 
-  if (warp == 4) {
+  if (warp == 5) {
+    // ---------------- TMA producer ----------------
     if (lane == 0) {
-      const uint32_t q_s = base + C_::Q_OFF, p_s = base + C_::P_OFF;
-      auto k_s = [&](int i) { return base + C_::K_OFF + i * C_::TILE_BYTES; };
-      auto v_s = [&](int i) { return base + C_::V_OFF + i * C_::TILE_BYTES; };
-      const uint32_t idesc_s = idesc_bf16(TK, false, false);
-      const uint32_t idesc_o = idesc_bf16(HD, false, true);
-      auto mma_s = [&](int buf) {
-#pragma unroll
-        for (int s = 0; s < HD / 16; ++s) {
-          const uint32_t off = (s / 4) * 16384 + (s % 4) * 32;
-          tc_mma_bf16(tmem_s, smem_desc(q_s + off, 16, 1024), smem_desc(k_s(buf) + off, 16, 1024), idesc_s, s ? 1u : 0u);
-        }
-        tc_commit(bar(5));
-      };
       load_tile<HD>(q_s, &tmap, bar(0), qcol, row0 + qi * TQ);
-      load_tile<HD>(k_s(0), &tmap, bar(1), kcol, row0);
-      load_tile<HD>(v_s(0), &tmap, bar(3), vcol, row0);
-      if (nkv > 1) {
-        load_tile<HD>(k_s(1), &tmap, bar(2), kcol, row0 + TK);
-        load_tile<HD>(v_s(1), &tmap, bar(4), vcol, row0 + TK);
-      }
-      bool ok = mbar_wait(bar(0), 0, abort_flag, p.status, 201) && mbar_wait(bar(1), 0, abort_flag, p.status, 202);
-      if (ok) { tc_fence_after(); mma_s(0); }
+      bool ok = true;
       for (int j = 0; j < nkv && ok; ++j) {
-        const int buf = j & 1;
-        const uint32_t ring_phase = (uint32_t)((j >> 1) & 1);
-        if (!mbar_wait(bar(6), j & 1, abort_flag, p.status, 203)) { ok = false; break; }       // P_j ready
-        if (!mbar_wait(bar(3 + buf), ring_phase, abort_flag, p.status, 204)) { ok = false; break; }
-        tc_fence_after();
-#pragma unroll
-        for (int s = 0; s < TK / 16; ++s) {
-          const uint64_t ad = smem_desc(p_s + (s / 4) * 16384 + (s % 4) * 32, 16, 1024);
-          const uint64_t bd = smem_desc(v_s(buf) + s * 2048, 16384, 1024);
-          tc_mma_bf16(tmem_o, ad, bd, idesc_o, s ? 1u : 0u);
-        }
-        tc_commit(bar(7));
-        if (j + 1 < nkv) {
-          if (!mbar_wait(bar(1 + (buf ^ 1)), (uint32_t)(((j + 1) >> 1) & 1), abort_flag, p.status, 205)) { ok = false; break; }
-          tc_fence_after();
-          mma_s(buf ^ 1);
-        }
-        if (j + 2 < nkv) {
-          // K[buf] was consumed by S_j (complete before P_j was signalled); V[buf] is free once O_j is done
-          load_tile<HD>(k_s(buf), &tmap, bar(1 + buf), kcol, row0 + (j + 2) * TK);
-          if (!mbar_wait(bar(7), j & 1, abort_flag, p.status, 206)) { ok = false; break; }
-          load_tile<HD>(v_s(buf), &tmap, bar(3 + buf), vcol, row0 + (j + 2) * TK);
-        }
+        const int s = j & 1;
+        const uint32_t ph = (uint32_t)((j >> 1) & 1);
+        if (!mbar_wait(bar(3 + s), ph ^ 1u, abort_flag, p.status, 201)) { ok = false; break; }
+        load_tile<HD>(k_s(s), &tmap, bar(1 + s), kcol, row0 + j * TK);
+        if (!mbar_wait(bar(7 + s), ph ^ 1u, abort_flag, p.status, 202)) { ok = false; break; }
+        load_tile<HD>(v_s(s), &tmap, bar(5 + s), vcol, row0 + j * TK);
       }
       if (!ok) { const long long t0 = clock64(); while (clock64() - t0 < 2000000LL) { } }
+    }
+  } else if (warp == 4) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      const uint32_t idesc_s = idesc_bf16(TK, false, false);
+      const uint32_t idesc_o = idesc_bf16(HD, false, true);
+      bool ok = mbar_wait(bar(0), 0, abort_flag, p.status, 203);
+      auto issue_s = [&](int j) -> bool {
+        const int s = j & 1;
+        if (!mbar_wait(bar(1 + s), (uint32_t)((j >> 1) & 1), abort_flag, p.status, 204)) return false;
+        tc_fence_after();
+#pragma unroll
+        for (int k = 0; k < HD / 16; ++k) {
+          const uint32_t off = (k / 4) * 16384 + (k % 4) * 32;
+          tc_mma_bf16(tmem + (uint32_t)(s * 128), smem_desc(q_s + off, 16, 1024), smem_desc(k_s(s) + off, 16, 1024),
+                      idesc_s, k ? 1u : 0u);
+        }
+        tc_commit(bar(3 + s));      // K buffer free
+        tc_commit(bar(9 + s));      // S ready
+        return true;
+      };
+      if (ok) ok = issue_s(0);
+      if (ok && nkv > 1) ok = issue_s(1);
+      for (int j = 0; j < nkv && ok; ++j) {
+        const int s = j & 1;
+        if (!mbar_wait(bar(11), (uint32_t)(j & 1), abort_flag, p.status, 205)) { ok = false; break; }
+        if (!mbar_wait(bar(5 + s), (uint32_t)((j >> 1) & 1), abort_flag, p.status, 206)) { ok = false; break; }
+        tc_fence_after();
+#pragma unroll
+        for (int k = 0; k < TK / 16; ++k) {
+          const uint64_t ad = smem_desc(p_s + (k / 4) * 16384 + (k % 4) * 32, 16, 1024);
+          const uint64_t bd = smem_desc(v_s(s) + k * 2048, 16384, 1024);
+          tc_mma_bf16(tmem_o, ad, bd, idesc_o, (j | k) ? 1u : 0u);
+        }
+        tc_commit(bar(7 + s));      // V buffer free
+        tc_commit(bar(12));         // O_j accumulated, P buffer free
+        if (j + 2 < nkv) ok = issue_s(j + 2);   // S buffer s was consumed before P_j was signalled
+      }
     }
   } else {
     // ---- row threads: online softmax, one query row each ----
     const int r = 32 * warp + lane;
     const uint32_t lane_base = (uint32_t)(32 * warp) << 16;
     uint8_t* p_row = gbase + C_::P_OFF + r * 128;
-    float m = -INFINITY, l = 0.f;
-    float o[HD];
-#pragma unroll
-    for (int c = 0; c < HD; ++c) o[c] = 0.f;
+    float m_used = -INFINITY, l = 0.f;
     bool ok = true;
     for (int j = 0; j < nkv; ++j) {
-      if (!mbar_wait(bar(5), j & 1, abort_flag, p.status, 207)) { ok = false; break; }
+      const int sb = j & 1;
+      if (!mbar_wait_warp(bar(9 + sb), (uint32_t)((j >> 1) & 1), abort_flag, p.status, 207)) { ok = false; break; }
       tc_fence_after();
+      uint32_t sv[4][32];
+#pragma unroll
+      for (int c = 0; c < 4; ++c) tc_ld32(tmem + lane_base + (uint32_t)(sb * 128 + 32 * c), sv[c]);
+      tc_wait_ld();
       const bool diag = (j == qi);
       float mx = -INFINITY;
-#pragma unroll 1
-      for (int c0 = 0; c0 < TK; c0 += 32) {
-        uint32_t v[32];
-        tc_ld32(tmem_s + lane_base + c0, v);
-        tc_wait_ld();
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-          float s = __uint_as_float(v[c]);
-          if (diag && (c0 + c > r)) s = -INFINITY;
+      for (int c = 0; c < 4; ++c)
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+          float s = __uint_as_float(sv[c][e]);
+          if (diag && (32 * c + e > r)) { s = -INFINITY; sv[c][e] = __float_as_uint(s); }
           mx = fmaxf(mx, s);
         }
-      }
-      const float m_new = fmaxf(m, mx * p.scale_log2);
-      const float corr = exp2f(m - m_new);
-      float rowsum = 0.f;
+      const float m_new = fmaxf(m_used, mx * p.scale_log2);
+      bool odone_waited = false;
+      if (__any_sync(0xffffffffu, m_new > m_used + 8.0f)) {
+        if (j > 0) {
+          if (!mbar_wait_warp(bar(12), (uint32_t)((j - 1) & 1), abort_flag, p.status, 208)) { ok = false; break; }
+          odone_waited = true;
+          tc_fence_after();
+          const float factor = ex2_approx(m_used - m_new);
+          l *= factor;
 #pragma unroll 1
-      for (int c0 = 0; c0 < TK; c0 += 32) {
-        uint32_t v[32];
-        tc_ld32(tmem_s + lane_base + c0, v);
-        tc_wait_ld();
-        uint32_t packed[16];
+          for (int c0 = 0; c0 < HD; c0 += 32) {
+            uint32_t ov[32];
+            tc_ld32(tmem_o + lane_base + c0, ov);
+            tc_wait_ld();
 #pragma unroll
-        for (int c = 0; c < 32; c += 2) {
-          float p0 = exp2f(__uint_as_float(v[c]) * p.scale_log2 - m_new);
-          float p1 = exp2f(__uint_as_float(v[c + 1]) * p.scale_log2 - m_new);
-          if (diag) { if (c0 + c > r) p0 = 0.f; if (c0 + c + 1 > r) p1 = 0.f; }
+            for (int e = 0; e < 32; ++e) ov[e] = __float_as_uint(__uint_as_float(ov[e]) * factor);
+            tc_st32(tmem_o + lane_base + c0, ov);
+          }
+          tc_wait_st();
+        }
+        m_used = m_new;
+      }
+      float rowsum = 0.f;
+      uint32_t packed[64];
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
+#pragma unroll
+        for (int e = 0; e < 32; e += 2) {
+          const float p0 = ex2_approx(__uint_as_float(sv[c][e]) * p.scale_log2 - m_used);
+          const float p1 = ex2_approx(__uint_as_float(sv[c][e + 1]) * p.scale_log2 - m_used);
           rowsum += p0 + p1;
           __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
-          packed[c >> 1] = *reinterpret_cast<uint32_t*>(&h2);
+          packed[16 * c + (e >> 1)] = *reinterpret_cast<uint32_t*>(&h2);
         }
-        uint8_t* blk = p_row + (c0 >> 6) * 16384;
+      l += rowsum;
+      if (j > 0 && !odone_waited) {      // P buffer is free once P V of the previous tile is complete
+        if (!mbar_wait_warp(bar(12), (uint32_t)((j - 1) & 1), abort_flag, p.status, 209)) { ok = false; break; }
+      }
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint8_t* blk = p_row + (c >> 1) * 16384;
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-          const int chunk = ((c0 & 63) >> 3) + k;
+          const int chunk = ((c & 1) << 2) + k;
           *reinterpret_cast<uint4*>(blk + ((chunk ^ (r & 7)) << 4)) =
-              make_uint4(packed[4 * k], packed[4 * k + 1], packed[4 * k + 2], packed[4 * k + 3]);
+              make_uint4(packed[16 * c + 4 * k], packed[16 * c + 4 * k + 1], packed[16 * c + 4 * k + 2],
+                         packed[16 * c + 4 * k + 3]);
         }
       }
-      l = l * corr + rowsum;
-      m = m_new;
       fence_proxy_async();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar(6));
-      if (!mbar_wait(bar(7), j & 1, abort_flag, p.status, 208)) { ok = false; break; }
-      tc_fence_after();
-#pragma unroll
-      for (int c0 = 0; c0 < HD; c0 += 32) {
-        uint32_t v[32];
-        tc_ld32(tmem_o + lane_base + c0, v);
-        tc_wait_ld();
-#pragma unroll
-        for (int c = 0; c < 32; ++c) o[c0 + c] = o[c0 + c] * corr + __uint_as_float(v[c]);
-      }
-      tc_fence_before();
+      if (lane == 0) mbar_arrive(bar(11));
     }
-    if (ok) {
+    if (ok && mbar_wait_warp(bar(12), (uint32_t)((nkv - 1) & 1), abort_flag, p.status, 210)) {
+      tc_fence_after();
       const float inv = 1.f / l;
       const long long tok = (long long)row0 + qi * TQ + r;
       bf16* orow = p.o + tok * d + h * HD;
+#pragma unroll 1
+      for (int c0 = 0; c0 < HD; c0 += 32) {
+        uint32_t ov[32];
+        tc_ld32(tmem_o + lane_base + c0, ov);
+        tc_wait_ld();
 #pragma unroll
-      for (int c = 0; c < HD; c += 8) {
-        uint4 u;
-        __nv_bfloat162* hh = reinterpret_cast<__nv_bfloat162*>(&u);
+        for (int c = 0; c < 32; c += 8) {
+          uint4 u;
+          __nv_bfloat162* hh = reinterpret_cast<__nv_bfloat162*>(&u);
 #pragma unroll
-        for (int e = 0; e < 4; ++e) hh[e] = __floats2bfloat162_rn(o[c + 2 * e] * inv, o[c + 2 * e + 1] * inv);
-        *reinterpret_cast<uint4*>(orow + c) = u;
+          for (int e = 0; e < 4; ++e)
+            hh[e] = __floats2bfloat162_rn(__uint_as_float(ov[c + 2 * e]) * inv, __uint_as_float(ov[c + 2 * e + 1]) * inv);
+          *reinterpret_cast<uint4*>(orow + c0 + c) = u;
+        }
       }
-      p.lse[((long long)b * p.H + h) * p.T + qi * TQ + r] = (m + log2f(l)) * 0.6931471805599453f;
+      p.lse[((long long)b * p.H + h) * p.T + qi * TQ + r] = (m_used + log2f(l)) * 0.6931471805599453f;
     }
   }
   tc_fence_before();
@@ -394,7 +420,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_co
       const long long stat = ((long long)b * p.H + h) * p.T + qi * 128 + r;
       const float lse2 = p.lse[stat] * 1.4426950408889634f;
       const float Dr = p.Dv[stat];
-      if (!mbar_wait(bar(2), ph, abort_flag, p.status, 306)) { ok = false; break; }
+      if (!mbar_wait_warp(bar(2), ph, abort_flag, p.status, 306)) { ok = false; break; }
       tc_fence_after();
       const bool diag = (it == 0);
 #pragma unroll 1
@@ -427,7 +453,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_co
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(3));
-      if (!mbar_wait(bar(4), ph, abort_flag, p.status, 307)) { ok = false; break; }
+      if (!mbar_wait_warp(bar(4), ph, abort_flag, p.status, 307)) { ok = false; break; }
       tc_fence_after();
       float* dq_row = p.dq_acc + tok * d + h * HD;
 #pragma unroll 1

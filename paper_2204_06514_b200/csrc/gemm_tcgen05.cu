@@ -181,7 +181,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       int tm, tn;
       tile_coords(tile, tiles_m, tiles_n, tm, tn);
       const int m0 = tm * BM, n0 = tn * BN;
-      if (!mbar_wait(tfull_bar(acc), acc_phase, abort_flag, p.status, 104)) { ok = false; break; }
+      if (!mbar_wait_warp(tfull_bar(acc), acc_phase, abort_flag, p.status, 104)) { ok = false; break; }
       tc_fence_after();
       const long long row = m0 + 32 * q + lane;
 #pragma unroll 1
