@@ -283,12 +283,14 @@ fax_status launch_fwd(fax_ctx* ctx, int B, int T, int H, const void* qkv, void* 
 // each) form P = exp(S/sqrt(hd) - LSE) and dS = P * (dP - D) and write both as
 // bf16 operand tiles; the elected thread then issues dV_j += P^T dO_i and
 // dK_j += dS^T Q_i (accumulating in tensor memory over the whole walk) and
-// dQ_i = dS K_j, which the row threads add into a float32 dQ buffer with vector
-// atomics.  The P / dS / Q / dO / K tiles are each used both as a K-major and as
+// dQ_i = dS K_j, which the row threads stage in shared memory and one thread adds
+// into a float32 dQ buffer with a bulk tensor reduction.  The P / dS / Q / dO / K tiles are each used both as a K-major and as
 // an MN-major operand: the bytes are the same, only the descriptor differs.
-// Tensor memory: [0,128) S then dQ, [128,256) dP, [256,256+HD) dV, [384,384+HD) dK.
+// Tensor memory: [0,128) S, [128,256) dP then dQ, [256,256+HD) dV, [384,384+HD) dK.  P is signalled
+// before dS so that dV runs while the row threads still work on dS; dK is issued before dQ so the Q
+// tile can be reloaded while dQ is computed and read out.
 // ---------------------------------------------------------------------------
-constexpr int BWD_THREADS = 160;
+constexpr int BWD_THREADS = 192;   // 4 row warps + MMA warp + TMA warp
 
 struct AttnBwdParams {
   int B, T, H;
@@ -299,29 +301,33 @@ struct AttnBwdParams {
 };
 
 template <int HD> struct BwdCfg {
+  static constexpr int NQ = (HD == 64) ? 2 : 1;          // Q / dO stages (shared memory allows 2 only at hd 64)
   static constexpr int TILE_BYTES = 128 * HD * 2;
   static constexpr int PS_BYTES = 128 * 128 * 2;
-  static constexpr int K_OFF = 0, V_OFF = TILE_BYTES, Q_OFF = 2 * TILE_BYTES, DO_OFF = 3 * TILE_BYTES;
-  static constexpr int P_OFF = 4 * TILE_BYTES, DS_OFF = P_OFF + PS_BYTES;
+  static constexpr int K_OFF = 0, V_OFF = TILE_BYTES;
+  static constexpr int Q_OFF = 2 * TILE_BYTES, DO_OFF = Q_OFF + NQ * TILE_BYTES;
+  static constexpr int P_OFF = DO_OFF + NQ * TILE_BYTES, DS_OFF = P_OFF + PS_BYTES;
   static constexpr int BAR_OFF = DS_OFF + PS_BYTES;
-  static constexpr int SMEM_BYTES = BAR_OFF + 128 + 1024;
-  static constexpr int TMEM_COLS = 512;
+  static constexpr int SMEM_BYTES = BAR_OFF + 256 + 1024;
+  static constexpr int TMEM_COLS = 512;                  // S [0,128) | dP then dQ [128,256) | dV [256,..) | dK [384,..)
 };
 
 template <int HD>
 __global__ void __launch_bounds__(BWD_THREADS, 1)
 attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_constant__ CUtensorMap tmap_do,
-                   const AttnBwdParams p) {
+                   const __grid_constant__ CUtensorMap tmap_dq, const AttnBwdParams p) {
   using C_ = BwdCfg<HD>;
+  constexpr int NQ = C_::NQ;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* gbase = smem_raw + (base - raw);
   const uint32_t bars = base + C_::BAR_OFF;
-  // barriers: 0 K/V, 1 Q/dO, 2 S+dP, 3 P+dS (4 arrivals), 4 dV/dK/dQ issued and done, 5 dQ read out (4 arrivals)
+  // barriers: 0 K/V full | 1,2 Q full | 3,4 dO full | 5,6 Q free | 7,8 dO free | 9 S full | 10 dP full |
+  //           11 P ready (4) | 12 dS ready (4) | 13 dQ full | 14 dQ read out (4)
   auto bar = [&](int i) { return bars + 8u * i; };
-  volatile uint32_t* tmem_slot = (volatile uint32_t*)(gbase + C_::BAR_OFF + 64);
-  volatile int* abort_flag = (volatile int*)(gbase + C_::BAR_OFF + 68);
+  volatile uint32_t* tmem_slot = (volatile uint32_t*)(gbase + C_::BAR_OFF + 128);
+  volatile int* abort_flag = (volatile int*)(gbase + C_::BAR_OFF + 132);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nq = p.T / 128;
@@ -335,7 +341,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_co
   const int nsteps = nq - kj;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < 6; ++i) mbar_init(bar(i), (i == 3 || i == 5) ? 4u : 1u);
+    for (int i = 0; i < 15; ++i) mbar_init(bar(i), (i == 11 || i == 12 || i == 14) ? 4u : 1u);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_qkv) : "memory");
@@ -347,65 +353,84 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_co
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   const uint32_t tm_s = tmem, tm_dp = tmem + 128, tm_dv = tmem + 256, tm_dk = tmem + 384;
+  const uint32_t k_s = base + C_::K_OFF, v_s = base + C_::V_OFF;
+  const uint32_t p_s = base + C_::P_OFF, ds_s = base + C_::DS_OFF;
+  auto q_s = [&](int i) { return base + C_::Q_OFF + i * C_::TILE_BYTES; };
+  auto do_s = [&](int i) { return base + C_::DO_OFF + i * C_::TILE_BYTES; };
 
-  if (warp == 4) {
+  if (warp == 5) {
+    // ---------------- TMA producer ----------------
     if (lane == 0) {
-      const uint32_t k_s = base + C_::K_OFF, v_s = base + C_::V_OFF, q_s = base + C_::Q_OFF, do_s = base + C_::DO_OFF;
-      const uint32_t p_s = base + C_::P_OFF, ds_s = base + C_::DS_OFF;
-      const uint32_t idesc_s = idesc_bf16(128, false, false);
-      const uint32_t idesc_kv = idesc_bf16(HD, true, true);
-      const uint32_t idesc_q = idesc_bf16(HD, false, true);
-      auto koff = [](int s) { return (uint32_t)((s / 4) * 16384 + (s % 4) * 32); };   // K-major k-step
-      // K_j, V_j once
       mbar_expect_tx(bar(0), 2 * C_::TILE_BYTES);
 #pragma unroll
       for (int i = 0; i < HD / 64; ++i) {
         tma_load_2d(k_s + i * 16384, &tmap_qkv, bar(0), kcol + 64 * i, row0 + kj * 128);
         tma_load_2d(v_s + i * 16384, &tmap_qkv, bar(0), vcol + 64 * i, row0 + kj * 128);
       }
-      auto load_q_do = [&](int qi) {
-        mbar_expect_tx(bar(1), 2 * C_::TILE_BYTES);
-#pragma unroll
-        for (int i = 0; i < HD / 64; ++i) {
-          tma_load_2d(q_s + i * 16384, &tmap_qkv, bar(1), qcol + 64 * i, row0 + qi * 128);
-          tma_load_2d(do_s + i * 16384, &tmap_do, bar(1), qcol + 64 * i, row0 + qi * 128);
-        }
-      };
-      load_q_do(kj);
-      bool ok = mbar_wait(bar(0), 0, abort_flag, p.status, 301);
+      bool ok = true;
       for (int it = 0; it < nsteps && ok; ++it) {
-        const uint32_t ph = (uint32_t)(it & 1);
-        if (!mbar_wait(bar(1), ph, abort_flag, p.status, 302)) { ok = false; break; }
-        if (it > 0 && !mbar_wait(bar(5), ph ^ 1u, abort_flag, p.status, 303)) { ok = false; break; }  // dQ of it-1 read
-        tc_fence_after();
+        const int st = it % NQ;
+        const uint32_t ph = (uint32_t)((it / NQ) & 1);
+        const int qrow = row0 + (kj + it) * 128;
+        if (!mbar_wait(bar(5 + st), ph ^ 1u, abort_flag, p.status, 301)) { ok = false; break; }
+        mbar_expect_tx(bar(1 + st), C_::TILE_BYTES);
 #pragma unroll
-        for (int s = 0; s < HD / 16; ++s)
-          tc_mma_bf16(tm_s, smem_desc(q_s + koff(s), 16, 1024), smem_desc(k_s + koff(s), 16, 1024), idesc_s, s ? 1u : 0u);
+        for (int i = 0; i < HD / 64; ++i) tma_load_2d(q_s(st) + i * 16384, &tmap_qkv, bar(1 + st), qcol + 64 * i, qrow);
+        if (!mbar_wait(bar(7 + st), ph ^ 1u, abort_flag, p.status, 302)) { ok = false; break; }
+        mbar_expect_tx(bar(3 + st), C_::TILE_BYTES);
 #pragma unroll
-        for (int s = 0; s < HD / 16; ++s)
-          tc_mma_bf16(tm_dp, smem_desc(do_s + koff(s), 16, 1024), smem_desc(v_s + koff(s), 16, 1024), idesc_s, s ? 1u : 0u);
-        tc_commit(bar(2));
-        if (!mbar_wait(bar(3), ph, abort_flag, p.status, 304)) { ok = false; break; }
-        tc_fence_after();
-#pragma unroll
-        for (int s = 0; s < 8; ++s)      // dV += P^T dO   (contraction over the 128 queries)
-          tc_mma_bf16(tm_dv, smem_desc(p_s + s * 2048, 16384, 1024), smem_desc(do_s + s * 2048, 16384, 1024),
-                      idesc_kv, (it | s) ? 1u : 0u);
-#pragma unroll
-        for (int s = 0; s < 8; ++s)      // dK += dS^T Q
-          tc_mma_bf16(tm_dk, smem_desc(ds_s + s * 2048, 16384, 1024), smem_desc(q_s + s * 2048, 16384, 1024),
-                      idesc_kv, (it | s) ? 1u : 0u);
-#pragma unroll
-        for (int s = 0; s < 8; ++s)      // dQ = dS K   (contraction over the 128 keys)
-          tc_mma_bf16(tm_s, smem_desc(ds_s + koff(s), 16, 1024), smem_desc(k_s + s * 2048, 16384, 1024),
-                      idesc_q, s ? 1u : 0u);
-        tc_commit(bar(4));
-        if (it + 1 < nsteps) {
-          if (!mbar_wait(bar(4), ph, abort_flag, p.status, 305)) { ok = false; break; }   // Q, dO tiles free
-          load_q_do(kj + it + 1);
-        }
+        for (int i = 0; i < HD / 64; ++i) tma_load_2d(do_s(st) + i * 16384, &tmap_do, bar(3 + st), qcol + 64 * i, qrow);
       }
       if (!ok) { const long long t0 = clock64(); while (clock64() - t0 < 2000000LL) { } }
+    }
+  } else if (warp == 4) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      const uint32_t idesc_s = idesc_bf16(128, false, false);
+      const uint32_t idesc_kv = idesc_bf16(HD, true, true);
+      const uint32_t idesc_q = idesc_bf16(HD, false, true);
+      auto koff = [](int s) { return (uint32_t)((s / 4) * 16384 + (s % 4) * 32); };   // K-major k-step
+      bool ok = mbar_wait(bar(0), 0, abort_flag, p.status, 303);
+      for (int it = 0; it < nsteps && ok; ++it) {
+        const int st = it % NQ;
+        const uint32_t sph = (uint32_t)((it / NQ) & 1), ph = (uint32_t)(it & 1);
+        // S = Q K^T  (the S columns were read out before P of the previous step was signalled)
+        if (!mbar_wait(bar(1 + st), sph, abort_flag, p.status, 304)) { ok = false; break; }
+        tc_fence_after();
+#pragma unroll
+        for (int s = 0; s < HD / 16; ++s)
+          tc_mma_bf16(tm_s, smem_desc(q_s(st) + koff(s), 16, 1024), smem_desc(k_s + koff(s), 16, 1024), idesc_s, s ? 1u : 0u);
+        tc_commit(bar(9));
+        // dP = dO V^T  (its columns double as dQ: wait until the previous dQ has been read out)
+        if (!mbar_wait(bar(3 + st), sph, abort_flag, p.status, 305)) { ok = false; break; }
+        if (it > 0 && !mbar_wait(bar(14), ph ^ 1u, abort_flag, p.status, 306)) { ok = false; break; }
+        tc_fence_after();
+#pragma unroll
+        for (int s = 0; s < HD / 16; ++s)
+          tc_mma_bf16(tm_dp, smem_desc(do_s(st) + koff(s), 16, 1024), smem_desc(v_s + koff(s), 16, 1024), idesc_s, s ? 1u : 0u);
+        tc_commit(bar(10));
+        // dV += P^T dO
+        if (!mbar_wait(bar(11), ph, abort_flag, p.status, 307)) { ok = false; break; }
+        tc_fence_after();
+#pragma unroll
+        for (int s = 0; s < 8; ++s)
+          tc_mma_bf16(tm_dv, smem_desc(p_s + s * 2048, 16384, 1024), smem_desc(do_s(st) + s * 2048, 16384, 1024),
+                      idesc_kv, (it | s) ? 1u : 0u);
+        tc_commit(bar(7 + st));          // dO stage free
+        // dK += dS^T Q, then dQ = dS K
+        if (!mbar_wait(bar(12), ph, abort_flag, p.status, 308)) { ok = false; break; }
+        tc_fence_after();
+#pragma unroll
+        for (int s = 0; s < 8; ++s)
+          tc_mma_bf16(tm_dk, smem_desc(ds_s + s * 2048, 16384, 1024), smem_desc(q_s(st) + s * 2048, 16384, 1024),
+                      idesc_kv, (it | s) ? 1u : 0u);
+        tc_commit(bar(5 + st));          // Q stage free
+#pragma unroll
+        for (int s = 0; s < 8; ++s)
+          tc_mma_bf16(tm_dp, smem_desc(ds_s + koff(s), 16, 1024), smem_desc(k_s + s * 2048, 16384, 1024),
+                      idesc_q, s ? 1u : 0u);
+        tc_commit(bar(13));              // dQ ready; also: every MMA issued so far is complete
+      }
     }
   } else {
     const int r = 32 * warp + lane;
@@ -416,63 +441,113 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_co
     for (int it = 0; it < nsteps; ++it) {
       const uint32_t ph = (uint32_t)(it & 1);
       const int qi = kj + it;
-      const long long tok = (long long)row0 + qi * 128 + r;
       const long long stat = ((long long)b * p.H + h) * p.T + qi * 128 + r;
       const float lse2 = p.lse[stat] * 1.4426950408889634f;
       const float Dr = p.Dv[stat];
-      if (!mbar_wait_warp(bar(2), ph, abort_flag, p.status, 306)) { ok = false; break; }
-      tc_fence_after();
       const bool diag = (it == 0);
-#pragma unroll 1
-      for (int c0 = 0; c0 < 128; c0 += 32) {
-        uint32_t sv[32], dv[32];
-        tc_ld32(tm_s + lane_base + c0, sv);
-        tc_ld32(tm_dp + lane_base + c0, dv);
-        tc_wait_ld();
-        uint32_t pp[16], dd[16];
+      uint32_t pp[64];
+      // P = exp(S / sqrt(hd) - LSE): the P tile is also needed (as bf16) by dS below
+      if (!mbar_wait_warp(bar(9), ph, abort_flag, p.status, 309)) { ok = false; break; }
+      tc_fence_after();
+      {
+        uint32_t sv[4][32];
 #pragma unroll
-        for (int c = 0; c < 32; c += 2) {
-          float p0 = exp2f(__uint_as_float(sv[c]) * p.scale_log2 - lse2);
-          float p1 = exp2f(__uint_as_float(sv[c + 1]) * p.scale_log2 - lse2);
-          if (diag) { if (c0 + c > r) p0 = 0.f; if (c0 + c + 1 > r) p1 = 0.f; }
-          float d0 = p0 * (__uint_as_float(dv[c]) - Dr);
-          float d1 = p1 * (__uint_as_float(dv[c + 1]) - Dr);
-          __nv_bfloat162 hp = __floats2bfloat162_rn(p0, p1), hd2 = __floats2bfloat162_rn(d0, d1);
-          pp[c >> 1] = *reinterpret_cast<uint32_t*>(&hp);
-          dd[c >> 1] = *reinterpret_cast<uint32_t*>(&hd2);
-        }
-        const int blk = (c0 >> 6) * 16384;
+        for (int c = 0; c < 4; ++c) tc_ld32(tm_s + lane_base + 32 * c, sv[c]);
+        tc_wait_ld();
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            float p0 = ex2_approx(__uint_as_float(sv[c][e]) * p.scale_log2 - lse2);
+            float p1 = ex2_approx(__uint_as_float(sv[c][e + 1]) * p.scale_log2 - lse2);
+            if (diag) { if (32 * c + e > r) p0 = 0.f; if (32 * c + e + 1 > r) p1 = 0.f; }
+            __nv_bfloat162 hp = __floats2bfloat162_rn(p0, p1);
+            pp[16 * c + (e >> 1)] = *reinterpret_cast<uint32_t*>(&hp);
+          }
+      }
+      if (it > 0) {
+        // the P / dS buffers staged the previous dQ tile: its bulk reduction must have read them
+        if (threadIdx.x == 0) bulk_wait_read_all();
+        named_barrier_sync(1, 128);
+      }
+#pragma unroll
+      for (int c = 0; c < 4; ++c)
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-          const int off = blk + ((((c0 & 63) >> 3) + k) ^ (r & 7)) * 16;
-          *reinterpret_cast<uint4*>(p_row + off) = make_uint4(pp[4 * k], pp[4 * k + 1], pp[4 * k + 2], pp[4 * k + 3]);
-          *reinterpret_cast<uint4*>(ds_row + off) = make_uint4(dd[4 * k], dd[4 * k + 1], dd[4 * k + 2], dd[4 * k + 3]);
+          const int off = (c >> 1) * 16384 + (((((c & 1) << 2) + k) ^ (r & 7)) << 4);
+          *reinterpret_cast<uint4*>(p_row + off) =
+              make_uint4(pp[16 * c + 4 * k], pp[16 * c + 4 * k + 1], pp[16 * c + 4 * k + 2], pp[16 * c + 4 * k + 3]);
+        }
+      fence_proxy_async();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(11));
+      // dS = P * (dP - D), from the bf16 P that the products use
+      if (!mbar_wait_warp(bar(10), ph, abort_flag, p.status, 310)) { ok = false; break; }
+      tc_fence_after();
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        uint32_t dv[2][32];
+        tc_ld32(tm_dp + lane_base + 64 * half, dv[0]);
+        tc_ld32(tm_dp + lane_base + 64 * half + 32, dv[1]);
+        tc_wait_ld();
+#pragma unroll
+        for (int cc = 0; cc < 2; ++cc) {
+          const int c = 2 * half + cc;
+          uint32_t dd[16];
+#pragma unroll
+          for (int e = 0; e < 32; e += 2) {
+            const float2 pf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pp[16 * c + (e >> 1)]));
+            __nv_bfloat162 hd2 = __floats2bfloat162_rn(pf.x * (__uint_as_float(dv[cc][e]) - Dr),
+                                                       pf.y * (__uint_as_float(dv[cc][e + 1]) - Dr));
+            dd[e >> 1] = *reinterpret_cast<uint32_t*>(&hd2);
+          }
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {
+            const int off = (c >> 1) * 16384 + (((((c & 1) << 2) + k) ^ (r & 7)) << 4);
+            *reinterpret_cast<uint4*>(ds_row + off) = make_uint4(dd[4 * k], dd[4 * k + 1], dd[4 * k + 2], dd[4 * k + 3]);
+          }
         }
       }
       fence_proxy_async();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar(3));
-      if (!mbar_wait_warp(bar(4), ph, abort_flag, p.status, 307)) { ok = false; break; }
+      if (lane == 0) mbar_arrive(bar(12));
+      // dQ tile of this step: tensor memory -> shared memory (the P / dS buffers, free by now, as
+      // 32-column boxes in the 128-byte-swizzled layout) -> one bulk add-reduction into the
+      // float32 dQ accumulator in global memory
+      if (!mbar_wait_warp(bar(13), ph, abort_flag, p.status, 311)) { ok = false; break; }
       tc_fence_after();
-      float* dq_row = p.dq_acc + tok * d + h * HD;
-#pragma unroll 1
-      for (int c0 = 0; c0 < HD; c0 += 32) {
-        uint32_t v[32];
-        tc_ld32(tm_s + lane_base + c0, v);
+#pragma unroll
+      for (int c0 = 0; c0 < HD; c0 += 64) {
+        uint32_t v[2][32];
+        tc_ld32(tm_dp + lane_base + c0, v[0]);
+        tc_ld32(tm_dp + lane_base + c0 + 32, v[1]);
         tc_wait_ld();
 #pragma unroll
-        for (int c = 0; c < 32; c += 4)
-          atomicAdd(reinterpret_cast<float4*>(dq_row + c0 + c),
-                    make_float4(__uint_as_float(v[c]), __uint_as_float(v[c + 1]), __uint_as_float(v[c + 2]),
-                                __uint_as_float(v[c + 3])));
+        for (int cc = 0; cc < 2; ++cc) {
+          uint8_t* box = gbase + C_::P_OFF + ((c0 >> 5) + cc) * 16384 + r * 128;
+#pragma unroll
+          for (int k = 0; k < 8; ++k)
+            *reinterpret_cast<uint4*>(box + ((k ^ (r & 7)) << 4)) =
+                make_uint4(v[cc][4 * k], v[cc][4 * k + 1], v[cc][4 * k + 2], v[cc][4 * k + 3]);
+        }
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar(5));
+      if (lane == 0) mbar_arrive(bar(14));
+      fence_proxy_async();
+      named_barrier_sync(1, 128);
+      if (threadIdx.x == 0) {
+#pragma unroll
+        for (int i = 0; i < HD / 32; ++i)
+          tma_reduce_add_2d(&tmap_dq, base + C_::P_OFF + i * 16384, h * HD + 32 * i, (int)(row0 + qi * 128));
+        bulk_commit_group();
+      }
     }
+    if (threadIdx.x == 0) bulk_wait_all();
     if (ok) {
-      // the last wait on barrier 4 covered every MMA: dV and dK of this key tile are final
+      // the last wait on the dQ barrier covered every MMA: dV and dK of this key tile are final
       const long long tok = (long long)row0 + kj * 128 + r;
       bf16* dk_row = p.dqkv + tok * 3 * d + d + h * HD;
       bf16* dv_row = p.dqkv + tok * 3 * d + 2 * d + h * HD;
@@ -538,11 +613,12 @@ __global__ void attn_dq_convert_kernel(long long n_tok, int d, const float* __re
 template <int HD>
 fax_status launch_bwd(fax_ctx* ctx, int B, int T, int H, const void* qkv, const void* o, const float* lse,
                       const void* d_o, void* dqkv, float* Dv, float* dq_acc) {
-  CUtensorMap mq, md;
+  CUtensorMap mq, md, mdq;
   const uint64_t d = (uint64_t)H * HD;
   const long long n_tok = (long long)B * T;
   if (!make_map(ctx, &mq, qkv, 3 * d, (uint64_t)n_tok, 3 * d, 64, 128)) return FAX_ERR_INVALID_ARG;
   if (!make_map(ctx, &md, d_o, d, (uint64_t)n_tok, d, 64, 128)) return FAX_ERR_INVALID_ARG;
+  if (!make_map_f32(ctx, &mdq, dq_acc, d, (uint64_t)n_tok, d, 32, 128)) return FAX_ERR_INVALID_ARG;
   FAX_CUDA_TRY(ctx, cudaMemsetAsync(dq_acc, 0, (size_t)n_tok * d * sizeof(float), ctx->stream));
   {
     const long long warps = n_tok * H;
@@ -564,7 +640,7 @@ fax_status launch_bwd(fax_ctx* ctx, int B, int T, int H, const void* qkv, const 
     attr_set = true;
   }
   const int grid = B * H * (T / 128);
-  attn_bwd_tc_kernel<HD><<<grid, BWD_THREADS, BwdCfg<HD>::SMEM_BYTES, ctx->stream>>>(mq, md, p);
+  attn_bwd_tc_kernel<HD><<<grid, BWD_THREADS, BwdCfg<HD>::SMEM_BYTES, ctx->stream>>>(mq, md, mdq, p);
   FAX_TRY(fax_after_launch(ctx));
   const long long quads = n_tok * (long long)d / 4;
   attn_dq_convert_kernel<<<(unsigned)((quads + 255) / 256), 256, 0, ctx->stream>>>(n_tok, (int)d, dq_acc, p.scale,
