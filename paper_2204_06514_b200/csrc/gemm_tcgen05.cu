@@ -5,7 +5,7 @@
 //
 //   warp 0      : TMA producer (one elected lane)
 //   warp 1      : tensor-memory allocation, MMA issue (one elected lane)
-//   warps 2..5  : epilogue; warp w reads TMEM lanes 32*(w%4) .. +31
+//   warps 2..9  : epilogue; warp w reads TMEM lanes 32*(w%4) .. +31, columns half (w-2)/4
 //
 // Operand layouts (both for A and B, chosen at run time):
 //   K-major  : [rows, K] row-major; one TMA box of 64 k x rows, 128-byte swizzle;
@@ -23,7 +23,7 @@ using namespace tc;
 
 constexpr int BM = 128;
 constexpr int BK = 64;
-constexpr int NUM_EPI_WARPS = 4;
+constexpr int NUM_EPI_WARPS = 8;      // two per tensor-memory lane quarter, each storing half of the columns
 constexpr int NUM_THREADS = 32 * (2 + NUM_EPI_WARPS);
 struct GemmParams {
   int M, N, K;
@@ -35,7 +35,25 @@ struct GemmParams {
   bf16* aux; long long ldaux;
   float alpha;
   int32_t* status;
+  int splits;          // > 1: each work item covers a slice of K and adds its partial tile into a float C
 };
+
+// GELU (tanh form) and its derivative with the hardware tanh approximation: its error
+// (about 5e-4 relative) is below the bf16 rounding of the values the epilogue stores.
+__device__ __forceinline__ float tanh_fast(float x) {
+  float y;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+__device__ __forceinline__ float gelu_fast(float h) {
+  const float t = tanh_fast(0.7978845608028654f * (h + 0.044715f * h * h * h));
+  return 0.5f * h * (1.0f + t);
+}
+__device__ __forceinline__ float gelu_grad_fast(float h) {
+  const float c = 0.7978845608028654f, a = 0.044715f;
+  const float t = tanh_fast(c * (h + a * h * h * h));
+  return 0.5f * (1.0f + t) + 0.5f * h * (1.0f - t * t) * c * (1.0f + 3.0f * a * h * h);
+}
 
 // Tile order: groups of GROUP_M row-tiles are swept across all column-tiles before the next
 // group starts, so the ~148 tiles in flight share few A row-panels and B column-panels in L2.
@@ -80,8 +98,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tiles_m = p.M / BM, tiles_n = p.N / BN;
-  const int num_tiles = tiles_m * tiles_n;
-  const int kblocks = p.K / BK;
+  const int out_tiles = tiles_m * tiles_n;
+  const int num_tiles = out_tiles * p.splits;          // work items: (output tile, K slice)
+  const int kb_total = p.K / BK;
+  const int kb_per = (kb_total + p.splits - 1) / p.splits;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < C_::STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -108,9 +128,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       bool ok = true;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
         int tm, tn;
-        tile_coords(tile, tiles_m, tiles_n, tm, tn);
+        tile_coords(tile % out_tiles, tiles_m, tiles_n, tm, tn);
         const int m0 = tm * BM, n0 = tn * BN;
-        for (int kb = 0; kb < kblocks; ++kb) {
+        const int kb0 = (tile / out_tiles) * kb_per, kb1 = min(kb_total, kb0 + kb_per);
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status, 101)) { ok = false; break; }
           const uint32_t a_dst = tiles_base + stage * C_::STAGE_BYTES;
           const uint32_t b_dst = a_dst + C_::A_BYTES;
@@ -153,7 +174,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         if (!mbar_wait(tempty_bar(acc), acc_phase ^ 1u, abort_flag, p.status, 102)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-        for (int kb = 0; kb < kblocks; ++kb) {
+        const int kb0 = (tile / out_tiles) * kb_per, kb1 = min(kb_total, kb0 + kb_per);
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status, 103)) { ok = false; break; }
           tc_fence_after();
           const uint32_t a_src = tiles_base + stage * C_::STAGE_BYTES;
@@ -162,7 +184,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
           for (int k = 0; k < BK / 16; ++k) {
             const uint64_t ad = smem_desc(a_src + k * a_kstep, a_lbo, 1024u);
             const uint64_t bd = smem_desc(b_src + k * b_kstep, b_lbo, 1024u);
-            tc_mma_bf16(d_tmem, ad, bd, idesc, (kb | k) ? 1u : 0u);
+            tc_mma_bf16(d_tmem, ad, bd, idesc, ((kb - kb0) | k) ? 1u : 0u);
           }
           tc_commit(empty_bar(stage));          // frees the smem stage once these MMAs have read it
           if (++stage == C_::STAGES) { stage = 0; phase ^= 1u; }
@@ -175,21 +197,20 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   } else {
     // ---------------- epilogue ----------------
     const int q = warp & 3;                      // TMEM lane quarter this warp may read
+    const int half = (warp - 2) >> 2;            // which half of the tile's columns this warp stores
+    constexpr int NCH = BN / 64;                 // 32-column chunks per warp
     int acc = 0; uint32_t acc_phase = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
       int tm, tn;
-      tile_coords(tile, tiles_m, tiles_n, tm, tn);
+      tile_coords(tile % out_tiles, tiles_m, tiles_n, tm, tn);
       const int m0 = tm * BM, n0 = tn * BN;
       if (!mbar_wait_warp(tfull_bar(acc), acc_phase, abort_flag, p.status, 104)) { ok = false; break; }
       tc_fence_after();
       const long long row = m0 + 32 * q + lane;
-#pragma unroll 1
-      for (int c0 = 0; c0 < BN; c0 += 32) {
-        uint32_t r[32];
-        tc_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(acc * BN + c0), r);
-        tc_wait_ld();
-        const int col = n0 + c0;
+      const uint32_t t_base = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(acc * BN + half * (BN / 2));
+      auto process = [&](const uint32_t (&r)[32], int c0) {
+        const int col = n0 + half * (BN / 2) + c0;
         float v[32];
 #pragma unroll
         for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) * p.alpha;
@@ -204,59 +225,88 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
           }
         }
         if (p.epi == EPI_BIAS_RESID) {
-          const uint4* rp = reinterpret_cast<const uint4*>(p.resid + row * p.ldr + col);
+          const bf16* rp = p.resid + row * p.ldr + col;
 #pragma unroll
-          for (int j4 = 0; j4 < 4; ++j4) {
-            uint4 u = rp[j4];
-            const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+          for (int j8 = 0; j8 < 2; ++j8) {
+            const U8 u = ld_global_v8(rp + 16 * j8);
 #pragma unroll
-            for (int e = 0; e < 4; ++e) { float2 f = __bfloat1622float2(h[e]); v[8 * j4 + 2 * e] += f.x; v[8 * j4 + 2 * e + 1] += f.y; }
+            for (int e = 0; e < 8; ++e) {
+              float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u.w[e]));
+              v[16 * j8 + 2 * e] += f.x; v[16 * j8 + 2 * e + 1] += f.y;
+            }
           }
         }
         if (p.epi == EPI_DGELU) {
-          const uint4* ap = reinterpret_cast<const uint4*>(p.aux + row * p.ldaux + col);
+          const bf16* ap = p.aux + row * p.ldaux + col;
 #pragma unroll
-          for (int j4 = 0; j4 < 4; ++j4) {
-            uint4 u = ap[j4];
-            const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+          for (int j8 = 0; j8 < 2; ++j8) {
+            const U8 u = ld_global_v8(ap + 16 * j8);
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              float2 f = __bfloat1622float2(h[e]);
-              v[8 * j4 + 2 * e] *= gelu_tanh_grad_f(f.x);
-              v[8 * j4 + 2 * e + 1] *= gelu_tanh_grad_f(f.y);
+            for (int e = 0; e < 8; ++e) {
+              float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u.w[e]));
+              v[16 * j8 + 2 * e] *= gelu_grad_fast(f.x);
+              v[16 * j8 + 2 * e + 1] *= gelu_grad_fast(f.y);
             }
           }
         }
         if (p.c_f32) {
-          float4* cp = reinterpret_cast<float4*>((float*)p.C + row * p.ldc + col);
+          float* cp = (float*)p.C + row * p.ldc + col;
+          if (p.splits > 1) {
 #pragma unroll
-          for (int j4 = 0; j4 < 8; ++j4) {
-            float4 o = make_float4(v[4 * j4], v[4 * j4 + 1], v[4 * j4 + 2], v[4 * j4 + 3]);
-            if (p.accumulate) { float4 c = cp[j4]; o.x += c.x; o.y += c.y; o.z += c.z; o.w += c.w; }
-            cp[j4] = o;
-          }
-        } else {
-          uint4* cp = reinterpret_cast<uint4*>((bf16*)p.C + row * p.ldc + col);
-          uint4* gp = (p.epi == EPI_BIAS_GELU) ? reinterpret_cast<uint4*>(p.aux + row * p.ldaux + col) : nullptr;
+            for (int j4 = 0; j4 < 8; ++j4)
+              atomicAdd(reinterpret_cast<float4*>(cp) + j4, make_float4(v[4 * j4], v[4 * j4 + 1], v[4 * j4 + 2], v[4 * j4 + 3]));
+          } else {
 #pragma unroll
-          for (int j4 = 0; j4 < 4; ++j4) {
-            uint4 u;
-            __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&u);
+            for (int j8 = 0; j8 < 4; ++j8) {
+              U8 o;
 #pragma unroll
-            for (int e = 0; e < 4; ++e) h[e] = __floats2bfloat162_rn(v[8 * j4 + 2 * e], v[8 * j4 + 2 * e + 1]);
-            cp[j4] = u;
-            if (gp) {
-              // GELU of the stored (rounded) pre-activation, so backward sees the same h
-              uint4 g;
-              __nv_bfloat162* gh = reinterpret_cast<__nv_bfloat162*>(&g);
+              for (int e = 0; e < 8; ++e) o.w[e] = __float_as_uint(v[8 * j8 + e]);
+              if (p.accumulate) {
+                const U8 c = ld_global_v8(cp + 8 * j8);
 #pragma unroll
-              for (int e = 0; e < 4; ++e) {
-                float2 f = __bfloat1622float2(h[e]);
-                gh[e] = __floats2bfloat162_rn(gelu_tanh_f(f.x), gelu_tanh_f(f.y));
+                for (int e = 0; e < 8; ++e) o.w[e] = __float_as_uint(__uint_as_float(o.w[e]) + __uint_as_float(c.w[e]));
               }
-              gp[j4] = g;
+              st_global_v8(cp + 8 * j8, o);
             }
           }
+        } else {
+          bf16* cp = (bf16*)p.C + row * p.ldc + col;
+          bf16* gp = (p.epi == EPI_BIAS_GELU) ? (p.aux + row * p.ldaux + col) : nullptr;
+#pragma unroll
+          for (int j8 = 0; j8 < 2; ++j8) {
+            U8 u;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              __nv_bfloat162 h2 = __floats2bfloat162_rn(v[16 * j8 + 2 * e], v[16 * j8 + 2 * e + 1]);
+              u.w[e] = *reinterpret_cast<uint32_t*>(&h2);
+            }
+            st_global_v8(cp + 16 * j8, u);
+            if (gp) {
+              // GELU of the stored (rounded) pre-activation, so backward sees the same h
+              U8 g;
+#pragma unroll
+              for (int e = 0; e < 8; ++e) {
+                float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u.w[e]));
+                __nv_bfloat162 g2 = __floats2bfloat162_rn(gelu_fast(f.x), gelu_fast(f.y));
+                g.w[e] = *reinterpret_cast<uint32_t*>(&g2);
+              }
+              st_global_v8(gp + 16 * j8, g);
+            }
+          }
+        }
+      };
+      // two register buffers: the tensor-memory load of the next chunk is in flight while this one is stored
+      uint32_t ra[32], rb[32];
+      tc_ld32(t_base, ra);
+#pragma unroll
+      for (int i = 0; i < NCH; i += 2) {
+        tc_wait_ld();
+        if (i + 1 < NCH) tc_ld32(t_base + 32 * (i + 1), rb);
+        process(ra, 32 * i);
+        if (i + 1 < NCH) {
+          tc_wait_ld();
+          if (i + 2 < NCH) tc_ld32(t_base + 32 * (i + 2), ra);
+          process(rb, 32 * (i + 1));
         }
       }
       tc_fence_before();
@@ -296,7 +346,24 @@ fax_status launch(fax_ctx* ctx, const FaxGemm& g) {
     attr_set = true;
   }
   const int tiles = (g.M / BM) * (g.N / BN);
-  const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
+  // Few output tiles and a long K (the weight-gradient shapes of narrow models): slice K so that
+  // the machine is filled; partial tiles are added into the float output with vector atomics.
+  p.splits = 1;
+  const int kb_total = g.K / BK;
+  if (g.c_f32 && g.epi == EPI_NONE && g.alpha == 1.f && tiles * 2 <= ctx->sm_count && kb_total >= 16) {
+    int sp = ctx->sm_count / tiles;
+    if (sp > kb_total / 8) sp = kb_total / 8;
+    if (sp > 16) sp = 16;
+    if (sp > 1) {
+      const int kb_per = (kb_total + sp - 1) / sp;
+      sp = (kb_total + kb_per - 1) / kb_per;          // no empty slices
+      p.splits = sp;
+    }
+  }
+  if (p.splits > 1 && !g.accumulate)
+    FAX_CUDA_TRY(ctx, cudaMemset2DAsync(g.C, (size_t)g.ldc * 4, 0, (size_t)g.N * 4, (size_t)g.M, ctx->stream));
+  const int items = tiles * p.splits;
+  const int grid = items < ctx->sm_count ? items : ctx->sm_count;
   gemm_tcgen05_kernel<BN><<<grid, NUM_THREADS, Cfg<BN>::SMEM_BYTES, ctx->stream>>>(ma, mb, p);
   return fax_after_launch(ctx);
 }
@@ -306,11 +373,11 @@ fax_status launch(fax_ctx* ctx, const FaxGemm& g) {
 bool fax_gemm_tc_supported(const FaxGemm& g) {
   if (g.M % BM || g.K % BK || pick_bn(g.N) == 0) return false;
   if (g.lda % 8 || g.ldb % 8) return false;
-  if (!fax_aligned(g.A, 16) || !fax_aligned(g.B, 16) || !fax_aligned(g.C, 16)) return false;
-  if (g.ldc % (g.c_f32 ? 4 : 8)) return false;
+  if (!fax_aligned(g.A, 16) || !fax_aligned(g.B, 16) || !fax_aligned(g.C, 32)) return false;
+  if (g.ldc % (g.c_f32 ? 8 : 16)) return false;             // the epilogue stores whole 32-byte sectors
   if (g.bias && !fax_aligned(g.bias, 16)) return false;
-  if (g.resid && (!fax_aligned(g.resid, 16) || g.ldr % 8)) return false;
-  if (g.aux && (!fax_aligned(g.aux, 16) || g.ldaux % 8)) return false;
+  if (g.resid && (!fax_aligned(g.resid, 32) || g.ldr % 16)) return false;
+  if (g.aux && (!fax_aligned(g.aux, 32) || g.ldaux % 16)) return false;
   return true;
 }
 

@@ -166,6 +166,26 @@ def test_gemm_epilogues(sess, prec, force_simt):
     assert relerr(run(ops.FAX_EPI_NONE, c_f32=1, accumulate=1, C0=C0), acc + C0) <= (1e-5 if prec == 1 else tol)
 
 
+@pytest.mark.parametrize("M,N,K", [(128, 256, 4096), (768, 768, 16384), (256, 128, 1088)])
+@pytest.mark.parametrize("accumulate", [0, 1])
+def test_gemm_weight_gradient_shapes_split_k(sess, M, N, K, accumulate):
+    """Few output tiles, long K: the kernel slices K and adds partial tiles into the float output."""
+    rng = np.random.default_rng(M + N + K)
+    A = synth.round_to_bf16(rng.standard_normal((K, M)).astype(np.float32))      # stored [K, M]
+    B = synth.round_to_bf16(rng.standard_normal((K, N)).astype(np.float32))      # stored [K, N]
+    C0 = rng.standard_normal((M, N)).astype(np.float32)
+    tA, tB = dev(A, torch.bfloat16, sess), dev(B, torch.bfloat16, sess)
+    tC = torch.as_tensor(C0).to(sess.device).contiguous()
+    desc = ops.GemmDesc(M, N, K, ptr(tA), M, 1, ptr(tB), N, 1, ptr(tC), N, 1, accumulate, ops.FAX_EPI_NONE,
+                        None, None, 0, None, 0, 1.0, 0)
+    for _ in range(2 if not accumulate else 1):          # overwrite mode is idempotent
+        ops.fax_op_gemm(sess.ctx, 0, desc)
+    ref = A.astype(np.float64).T @ B.astype(np.float64) + (C0 if accumulate else 0.0)
+    assert relerr(host(tC), ref) <= 1e-5
+    st, detail = fx.fax_check_device_status(sess.ctx)
+    assert st == fx.FAX_OK, detail
+
+
 ATTN_SHAPES = [(0, 2, 128, 4, 64), (0, 1, 384, 2, 128), (0, 2, 1024, 2, 64), (0, 1, 2048, 1, 128),
                (1, 2, 5, 2, 4), (1, 2, 130, 3, 64), (1, 1, 77, 2, 128)]
 
