@@ -300,11 +300,14 @@ def run_ours(args):
     ms_e2e = timed(step_host, e2e_steps)
 
     # per-kernel profile over whole steps (events around every operator launch)
+    # (AdamW is kept on the main stream here so that no kernel's events include another's work)
+    fx.fax_set_adamw_overlap(sess.ctx, False)
     fx.fax_profile_begin(sess.ctx)
     prof_steps = max(1, min(args.steps, 5))
     for _ in range(prof_steps):
         step()
     prof = fx.fax_profile_end(sess.ctx)
+    fx.fax_set_adamw_overlap(sess.ctx, True)
 
     if rank != 0:
         if world > 1:

@@ -201,7 +201,8 @@ fax_status fax_block_step(fax_ctx* ctx, const fax_block_cfg* cfg, const fax_bloc
 
 /* Same step with HOST buffers (pinned memory recommended): copies x and dy to
  * the device (staged in the scratch arena), runs the step, copies y and dx
- * back and synchronises.  scratch must hold fax_block_sizes' bytes plus
+ * back and synchronises.  dy travels to the device and y back to the host on
+ * a copy stream owned by the context while forward / backward run.  scratch must hold fax_block_sizes' bytes plus
  * 4*N*d*sizeof(T) of staging (fax_block_host_scratch_bytes). */
 fax_status fax_block_host_scratch_bytes(const fax_block_cfg* cfg, size_t* scratch_bytes);
 fax_status fax_block_step_host(fax_ctx* ctx, const fax_block_cfg* cfg, const fax_block_state* st,

@@ -36,6 +36,7 @@ extern "C" fax_status fax_create(fax_ctx** out, int32_t device_ordinal, void* cu
   c->encode_tiled = nullptr;
   c->prof_on = false;
   c->side = nullptr; c->ev_fork = nullptr; c->ev_join = nullptr; c->side_busy = false;
+  c->copy = nullptr; c->ev_copy_a = nullptr; c->ev_copy_b = nullptr;
   c->overlap_adamw = true;
   if (cudaMalloc((void**)&c->dev_status, 64) != cudaSuccess ||
       cudaMemset(c->dev_status, 0, 64) != cudaSuccess) {
@@ -54,7 +55,10 @@ extern "C" fax_status fax_create(fax_ctx** out, int32_t device_ordinal, void* cu
   c->encode_tiled = fn;
   if (cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) != cudaSuccess ||
       cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
-      cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess) {
+      cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess ||
+      cudaStreamCreateWithFlags(&c->copy, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaEventCreateWithFlags(&c->ev_copy_a, cudaEventDisableTiming) != cudaSuccess ||
+      cudaEventCreateWithFlags(&c->ev_copy_b, cudaEventDisableTiming) != cudaSuccess) {
     cudaFree(c->dev_status);
     delete c;
     return FAX_ERR_CUDA;
@@ -68,6 +72,9 @@ extern "C" fax_status fax_destroy(fax_ctx* ctx) {
   cudaSetDevice(ctx->device);
   cudaStreamSynchronize(ctx->stream);
   if (ctx->side) { cudaStreamSynchronize(ctx->side); cudaStreamDestroy(ctx->side); }
+  if (ctx->copy) { cudaStreamSynchronize(ctx->copy); cudaStreamDestroy(ctx->copy); }
+  if (ctx->ev_copy_a) cudaEventDestroy(ctx->ev_copy_a);
+  if (ctx->ev_copy_b) cudaEventDestroy(ctx->ev_copy_b);
   if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
   if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
   if (ctx->dev_status) cudaFree(ctx->dev_status);

@@ -260,9 +260,13 @@ fax_status fax_layer_check(const fax_layer_state* L, const fax_block_cfg* c) {
   return FAX_OK;
 }
 
+// hooks of the host-buffer variant: dY arrives and y leaves on the copy stream while the
+// forward / backward kernels run on the main stream
+struct HostIo { const void* dy_host; void* dy_dev; void* y_host; size_t bytes; };
+
 static fax_status block_step_impl(fax_ctx* ctx, const fax_block_cfg* cfg, const fax_block_state* st,
                                   const void* x, const void* dy, void* y, void* dx,
-                                  const fax_adamw_hparams* hp, size_t scratch_skip) {
+                                  const fax_adamw_hparams* hp, size_t scratch_skip, const HostIo* io = nullptr) {
   FaxArena ar(st->saved, st->saved_bytes), aw((char*)st->scratch + scratch_skip, st->scratch_bytes - scratch_skip);
   BlockSaved s; BlockScratch w;
   fax_block_carve_saved(cfg, ar, true, &s);
@@ -276,7 +280,20 @@ static fax_status block_step_impl(fax_ctx* ctx, const fax_block_cfg* cfg, const 
   h.grad_is_bf16 = 0;
   if (h.step < 1) return FAX_ERR_INVALID_ARG;
   FaxAdamHook hook = {t, &h};
+  if (io) {
+    // the copy stream may start once the main stream has reached this call (the staging buffers are free)
+    FAX_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_copy_a, ctx->stream));
+    FAX_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->copy, ctx->ev_copy_a, 0));
+    FAX_CUDA_TRY(ctx, cudaMemcpyAsync(io->dy_dev, io->dy_host, io->bytes, cudaMemcpyHostToDevice, ctx->copy));
+    FAX_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_copy_b, ctx->copy));
+  }
   FAX_TRY(fax_block_forward_impl(ctx, cfg, &p, x, y, s, true));
+  if (io) {
+    FAX_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_copy_a, ctx->stream));              // y is complete
+    FAX_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->copy, ctx->ev_copy_a, 0));
+    FAX_CUDA_TRY(ctx, cudaMemcpyAsync(io->y_host, y, io->bytes, cudaMemcpyDeviceToHost, ctx->copy));
+    FAX_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->stream, ctx->ev_copy_b, 0));       // dY has arrived
+  }
   FAX_TRY(fax_block_backward_impl(ctx, cfg, &p, dy, s, s.x, dx, &g, false, w, &hook));
   return fax_adamw_join(ctx);
 }
@@ -310,11 +327,11 @@ extern "C" fax_status fax_block_step_host(fax_ctx* ctx, const fax_block_cfg* cfg
   if (st->scratch_bytes < 4 * nd) return FAX_ERR_WORKSPACE_TOO_SMALL;
   char* base = (char*)st->scratch;
   void *x = base, *dy = base + nd, *y = base + 2 * nd, *dx = base + 3 * nd;
+  HostIo io = {dy_host, dy, y_host, bytes};
   FAX_CUDA_TRY(ctx, cudaMemcpyAsync(x, x_host, bytes, cudaMemcpyHostToDevice, ctx->stream));
-  FAX_CUDA_TRY(ctx, cudaMemcpyAsync(dy, dy_host, bytes, cudaMemcpyHostToDevice, ctx->stream));
-  FAX_TRY(block_step_impl(ctx, cfg, st, x, dy, y, dx, hp, 4 * nd));
-  FAX_CUDA_TRY(ctx, cudaMemcpyAsync(y_host, y, bytes, cudaMemcpyDeviceToHost, ctx->stream));
+  FAX_TRY(block_step_impl(ctx, cfg, st, x, dy, y, dx, hp, 4 * nd, &io));
   FAX_CUDA_TRY(ctx, cudaMemcpyAsync(dx_host, dx, bytes, cudaMemcpyDeviceToHost, ctx->stream));
   FAX_CUDA_TRY(ctx, cudaStreamSynchronize(ctx->stream));
+  FAX_CUDA_TRY(ctx, cudaStreamSynchronize(ctx->copy));
   return FAX_OK;
 }

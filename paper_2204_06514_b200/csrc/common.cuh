@@ -33,6 +33,8 @@ struct fax_ctx {
   std::vector<FaxProfRec> prof;
   cudaStream_t side;         // optimizer stream: AdamW of finished tensors overlaps the rest of backward
   cudaEvent_t ev_fork, ev_join;
+  cudaStream_t copy;         // host <-> device copies of the *_host entry points
+  cudaEvent_t ev_copy_a, ev_copy_b;
   bool side_busy;
   bool overlap_adamw;
 };

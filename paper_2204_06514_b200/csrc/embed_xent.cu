@@ -89,6 +89,64 @@ xent_kernel(int rows, int vocab, T* __restrict__ logits, int64_t ld, const int32
   }
 }
 
+// bf16 rows that fit in shared memory: the row is read from HBM once.  Pass 1 copies it to
+// shared memory and takes the maximum; pass 2 replaces each logit by exp(logit - max)
+// (bf16) while summing the unrounded exponentials; pass 3 writes (e / sum - onehot) * inv_n.
+__global__ void __launch_bounds__(512)
+xent_smem_kernel(int rows, int vocab, bf16* __restrict__ logits, int64_t ld, const int32_t* __restrict__ targets,
+                 float inv_n, float* __restrict__ row_loss) {
+  extern __shared__ uint4 xrow[];               // vocab / 8 vectors of 8 bf16
+  __shared__ float red[32];
+  const int r = blockIdx.x;
+  uint4* grow = reinterpret_cast<uint4*>(logits + (size_t)r * ld);
+  const int nvec = vocab >> 3;
+  float mx = -INFINITY;
+  for (int i = threadIdx.x; i < nvec; i += blockDim.x) {
+    const uint4 u = grow[i];
+    xrow[i] = u;
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) { float2 f = __bfloat1622float2(h[e]); mx = fmaxf(mx, fmaxf(f.x, f.y)); }
+  }
+  mx = block_reduce_max(mx, red);
+  const int tg = targets[r];
+  float s = 0.f;
+  for (int i = threadIdx.x; i < nvec; i += blockDim.x) {
+    uint4 u = xrow[i];
+    __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&u);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      float2 f = __bfloat1622float2(h[e]);
+      const float e0 = __expf(f.x - mx), e1 = __expf(f.y - mx);
+      s += e0 + e1;
+      h[e] = __floats2bfloat162_rn(e0, e1);
+    }
+    xrow[i] = u;
+  }
+  float lt = 0.f;
+  if (threadIdx.x == 0 && tg >= 0 && tg < vocab) lt = __bfloat162float(logits[(size_t)r * ld + tg]);   // still the logit: global row not yet rewritten
+  s = block_reduce_sum(s, red);
+  if (threadIdx.x == 0) {
+    const float lse = mx + logf(s);
+    row_loss[r] = (tg >= 0 && tg < vocab) ? lse - lt : 0.f;
+  }
+  const float k = inv_n / s;
+  for (int i = threadIdx.x; i < nvec; i += blockDim.x) {
+    uint4 u = xrow[i];
+    __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&u);
+    const int c0 = i << 3;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      float2 f = __bfloat1622float2(h[e]);
+      float p0 = f.x * k, p1 = f.y * k;
+      if (c0 + 2 * e == tg) p0 -= inv_n;
+      if (c0 + 2 * e + 1 == tg) p1 -= inv_n;
+      h[e] = __floats2bfloat162_rn(p0, p1);
+    }
+    grow[i] = u;
+  }
+}
+
 __global__ void loss_mean_kernel(int n, const float* __restrict__ row_loss, float* __restrict__ loss) {
   __shared__ double red[32];
   double s = 0.0;
@@ -137,7 +195,15 @@ fax_status fax_xent(fax_ctx* ctx, int prec, int rows, int vocab, void* logits, i
                     const int32_t* targets, float inv_n, float* row_loss) {
   // read the logits once, write dlogits once
   FaxProfScope prof(ctx, KC_XENT, 0.0, 2.0 * rows * (double)vocab * fax_elem_size(prec));
-  if (prec == FAX_PREC_BF16)
+  const size_t row_bytes = (size_t)vocab * 2;
+  if (prec == FAX_PREC_BF16 && vocab % 8 == 0 && ld % 8 == 0 && row_bytes <= 110 * 1024 && fax_aligned(logits, 16)) {
+    static bool attr_set = false;
+    if (!attr_set) {
+      FAX_CUDA_TRY(ctx, cudaFuncSetAttribute(xent_smem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024));
+      attr_set = true;
+    }
+    xent_smem_kernel<<<rows, 512, row_bytes, ctx->stream>>>(rows, vocab, (bf16*)logits, ld, targets, inv_n, row_loss);
+  } else if (prec == FAX_PREC_BF16)
     xent_kernel<bf16><<<rows, 512, 0, ctx->stream>>>(rows, vocab, (bf16*)logits, ld, targets, inv_n, row_loss);
   else
     xent_kernel<float><<<rows, 512, 0, ctx->stream>>>(rows, vocab, (float*)logits, ld, targets, inv_n, row_loss);
