@@ -174,6 +174,11 @@ fax_status fax_adamw_step(fax_ctx* ctx, const fax_adamw_tensor* tensors, int32_t
  * Results are identical either way.  Default: enabled. */
 fax_status fax_set_adamw_overlap(fax_ctx* ctx, int32_t enable);
 
+/* GEMMs whose M and N are multiples of 256 run on pairs of SMs (two-CTA
+ * clusters, one 256 x 256 tile per pair); enable = 0 keeps every GEMM on the
+ * one-CTA 128 x N kernel.  Same arithmetic either way.  Default: enabled. */
+fax_status fax_set_gemm_two_cta(fax_ctx* ctx, int32_t enable);
+
 /* One trainable tensor of a training state: float32 master, compute-precision
  * copy (bf16; in FP32_VALIDATE may equal w or be NULL), Adam moments, float32
  * gradient, element count and its weight decay. */

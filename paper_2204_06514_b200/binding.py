@@ -92,6 +92,7 @@ _SIGNATURES = {
     "fax_check_device_status": (C.c_int32, [_P, C.POINTER(C.c_int32)]),
     "fax_launch_count": (C.c_uint64, [_P]),
     "fax_set_adamw_overlap": (C.c_int32, [_P, C.c_int32]),
+    "fax_set_gemm_two_cta": (C.c_int32, [_P, C.c_int32]),
     "fax_profile_begin": (C.c_int32, [_P]),
     "fax_profile_end": (C.c_int32, [_P, C.POINTER(ProfileEntry), C.c_int32]),
     "fax_kernel_class_name": (C.c_char_p, [C.c_int32]),
@@ -182,6 +183,10 @@ def fax_check_device_status(ctx) -> tuple[int, int]:
 
 def fax_set_adamw_overlap(ctx, enable: bool):
     _check(load_library().fax_set_adamw_overlap(ctx, int(bool(enable))), "fax_set_adamw_overlap")
+
+
+def fax_set_gemm_two_cta(ctx, enable: bool):
+    _check(load_library().fax_set_gemm_two_cta(ctx, int(bool(enable))), "fax_set_gemm_two_cta")
 
 
 def fax_profile_begin(ctx):

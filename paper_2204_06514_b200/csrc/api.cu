@@ -38,6 +38,7 @@ extern "C" fax_status fax_create(fax_ctx** out, int32_t device_ordinal, void* cu
   c->side = nullptr; c->ev_fork = nullptr; c->ev_join = nullptr; c->side_busy = false;
   c->copy = nullptr; c->ev_copy_a = nullptr; c->ev_copy_b = nullptr;
   c->overlap_adamw = true;
+  c->use_2cta = true;
   if (cudaMalloc((void**)&c->dev_status, 64) != cudaSuccess ||
       cudaMemset(c->dev_status, 0, 64) != cudaSuccess) {
     delete c;
@@ -102,6 +103,12 @@ extern "C" fax_status fax_check_device_status(fax_ctx* ctx, int32_t* detail_host
 extern "C" fax_status fax_set_adamw_overlap(fax_ctx* ctx, int32_t enable) {
   if (!ctx) return FAX_ERR_INVALID_ARG;
   ctx->overlap_adamw = enable != 0;
+  return FAX_OK;
+}
+
+extern "C" fax_status fax_set_gemm_two_cta(fax_ctx* ctx, int32_t enable) {
+  if (!ctx) return FAX_ERR_INVALID_ARG;
+  ctx->use_2cta = enable != 0;
   return FAX_OK;
 }
 

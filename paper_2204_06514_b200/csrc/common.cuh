@@ -37,6 +37,7 @@ struct fax_ctx {
   cudaEvent_t ev_copy_a, ev_copy_b;
   bool side_busy;
   bool overlap_adamw;
+  bool use_2cta;             // GEMMs whose M and N are multiples of 256 use the two-CTA kernel
 };
 
 // Brackets the launches of one operator with CUDA events while profiling is on.
@@ -151,6 +152,8 @@ struct FaxGemm {
 fax_status fax_gemm_simt(fax_ctx* ctx, int prec, const FaxGemm& g);
 fax_status fax_gemm_tc(fax_ctx* ctx, const FaxGemm& g);       // bf16 tcgen05 path
 bool fax_gemm_tc_supported(const FaxGemm& g);
+bool fax_gemm_tc2_supported(const FaxGemm& g);                 // two-CTA 256 x 256 tiles
+fax_status fax_gemm_tc2(fax_ctx* ctx, const FaxGemm& g);
 fax_status fax_gemm(fax_ctx* ctx, int prec, const FaxGemm& g); // dispatch
 
 fax_status fax_layernorm_fwd(fax_ctx* ctx, int prec, int rows, int d, const void* x, const void* gamma,

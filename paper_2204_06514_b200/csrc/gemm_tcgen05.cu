@@ -15,7 +15,7 @@
 //              is +2048 B.
 // Every device-side wait is bounded; on expiry the kernel records an error in
 // the context's status word, drains and returns.
-#include "tc_common.cuh"
+#include "gemm_common.cuh"
 
 namespace {
 
@@ -25,49 +25,6 @@ constexpr int BM = 128;
 constexpr int BK = 64;
 constexpr int NUM_EPI_WARPS = 8;      // two per tensor-memory lane quarter, each storing half of the columns
 constexpr int NUM_THREADS = 32 * (2 + NUM_EPI_WARPS);
-struct GemmParams {
-  int M, N, K;
-  int a_mn, b_mn;
-  void* C; long long ldc; int c_f32; int accumulate;
-  int epi;
-  const bf16* bias;
-  const bf16* resid; long long ldr;
-  bf16* aux; long long ldaux;
-  float alpha;
-  int32_t* status;
-  int splits;          // > 1: each work item covers a slice of K and adds its partial tile into a float C
-};
-
-// GELU (tanh form) and its derivative with the hardware tanh approximation: its error
-// (about 5e-4 relative) is below the bf16 rounding of the values the epilogue stores.
-__device__ __forceinline__ float tanh_fast(float x) {
-  float y;
-  asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-__device__ __forceinline__ float gelu_fast(float h) {
-  const float t = tanh_fast(0.7978845608028654f * (h + 0.044715f * h * h * h));
-  return 0.5f * h * (1.0f + t);
-}
-__device__ __forceinline__ float gelu_grad_fast(float h) {
-  const float c = 0.7978845608028654f, a = 0.044715f;
-  const float t = tanh_fast(c * (h + a * h * h * h));
-  return 0.5f * (1.0f + t) + 0.5f * h * (1.0f - t * t) * c * (1.0f + 3.0f * a * h * h);
-}
-
-// Tile order: groups of GROUP_M row-tiles are swept across all column-tiles before the next
-// group starts, so the ~148 tiles in flight share few A row-panels and B column-panels in L2.
-constexpr int GROUP_M = 8;
-__device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int& tm, int& tn) {
-  const int per_group = GROUP_M * tiles_n;
-  const int g = tile / per_group;
-  const int first_m = g * GROUP_M;
-  const int rows = min(GROUP_M, tiles_m - first_m);
-  const int in = tile - g * per_group;
-  tm = first_m + in % rows;
-  tn = in / rows;
-}
-
 template <int BN> struct Cfg {
   static constexpr int A_BYTES = BM * BK * 2;
   static constexpr int B_BYTES = BN * BK * 2;
@@ -209,106 +166,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       tc_fence_after();
       const long long row = m0 + 32 * q + lane;
       const uint32_t t_base = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(acc * BN + half * (BN / 2));
-      auto process = [&](const uint32_t (&r)[32], int c0) {
-        const int col = n0 + half * (BN / 2) + c0;
-        float v[32];
-#pragma unroll
-        for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) * p.alpha;
-        if (p.epi == EPI_BIAS || p.epi == EPI_BIAS_GELU || p.epi == EPI_BIAS_RESID) {
-          const uint4* bp = reinterpret_cast<const uint4*>(p.bias + col);
-#pragma unroll
-          for (int j4 = 0; j4 < 4; ++j4) {
-            uint4 u = __ldg(bp + j4);
-            const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
-#pragma unroll
-            for (int e = 0; e < 4; ++e) { float2 f = __bfloat1622float2(h[e]); v[8 * j4 + 2 * e] += f.x; v[8 * j4 + 2 * e + 1] += f.y; }
-          }
-        }
-        if (p.epi == EPI_BIAS_RESID) {
-          const bf16* rp = p.resid + row * p.ldr + col;
-#pragma unroll
-          for (int j8 = 0; j8 < 2; ++j8) {
-            const U8 u = ld_global_v8(rp + 16 * j8);
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u.w[e]));
-              v[16 * j8 + 2 * e] += f.x; v[16 * j8 + 2 * e + 1] += f.y;
-            }
-          }
-        }
-        if (p.epi == EPI_DGELU) {
-          const bf16* ap = p.aux + row * p.ldaux + col;
-#pragma unroll
-          for (int j8 = 0; j8 < 2; ++j8) {
-            const U8 u = ld_global_v8(ap + 16 * j8);
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u.w[e]));
-              v[16 * j8 + 2 * e] *= gelu_grad_fast(f.x);
-              v[16 * j8 + 2 * e + 1] *= gelu_grad_fast(f.y);
-            }
-          }
-        }
-        if (p.c_f32) {
-          float* cp = (float*)p.C + row * p.ldc + col;
-          if (p.splits > 1) {
-#pragma unroll
-            for (int j4 = 0; j4 < 8; ++j4)
-              atomicAdd(reinterpret_cast<float4*>(cp) + j4, make_float4(v[4 * j4], v[4 * j4 + 1], v[4 * j4 + 2], v[4 * j4 + 3]));
-          } else {
-#pragma unroll
-            for (int j8 = 0; j8 < 4; ++j8) {
-              U8 o;
-#pragma unroll
-              for (int e = 0; e < 8; ++e) o.w[e] = __float_as_uint(v[8 * j8 + e]);
-              if (p.accumulate) {
-                const U8 c = ld_global_v8(cp + 8 * j8);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) o.w[e] = __float_as_uint(__uint_as_float(o.w[e]) + __uint_as_float(c.w[e]));
-              }
-              st_global_v8(cp + 8 * j8, o);
-            }
-          }
-        } else {
-          bf16* cp = (bf16*)p.C + row * p.ldc + col;
-          bf16* gp = (p.epi == EPI_BIAS_GELU) ? (p.aux + row * p.ldaux + col) : nullptr;
-#pragma unroll
-          for (int j8 = 0; j8 < 2; ++j8) {
-            U8 u;
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              __nv_bfloat162 h2 = __floats2bfloat162_rn(v[16 * j8 + 2 * e], v[16 * j8 + 2 * e + 1]);
-              u.w[e] = *reinterpret_cast<uint32_t*>(&h2);
-            }
-            st_global_v8(cp + 16 * j8, u);
-            if (gp) {
-              // GELU of the stored (rounded) pre-activation, so backward sees the same h
-              U8 g;
-#pragma unroll
-              for (int e = 0; e < 8; ++e) {
-                float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u.w[e]));
-                __nv_bfloat162 g2 = __floats2bfloat162_rn(gelu_fast(f.x), gelu_fast(f.y));
-                g.w[e] = *reinterpret_cast<uint32_t*>(&g2);
-              }
-              st_global_v8(gp + 16 * j8, g);
-            }
-          }
-        }
-      };
-      // two register buffers: the tensor-memory load of the next chunk is in flight while this one is stored
-      uint32_t ra[32], rb[32];
-      tc_ld32(t_base, ra);
-#pragma unroll
-      for (int i = 0; i < NCH; i += 2) {
-        tc_wait_ld();
-        if (i + 1 < NCH) tc_ld32(t_base + 32 * (i + 1), rb);
-        process(ra, 32 * i);
-        if (i + 1 < NCH) {
-          tc_wait_ld();
-          if (i + 2 < NCH) tc_ld32(t_base + 32 * (i + 2), ra);
-          process(rb, 32 * (i + 1));
-        }
-      }
+      gemm_epilogue_warp<NCH>(p, t_base, row, n0 + half * (BN / 2));
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(tempty_bar(acc));
@@ -384,6 +242,7 @@ bool fax_gemm_tc_supported(const FaxGemm& g) {
 fax_status fax_gemm_tc(fax_ctx* ctx, const FaxGemm& g) {
   if (!fax_gemm_tc_supported(g)) return FAX_ERR_UNSUPPORTED_SHAPE;
   FaxProfScope prof(ctx, KC_GEMM_TC, 2.0 * g.M * g.N * g.K, 0.0);
+  if (ctx->use_2cta && fax_gemm_tc2_supported(g)) return fax_gemm_tc2(ctx, g);
   switch (pick_bn(g.N)) {
     case 256: return launch<256>(ctx, g);
     case 128: return launch<128>(ctx, g);
