@@ -16,6 +16,7 @@ struct GemmParams {
   bf16* aux; long long ldaux;
   float alpha;
   int32_t* status;
+  int group_m;         // row-tiles per raster group
   int splits;          // > 1: each work item covers a slice of K and adds its partial tile into a float C
 };
 
@@ -36,14 +37,13 @@ __device__ __forceinline__ float gelu_grad_fast(float h) {
   return 0.5f * (1.0f + t) + 0.5f * h * (1.0f - t * t) * c * (1.0f + 3.0f * a * h * h);
 }
 
-// Tile order: groups of GROUP_M row-tiles are swept across all column-tiles before the next
+// Tile order: groups of group_m row-tiles are swept across all column-tiles before the next
 // group starts, so the ~148 tiles in flight share few A row-panels and B column-panels in L2.
-constexpr int GROUP_M = 8;
-__device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int& tm, int& tn) {
-  const int per_group = GROUP_M * tiles_n;
+__device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int group_m, int& tm, int& tn) {
+  const int per_group = group_m * tiles_n;
   const int g = tile / per_group;
-  const int first_m = g * GROUP_M;
-  const int rows = min(GROUP_M, tiles_m - first_m);
+  const int first_m = g * group_m;
+  const int rows = min(group_m, tiles_m - first_m);
   const int in = tile - g * per_group;
   tm = first_m + in % rows;
   tn = in / rows;

@@ -85,7 +85,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       bool ok = true;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
         int tm, tn;
-        tile_coords(tile % out_tiles, tiles_m, tiles_n, tm, tn);
+        tile_coords(tile % out_tiles, tiles_m, tiles_n, p.group_m, tm, tn);
         const int m0 = tm * BM, n0 = tn * BN;
         const int kb0 = (tile / out_tiles) * kb_per, kb1 = min(kb_total, kb0 + kb_per);
         for (int kb = kb0; kb < kb1; ++kb) {
@@ -160,7 +160,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     bool ok = true;
     for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
       int tm, tn;
-      tile_coords(tile % out_tiles, tiles_m, tiles_n, tm, tn);
+      tile_coords(tile % out_tiles, tiles_m, tiles_n, p.group_m, tm, tn);
       const int m0 = tm * BM, n0 = tn * BN;
       if (!mbar_wait_warp(tfull_bar(acc), acc_phase, abort_flag, p.status, 104)) { ok = false; break; }
       tc_fence_after();
@@ -197,6 +197,7 @@ fax_status launch(fax_ctx* ctx, const FaxGemm& g) {
   p.C = g.C; p.ldc = g.ldc; p.c_f32 = g.c_f32; p.accumulate = g.accumulate; p.epi = g.epi;
   p.bias = (const bf16*)g.bias; p.resid = (const bf16*)g.resid; p.ldr = g.ldr; p.aux = (bf16*)g.aux; p.ldaux = g.ldaux;
   p.alpha = g.alpha; p.status = ctx->dev_status;
+  p.group_m = 8;
   static bool attr_set = false;
   if (!attr_set) {
     FAX_CUDA_TRY(ctx, cudaFuncSetAttribute(gemm_tcgen05_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
