@@ -174,6 +174,15 @@ fax_status fax_adamw_step(fax_ctx* ctx, const fax_adamw_tensor* tensors, int32_t
  * Results are identical either way.  Default: enabled. */
 fax_status fax_set_adamw_overlap(fax_ctx* ctx, int32_t enable);
 
+/* fax_block_step and fax_lm_step replay a CUDA graph of the step from the third
+ * call on with the same configuration and the same buffers (first call: run as
+ * is; second call: captured on the context's stream in thread-local capture
+ * mode; later calls: the AdamW scalars are patched into the graph and it is
+ * launched).  Up to 8 graphs are kept per context.  enable = 0 turns this off
+ * and drops the graphs.  Do not call the whole-step functions while the stream
+ * is itself being captured by the caller.  Default: enabled. */
+fax_status fax_set_graph_replay(fax_ctx* ctx, int32_t enable);
+
 /* GEMMs whose M and N are multiples of 256 run on pairs of SMs (two-CTA
  * clusters, one 256 x 256 tile per pair); enable = 0 keeps every GEMM on the
  * one-CTA 128 x N kernel.  Same arithmetic either way.  Default: enabled. */

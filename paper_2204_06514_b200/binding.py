@@ -93,6 +93,7 @@ _SIGNATURES = {
     "fax_launch_count": (C.c_uint64, [_P]),
     "fax_set_adamw_overlap": (C.c_int32, [_P, C.c_int32]),
     "fax_set_gemm_two_cta": (C.c_int32, [_P, C.c_int32]),
+    "fax_set_graph_replay": (C.c_int32, [_P, C.c_int32]),
     "fax_profile_begin": (C.c_int32, [_P]),
     "fax_profile_end": (C.c_int32, [_P, C.POINTER(ProfileEntry), C.c_int32]),
     "fax_kernel_class_name": (C.c_char_p, [C.c_int32]),
@@ -183,6 +184,10 @@ def fax_check_device_status(ctx) -> tuple[int, int]:
 
 def fax_set_adamw_overlap(ctx, enable: bool):
     _check(load_library().fax_set_adamw_overlap(ctx, int(bool(enable))), "fax_set_adamw_overlap")
+
+
+def fax_set_graph_replay(ctx, enable: bool):
+    _check(load_library().fax_set_graph_replay(ctx, int(bool(enable))), "fax_set_graph_replay")
 
 
 def fax_set_gemm_two_cta(ctx, enable: bool):

@@ -4,6 +4,8 @@
 // (12 B) + write bf16 copy (2 B) = 30 B.
 #include "common.cuh"
 
+#include <cstring>
+
 namespace {
 
 constexpr int MAX_T = 40;              // tensors per launch (kernel-parameter space)
@@ -102,14 +104,29 @@ adamw_kernel(const __grid_constant__ AdamBatch batch, AdamScalars sc) {
 
 }  // namespace
 
-fax_status fax_adamw_launch(fax_ctx* ctx, const fax_adamw_tensor* tensors, int n, const fax_adamw_hparams* hp) {
-  if (!tensors || !hp || n < 0) return FAX_ERR_INVALID_ARG;
-  if (hp->step < 1 || !(hp->beta1 >= 0.f && hp->beta1 < 1.f) || !(hp->beta2 >= 0.f && hp->beta2 < 1.f))
-    return FAX_ERR_INVALID_ARG;
+static AdamScalars make_scalars(const fax_adamw_hparams* hp) {
   AdamScalars sc;
   sc.lr = hp->lr; sc.b1 = hp->beta1; sc.b2 = hp->beta2; sc.eps = hp->eps;
   sc.inv_bc1 = (float)(1.0 / (1.0 - pow((double)hp->beta1, (double)hp->step)));
   sc.inv_bc2 = (float)(1.0 / (1.0 - pow((double)hp->beta2, (double)hp->step)));
+  return sc;
+}
+
+bool fax_adamw_is_kernel(const void* func) {
+  return func == (const void*)adamw_kernel<false> || func == (const void*)adamw_kernel<true>;
+}
+
+void fax_adamw_scalars(const fax_adamw_hparams* hp, void* out32) {
+  static_assert(sizeof(AdamScalars) <= 32, "scalar block");
+  AdamScalars sc = make_scalars(hp);
+  memcpy(out32, &sc, sizeof(sc));
+}
+
+fax_status fax_adamw_launch(fax_ctx* ctx, const fax_adamw_tensor* tensors, int n, const fax_adamw_hparams* hp) {
+  if (!tensors || !hp || n < 0) return FAX_ERR_INVALID_ARG;
+  if (hp->step < 1 || !(hp->beta1 >= 0.f && hp->beta1 < 1.f) || !(hp->beta2 >= 0.f && hp->beta2 < 1.f))
+    return FAX_ERR_INVALID_ARG;
+  AdamScalars sc = make_scalars(hp);
   for (int i = 0; i < n; ++i) {
     const fax_adamw_tensor& t = tensors[i];
     if (!t.w || !t.m || !t.v || !t.g) return FAX_ERR_INVALID_ARG;

@@ -1,5 +1,5 @@
 // Context lifetime, status strings and the device status word.
-#include "common.cuh"
+#include "graph.cuh"
 
 extern "C" const char* fax_status_string(fax_status s) {
   switch (s) {
@@ -39,6 +39,8 @@ extern "C" fax_status fax_create(fax_ctx** out, int32_t device_ordinal, void* cu
   c->copy = nullptr; c->ev_copy_a = nullptr; c->ev_copy_b = nullptr;
   c->overlap_adamw = true;
   c->use_2cta = true;
+  c->use_graphs = true;
+  c->graph_clock = 0;
   if (cudaMalloc((void**)&c->dev_status, 64) != cudaSuccess ||
       cudaMemset(c->dev_status, 0, 64) != cudaSuccess) {
     delete c;
@@ -72,6 +74,7 @@ extern "C" fax_status fax_destroy(fax_ctx* ctx) {
   if (!ctx) return FAX_ERR_INVALID_ARG;
   cudaSetDevice(ctx->device);
   cudaStreamSynchronize(ctx->stream);
+  fax_graph_clear(ctx);
   if (ctx->side) { cudaStreamSynchronize(ctx->side); cudaStreamDestroy(ctx->side); }
   if (ctx->copy) { cudaStreamSynchronize(ctx->copy); cudaStreamDestroy(ctx->copy); }
   if (ctx->ev_copy_a) cudaEventDestroy(ctx->ev_copy_a);
@@ -103,12 +106,23 @@ extern "C" fax_status fax_check_device_status(fax_ctx* ctx, int32_t* detail_host
 extern "C" fax_status fax_set_adamw_overlap(fax_ctx* ctx, int32_t enable) {
   if (!ctx) return FAX_ERR_INVALID_ARG;
   ctx->overlap_adamw = enable != 0;
+  cudaStreamSynchronize(ctx->stream);
+  fax_graph_clear(ctx);
+  return FAX_OK;
+}
+
+extern "C" fax_status fax_set_graph_replay(fax_ctx* ctx, int32_t enable) {
+  if (!ctx) return FAX_ERR_INVALID_ARG;
+  ctx->use_graphs = enable != 0;
+  if (!ctx->use_graphs) { cudaStreamSynchronize(ctx->stream); fax_graph_clear(ctx); }
   return FAX_OK;
 }
 
 extern "C" fax_status fax_set_gemm_two_cta(fax_ctx* ctx, int32_t enable) {
   if (!ctx) return FAX_ERR_INVALID_ARG;
   ctx->use_2cta = enable != 0;
+  cudaStreamSynchronize(ctx->stream);
+  fax_graph_clear(ctx);
   return FAX_OK;
 }
 

@@ -2,6 +2,7 @@
 // backward (B1-B7) and the whole block training step with AdamW.  Only enqueues
 // kernels on the context's stream; every buffer is carved from caller arenas.
 #include "block.cuh"
+#include "graph.cuh"
 
 fax_status fax_block_validate(const fax_block_cfg* c) {
   if (!c) return FAX_ERR_INVALID_ARG;
@@ -304,7 +305,14 @@ extern "C" fax_status fax_block_step(fax_ctx* ctx, const fax_block_cfg* cfg, con
   if (!ctx || !st || !x || !dy || !y || !dx || !hp || !st->saved || !st->scratch || x == y) return FAX_ERR_INVALID_ARG;
   FAX_TRY(fax_block_validate(cfg));
   FAX_TRY(fax_layer_check(&st->layer, cfg));
-  return block_step_impl(ctx, cfg, st, x, dy, y, dx, hp, 0);
+  if (hp->step < 1) return FAX_ERR_INVALID_ARG;
+  uint64_t key = fax_hash(FAX_HASH_SEED, 'B');
+  key = fax_hash(key, *cfg);
+  key = fax_hash_layer(key, &st->layer);
+  key = fax_hash(key, st->saved); key = fax_hash(key, st->saved_bytes);
+  key = fax_hash(key, st->scratch); key = fax_hash(key, st->scratch_bytes);
+  key = fax_hash(key, x); key = fax_hash(key, dy); key = fax_hash(key, y); key = fax_hash(key, dx);
+  return fax_run_step(ctx, key, hp, [&]() { return block_step_impl(ctx, cfg, st, x, dy, y, dx, hp, 0); });
 }
 
 extern "C" fax_status fax_block_host_scratch_bytes(const fax_block_cfg* cfg, size_t* scratch_bytes) {

@@ -20,6 +20,15 @@ enum FaxKernelClass {
 };
 struct FaxProfRec { int cls; cudaEvent_t e0, e1; double flops, bytes; };
 
+struct FaxGraphEntry {
+  uint64_t key;
+  cudaGraph_t graph; cudaGraphExec_t exec;
+  std::vector<cudaGraphNode_t> adam_nodes;
+  std::vector<cudaKernelNodeParams> adam_params;
+  uint64_t launches, last_use;
+  bool failed;
+};
+
 // Device status block owned by the context: word 0 = error flag, word 1 = detail.
 struct fax_ctx {
   int device;
@@ -37,6 +46,9 @@ struct fax_ctx {
   cudaEvent_t ev_copy_a, ev_copy_b;
   bool side_busy;
   bool overlap_adamw;
+  bool use_graphs;           // whole-step calls are captured into CUDA graphs and replayed
+  std::vector<FaxGraphEntry> graphs;
+  uint64_t graph_clock;
   bool use_2cta;             // GEMMs whose M and N are multiples of 256 use the two-CTA kernel
 };
 
@@ -182,6 +194,8 @@ fax_status fax_adamw_launch(fax_ctx* ctx, const fax_adamw_tensor* tensors, int n
 // stream so far; fax_adamw_join makes the main stream wait for all of it.
 fax_status fax_adamw_async(fax_ctx* ctx, const fax_adamw_tensor* tensors, int n, const fax_adamw_hparams* hp);
 fax_status fax_adamw_join(fax_ctx* ctx);
+bool fax_adamw_is_kernel(const void* func);                        // one of the AdamW kernels?
+void fax_adamw_scalars(const fax_adamw_hparams* hp, void* out32);  // the kernels' by-value scalar argument
 struct FaxAdamHook { const fax_adamw_tensor* t; const fax_adamw_hparams* hp; };   // t: 12 tensors in parameter order
 
 fax_status fax_block_validate(const fax_block_cfg* cfg);

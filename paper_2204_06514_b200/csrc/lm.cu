@@ -3,6 +3,7 @@
 // (computed over row chunks so full logits never exist), backward through all
 // of it, and AdamW over every tensor.
 #include "block.cuh"
+#include "graph.cuh"
 
 #include <vector>
 
@@ -232,8 +233,17 @@ extern "C" fax_status fax_lm_forward_backward(fax_ctx* ctx, const fax_lm_cfg* cf
 extern "C" fax_status fax_lm_step(fax_ctx* ctx, const fax_lm_cfg* cfg, const fax_lm_state* st,
                                   const int32_t* ids, const int32_t* targets, const fax_adamw_hparams* hp,
                                   float* loss_device, float* loss_host) {
-  if (!ctx || !ids || !targets || !hp) return FAX_ERR_INVALID_ARG;
-  FAX_TRY(lm_run(ctx, cfg, st, ids, targets, hp, loss_device, nullptr, nullptr));
+  if (!ctx || !ids || !targets || !hp || !cfg || !st) return FAX_ERR_INVALID_ARG;
+  if (hp->step < 1 || cfg->n_layers <= 0 || !st->layers) return FAX_ERR_INVALID_ARG;
+  uint64_t key = fax_hash(FAX_HASH_SEED, 'L');
+  key = fax_hash(key, *cfg);
+  key = fax_hash_param(key, st->wte); key = fax_hash_param(key, st->wpe);
+  key = fax_hash_param(key, st->lnf_g); key = fax_hash_param(key, st->lnf_b);
+  for (int l = 0; l < cfg->n_layers; ++l) key = fax_hash_layer(key, &st->layers[l]);
+  key = fax_hash(key, st->saved); key = fax_hash(key, st->saved_bytes);
+  key = fax_hash(key, st->scratch); key = fax_hash(key, st->scratch_bytes);
+  key = fax_hash(key, ids); key = fax_hash(key, targets); key = fax_hash(key, loss_device);
+  FAX_TRY(fax_run_step(ctx, key, hp, [&]() { return lm_run(ctx, cfg, st, ids, targets, hp, loss_device, nullptr, nullptr); }));
   if (loss_host) {
     FAX_CUDA_TRY(ctx, cudaMemcpyAsync(loss_host, loss_device, sizeof(float), cudaMemcpyDeviceToHost, ctx->stream));
     FAX_CUDA_TRY(ctx, cudaStreamSynchronize(ctx->stream));

@@ -156,6 +156,48 @@ def test_block_step_host_matches_device_step(sess):
                 assert relerr(host(yh), host(a.y)) <= TOL_FWD_BF16
 
 
+def test_graph_replay_patches_the_adamw_scalars(sess):
+    """From the third call on a whole step is a replayed CUDA graph; the only arguments that change
+    are AdamW's scalars.  A step with lr = 0 must leave every weight exactly as it was."""
+    cfg = synth.CONFIGS["C1"]
+    params = synth.block_params(cfg)
+    x, dy = synth.block_inputs(cfg)
+    hp = dict(synth.ADAMW)
+    wd = hp.pop("weight_decay")
+    a = BlockRunner(sess, cfg, params, fx.FAX_PREC_BF16, weight_decay=wd)
+    tx, tdy = a.to_device(x), a.to_device(dy)
+    l0 = sess.launches()
+    a.step(tx, tdy, hparams(step=1, **hp))                 # as is
+    per_step = sess.launches() - l0
+    a.step(tx, tdy, hparams(step=2, **hp))                 # captured
+    torch.cuda.synchronize()
+    w2 = {k: a.p[k].w.clone() for k in O.PARAM_NAMES}
+    m2 = a.p["w_fc1"].m.clone()
+    frozen = dict(hp, lr=0.0)
+    a.step(tx, tdy, hparams(step=3, **frozen))             # replayed, lr = 0
+    torch.cuda.synchronize()
+    assert sess.launches() - l0 == 3 * per_step
+    for k in O.PARAM_NAMES:
+        assert torch.equal(a.p[k].w, w2[k]), k
+    assert not torch.equal(a.p["w_fc1"].m, m2)             # the step did run
+    a.step(tx, tdy, hparams(step=4, **hp))                 # replayed, lr back
+    torch.cuda.synchronize()
+    assert not torch.equal(a.p["w_fc1"].w, w2["w_fc1"])
+    # and the replayed forward equals a run without graphs on the same weights
+    fx.fax_set_graph_replay(sess.ctx, False)
+    y_graph = a.y.clone()
+    b = BlockRunner(sess, cfg, params, fx.FAX_PREC_BF16, weight_decay=wd)
+    for k in O.PARAM_NAMES:
+        b.p[k].w.copy_(w2[k]); b.p[k].wc.copy_(w2[k].to(torch.bfloat16))
+    # step 4 ran on the weights of step 2/3 (lr = 0 in between): same forward
+    b.forward(tx)
+    torch.cuda.synchronize()
+    fx.fax_set_graph_replay(sess.ctx, True)
+    assert torch.equal(b.y, y_graph)
+    st, detail = fx.fax_check_device_status(sess.ctx)
+    assert st == fx.FAX_OK, detail
+
+
 def test_block_error_paths(sess):
     cfg = synth.CONFIGS["C1"]
     r = BlockRunner(sess, cfg, synth.block_params(cfg), fx.FAX_PREC_BF16)
