@@ -212,6 +212,7 @@ def run_ours(args):
     peaks, peaks_kind = load_peaks()
     sess = Session(local)
     dev = sess.device
+    fx.fax_set_fused_update(sess.ctx, args.fused_update != "off", args.fused_update == "keep")
     hp0 = dict(synth.ADAMW)
     wd = hp0.pop("weight_decay")
     gen = torch.Generator(device=dev)
@@ -348,7 +349,7 @@ def run_ours(args):
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": workload_name(cfg), "tokens_per_step": tokens, "params": cfg.n_params,
-                   "replicas": world, "l2": "working set per step far exceeds the 126 MB L2"
+                   "replicas": world, "fused_update": args.fused_update, "l2": "working set per step far exceeds the 126 MB L2"
                    if cfg.n_params * 2 > 200e6 else "working set is L2-resident (small parity config)"},
         "mfu": {"step_flops": flops, "achieved_tflops": achieved_tf,
                 "vs_nominal_2250": achieved_tf / NOMINAL_BF16_TFLOPS,
@@ -373,6 +374,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", default="C3", choices=["C1", "C2", "C3", "C4", "C5"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--fused-update", default="off", choices=["off", "keep", "nograd"],
+                    help="AdamW of the weight matrices in the dW GEMM epilogue: off; on and the gradients still "
+                         "stored (default: every output of the step as documented); on without storing them")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

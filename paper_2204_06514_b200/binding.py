@@ -94,6 +94,7 @@ _SIGNATURES = {
     "fax_set_adamw_overlap": (C.c_int32, [_P, C.c_int32]),
     "fax_set_gemm_two_cta": (C.c_int32, [_P, C.c_int32]),
     "fax_set_graph_replay": (C.c_int32, [_P, C.c_int32]),
+    "fax_set_fused_update": (C.c_int32, [_P, C.c_int32, C.c_int32]),
     "fax_profile_begin": (C.c_int32, [_P]),
     "fax_profile_end": (C.c_int32, [_P, C.POINTER(ProfileEntry), C.c_int32]),
     "fax_kernel_class_name": (C.c_char_p, [C.c_int32]),
@@ -184,6 +185,11 @@ def fax_check_device_status(ctx) -> tuple[int, int]:
 
 def fax_set_adamw_overlap(ctx, enable: bool):
     _check(load_library().fax_set_adamw_overlap(ctx, int(bool(enable))), "fax_set_adamw_overlap")
+
+
+def fax_set_fused_update(ctx, enable: bool, keep_gradients: bool = False):
+    _check(load_library().fax_set_fused_update(ctx, int(bool(enable)), int(bool(keep_gradients))),
+           "fax_set_fused_update")
 
 
 def fax_set_graph_replay(ctx, enable: bool):

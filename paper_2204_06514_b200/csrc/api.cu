@@ -40,6 +40,8 @@ extern "C" fax_status fax_create(fax_ctx** out, int32_t device_ordinal, void* cu
   c->overlap_adamw = true;
   c->use_2cta = true;
   c->use_graphs = true;
+  c->fused_update = false;
+  c->keep_fused_grads = false;
   c->graph_clock = 0;
   if (cudaMalloc((void**)&c->dev_status, 64) != cudaSuccess ||
       cudaMemset(c->dev_status, 0, 64) != cudaSuccess) {
@@ -106,6 +108,15 @@ extern "C" fax_status fax_check_device_status(fax_ctx* ctx, int32_t* detail_host
 extern "C" fax_status fax_set_adamw_overlap(fax_ctx* ctx, int32_t enable) {
   if (!ctx) return FAX_ERR_INVALID_ARG;
   ctx->overlap_adamw = enable != 0;
+  cudaStreamSynchronize(ctx->stream);
+  fax_graph_clear(ctx);
+  return FAX_OK;
+}
+
+extern "C" fax_status fax_set_fused_update(fax_ctx* ctx, int32_t enable, int32_t keep_gradients) {
+  if (!ctx) return FAX_ERR_INVALID_ARG;
+  ctx->fused_update = enable != 0;
+  ctx->keep_fused_grads = keep_gradients != 0;
   cudaStreamSynchronize(ctx->stream);
   fax_graph_clear(ctx);
   return FAX_OK;

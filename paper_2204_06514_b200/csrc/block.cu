@@ -96,6 +96,7 @@ static FaxGemm gemm_desc(int M, int N, int K) {
   g.C = nullptr; g.ldc = N; g.c_f32 = false; g.accumulate = false;
   g.epi = EPI_NONE; g.bias = nullptr; g.resid = nullptr; g.ldr = 0; g.aux = nullptr; g.ldaux = 0;
   g.alpha = 1.f;
+  g.adam = nullptr;
   return g;
 }
 
@@ -120,12 +121,27 @@ static fax_status linear_bwd_data(fax_ctx* ctx, int prec, int N, int K, int Nout
   return fax_gemm(ctx, prec, g);
 }
 // dW (+)= x^T dy: x [N,K], dy [N,Nout] -> dW [K,Nout] float
+// With `fuse` (the AdamW descriptor and hyper-parameters of this weight) the update happens in the
+// GEMM's epilogue where that is possible; *fused tells the caller whether it did.
 static fax_status linear_bwd_weight(fax_ctx* ctx, int prec, int N, int K, int Nout, const void* x,
-                                    const void* dy, float* dW, bool accumulate) {
+                                    const void* dy, float* dW, bool accumulate,
+                                    const fax_adamw_tensor* fuse = nullptr, const fax_adamw_hparams* hp = nullptr,
+                                    bool* fused = nullptr) {
   FaxGemm g = gemm_desc(K, Nout, N);
   g.A = x; g.lda = K; g.a_mn_major = true;
   g.B = dy; g.ldb = Nout; g.b_mn_major = true;
   g.C = dW; g.ldc = Nout; g.c_f32 = true; g.accumulate = accumulate;
+  if (fused) *fused = false;
+  FaxFusedAdam ad;
+  if (fuse && hp && fuse->w_compute && fuse->n == (uint64_t)K * Nout && fax_gemm_can_fuse_adam(ctx, g)) {
+    ad.w = fuse->w; ad.m = fuse->m; ad.v = fuse->v; ad.w_compute = fuse->w_compute;
+    ad.weight_decay = fuse->weight_decay;
+    for (int i = 0; i < 8; ++i) ad.sc[i] = 0.f;
+    fax_adamw_scalars(hp, ad.sc);
+    ad.keep_grad = ctx->keep_fused_grads;
+    g.adam = &ad;
+    if (fused) *fused = true;
+  }
   return fax_gemm(ctx, prec, g);
 }
 
@@ -150,36 +166,44 @@ fax_status fax_block_backward_impl(fax_ctx* ctx, const fax_block_cfg* c, const f
   const int N = c->batch * c->seq, d = c->d_model, f = c->d_ff, prec = c->prec;
   // once both gradients of a linear layer (or LayerNorm) exist and the data-gradient GEMM has
   // consumed the old weight, its AdamW update runs on the optimizer stream under the rest of backward
-  auto update = [&](int first) -> fax_status {
-    return hook ? fax_adamw_async(ctx, hook->t + first, 2, hook->hp) : FAX_OK;
+  const bool try_fuse = hook && ctx->fused_update && prec == FAX_PREC_BF16 && !acc;
+  auto update = [&](int first, bool matrix_done = false) -> fax_status {
+    if (!hook) return FAX_OK;
+    return matrix_done ? fax_adamw_async(ctx, hook->t + first + 1, 1, hook->hp)      // only the bias is left
+                       : fax_adamw_async(ctx, hook->t + first, 2, hook->hp);
   };
+  bool fz = false;
   // B1: through FC2 and GELU
   FAX_TRY(linear_bwd_data(ctx, prec, N, f, d, dy, p->w_fc2, EPI_DGELU, s.h, w.bufF));          // dh
-  FAX_TRY(linear_bwd_weight(ctx, prec, N, f, d, s.g, dy, gr->w_fc2, acc));
+  FAX_TRY(linear_bwd_weight(ctx, prec, N, f, d, s.g, dy, gr->w_fc2, acc, try_fuse ? hook->t + 10 : nullptr,
+                            try_fuse ? hook->hp : nullptr, &fz));
   FAX_TRY(fax_colsum(ctx, prec, N, d, dy, d, gr->b_fc2, acc, w.partial, w.partial_floats));
-  FAX_TRY(update(10));
+  FAX_TRY(update(10, fz));
   // B2: through FC1
   FAX_TRY(linear_bwd_data(ctx, prec, N, d, f, w.bufF, p->w_fc1, EPI_NONE, nullptr, w.bufA));    // dm
-  FAX_TRY(linear_bwd_weight(ctx, prec, N, d, f, s.m, w.bufF, gr->w_fc1, acc));
+  FAX_TRY(linear_bwd_weight(ctx, prec, N, d, f, s.m, w.bufF, gr->w_fc1, acc, try_fuse ? hook->t + 8 : nullptr,
+                            try_fuse ? hook->hp : nullptr, &fz));
   FAX_TRY(fax_colsum(ctx, prec, N, f, w.bufF, f, gr->b_fc1, acc, w.partial, w.partial_floats));
-  FAX_TRY(update(8));
+  FAX_TRY(update(8, fz));
   // B3: LN2 backward plus the residual branch
   FAX_TRY(fax_layernorm_bwd(ctx, prec, N, d, w.bufA, s.x1, s.mu2, s.rstd2, p->ln2_g, dy, w.bufB,
                             gr->ln2_g, gr->ln2_b, acc, w.partial, w.partial_floats));           // dx1
   FAX_TRY(update(6));
   // B4: through the attention output projection
   FAX_TRY(linear_bwd_data(ctx, prec, N, d, d, w.bufB, p->w_o, EPI_NONE, nullptr, w.bufA));      // do
-  FAX_TRY(linear_bwd_weight(ctx, prec, N, d, d, s.o, w.bufB, gr->w_o, acc));
+  FAX_TRY(linear_bwd_weight(ctx, prec, N, d, d, s.o, w.bufB, gr->w_o, acc, try_fuse ? hook->t + 4 : nullptr,
+                            try_fuse ? hook->hp : nullptr, &fz));
   FAX_TRY(fax_colsum(ctx, prec, N, d, w.bufB, d, gr->b_o, acc, w.partial, w.partial_floats));
-  FAX_TRY(update(4));
+  FAX_TRY(update(4, fz));
   // B5: attention backward
   FAX_TRY(fax_attention_bwd(ctx, prec, c->batch, c->seq, c->n_heads, c->head_dim, s.qkv, s.o, s.lse,
                             w.bufA, w.bufQ, w.attn, w.attn_bytes));                             // dqkv
   // B6: through the QKV projection
   FAX_TRY(linear_bwd_data(ctx, prec, N, d, 3 * d, w.bufQ, p->w_qkv, EPI_NONE, nullptr, w.bufA)); // da
-  FAX_TRY(linear_bwd_weight(ctx, prec, N, d, 3 * d, s.a, w.bufQ, gr->w_qkv, acc));
+  FAX_TRY(linear_bwd_weight(ctx, prec, N, d, 3 * d, s.a, w.bufQ, gr->w_qkv, acc, try_fuse ? hook->t + 2 : nullptr,
+                            try_fuse ? hook->hp : nullptr, &fz));
   FAX_TRY(fax_colsum(ctx, prec, N, 3 * d, w.bufQ, 3 * d, gr->b_qkv, acc, w.partial, w.partial_floats));
-  FAX_TRY(update(2));
+  FAX_TRY(update(2, fz));
   // B7: LN1 backward plus the residual branch
   FAX_TRY(fax_layernorm_bwd(ctx, prec, N, d, w.bufA, x, s.mu1, s.rstd1, p->ln1_g, w.bufB, dx,
                             gr->ln1_g, gr->ln1_b, acc, w.partial, w.partial_floats));

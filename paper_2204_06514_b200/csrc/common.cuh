@@ -20,7 +20,13 @@ enum FaxKernelClass {
 };
 struct FaxProfRec { int cls; cudaEvent_t e0, e1; double flops, bytes; };
 
+struct FaxGemmPatch {
+  cudaGraphNode_t node; cudaKernelNodeParams params;
+  std::vector<unsigned char> blob;     // copy of the kernel's parameter struct, scalars patched per launch
+  size_t sc_offset;
+};
 struct FaxGraphEntry {
+  std::vector<FaxGemmPatch> gemm_nodes;
   uint64_t key;
   cudaGraph_t graph; cudaGraphExec_t exec;
   std::vector<cudaGraphNode_t> adam_nodes;
@@ -49,6 +55,8 @@ struct fax_ctx {
   bool use_graphs;           // whole-step calls are captured into CUDA graphs and replayed
   std::vector<FaxGraphEntry> graphs;
   uint64_t graph_clock;
+  bool fused_update;         // whole-step calls fuse AdamW of the weight matrices into the dW GEMM epilogue
+  bool keep_fused_grads;     // ... and still store those gradients
   bool use_2cta;             // GEMMs whose M and N are multiples of 256 use the two-CTA kernel
 };
 
@@ -145,7 +153,18 @@ enum FaxEpilogue {
   EPI_BIAS = 1,        // C = acc + bias[n]
   EPI_BIAS_GELU = 2,   // C = acc + bias (pre-activation), aux = GELU(C)
   EPI_BIAS_RESID = 3,  // C = acc + bias + resid
-  EPI_DGELU = 4        // C = acc * GELU'(aux)          (aux read-only, [M,N])
+  EPI_DGELU = 4,       // C = acc * GELU'(aux)          (aux read-only, [M,N])
+  EPI_ADAMW = 5        // internal: acc is a weight gradient, consumed by AdamW in the epilogue
+};
+
+// AdamW fused into the epilogue of a weight-gradient GEMM: the accumulator tile is the
+// gradient; w, m, v (float, [M,N] with the row pitch of C) are updated in place and the
+// bf16 copy refreshed, so the gradient never travels to HBM and back.
+struct FaxFusedAdam {
+  float* w; float* m; float* v; void* w_compute;
+  float weight_decay;
+  float sc[8];               // lr, beta1, beta2, eps, 1/(1-beta1^t), 1/(1-beta2^t)
+  bool keep_grad;            // also store the gradient to C
 };
 
 struct FaxGemm {
@@ -159,6 +178,7 @@ struct FaxGemm {
   const void* resid; int64_t ldr;               // [M,N] type T
   void* aux; int64_t ldaux;                     // [M,N] type T
   float alpha;                                  // scales acc before the epilogue
+  const FaxFusedAdam* adam;                     // non-null: EPI_ADAMW (float C, epi NONE, no accumulate)
 };
 
 fax_status fax_gemm_simt(fax_ctx* ctx, int prec, const FaxGemm& g);
@@ -167,6 +187,13 @@ bool fax_gemm_tc_supported(const FaxGemm& g);
 bool fax_gemm_tc2_supported(const FaxGemm& g);                 // two-CTA 256 x 256 tiles
 fax_status fax_gemm_tc2(fax_ctx* ctx, const FaxGemm& g);
 fax_status fax_gemm(fax_ctx* ctx, int prec, const FaxGemm& g); // dispatch
+// Would fax_gemm run this (bf16) problem on a tensor-core kernel without slicing K?  Only then
+// can AdamW be fused into its epilogue.
+bool fax_gemm_can_fuse_adam(fax_ctx* ctx, const FaxGemm& g);
+// If `func` is a GEMM kernel launched with EPI_ADAMW parameters at `param`, gives the size of the
+// parameter struct and the offset of the six AdamW scalars in it (for graph replay).
+bool fax_gemm_patch_info_1cta(const void* func, const void* param, size_t* size, size_t* sc_offset);
+bool fax_gemm_patch_info_2cta(const void* func, const void* param, size_t* size, size_t* sc_offset);
 
 fax_status fax_layernorm_fwd(fax_ctx* ctx, int prec, int rows, int d, const void* x, const void* gamma,
                              const void* beta, float eps, void* out, float* mu, float* rstd, void* x_copy);

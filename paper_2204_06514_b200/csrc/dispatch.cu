@@ -3,6 +3,7 @@
 
 fax_status fax_gemm(fax_ctx* ctx, int prec, const FaxGemm& g) {
   if (prec == FAX_PREC_BF16 && fax_gemm_tc_supported(g)) return fax_gemm_tc(ctx, g);
+  if (g.adam) return FAX_ERR_INVALID_ARG;               // callers ask fax_gemm_can_fuse_adam first
   return fax_gemm_simt(ctx, prec, g);
 }
 

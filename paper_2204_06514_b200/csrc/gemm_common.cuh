@@ -16,6 +16,8 @@ struct GemmParams {
   bf16* aux; long long ldaux;
   float alpha;
   int32_t* status;
+  float* ad_w; float* ad_m; float* ad_v; bf16* ad_wc;   // EPI_ADAMW: state of the weight this GEMM's result updates
+  float ad_wd; float ad_sc[8]; int ad_keep;
   int group_m;         // row-tiles per raster group
   int splits;          // > 1: each work item covers a slice of K and adds its partial tile into a float C
 };
@@ -89,7 +91,44 @@ __device__ __forceinline__ void gemm_epilogue_chunk(const GemmParams& p, const u
             }
           }
         }
-        if (p.c_f32) {
+        if (p.epi == EPI_ADAMW) {
+          // the accumulator is the gradient of w[row, col..]: AdamW here, w / m / v in place
+          const long long off = row * p.ldc + col;
+          const float lr = p.ad_sc[0], b1 = p.ad_sc[1], b2 = p.ad_sc[2], eps = p.ad_sc[3];
+          const float ibc1 = p.ad_sc[4], ibc2 = p.ad_sc[5];
+#pragma unroll
+          for (int j8 = 0; j8 < 4; ++j8) {
+            U8 w8 = ld_global_v8(p.ad_w + off + 8 * j8);
+            U8 m8 = ld_global_v8(p.ad_m + off + 8 * j8);
+            U8 v8 = ld_global_v8(p.ad_v + off + 8 * j8);
+            uint4 c8;
+            __nv_bfloat162* ch = reinterpret_cast<__nv_bfloat162*>(&c8);
+            float wn[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              const float g = v[8 * j8 + e];
+              float w = __uint_as_float(w8.w[e]), m = __uint_as_float(m8.w[e]), vv = __uint_as_float(v8.w[e]);
+              m = b1 * m + (1.f - b1) * g;
+              vv = b2 * vv + (1.f - b2) * g * g;
+              const float mh = m * ibc1, vh = vv * ibc2;
+              w = w - lr * p.ad_wd * w - lr * mh / (sqrtf(vh) + eps);
+              w8.w[e] = __float_as_uint(w); m8.w[e] = __float_as_uint(m); v8.w[e] = __float_as_uint(vv);
+              wn[e] = w;
+            }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) ch[e] = __floats2bfloat162_rn(wn[2 * e], wn[2 * e + 1]);
+            st_global_v8(p.ad_w + off + 8 * j8, w8);
+            st_global_v8(p.ad_m + off + 8 * j8, m8);
+            st_global_v8(p.ad_v + off + 8 * j8, v8);
+            *reinterpret_cast<uint4*>(p.ad_wc + off + 8 * j8) = c8;
+            if (p.ad_keep) {
+              U8 g8;
+#pragma unroll
+              for (int e = 0; e < 8; ++e) g8.w[e] = __float_as_uint(v[8 * j8 + e]);
+              st_global_v8((float*)p.C + off + 8 * j8, g8);
+            }
+          }
+        } else if (p.c_f32) {
           float* cp = (float*)p.C + row * p.ldc + col;
           if (p.splits > 1) {
 #pragma unroll
@@ -134,6 +173,37 @@ __device__ __forceinline__ void gemm_epilogue_chunk(const GemmParams& p, const u
             }
           }
         }
+}
+
+// Fills the kernel parameters that do not depend on the tile shape.
+static inline void fill_gemm_params(GemmParams& p, const FaxGemm& g, int32_t* status) {
+  p.M = g.M; p.N = g.N; p.K = g.K; p.a_mn = g.a_mn_major; p.b_mn = g.b_mn_major;
+  p.C = g.C; p.ldc = g.ldc; p.c_f32 = g.c_f32; p.accumulate = g.accumulate; p.epi = g.epi;
+  p.bias = (const bf16*)g.bias; p.resid = (const bf16*)g.resid; p.ldr = g.ldr; p.aux = (bf16*)g.aux; p.ldaux = g.ldaux;
+  p.alpha = g.alpha; p.status = status;
+  p.group_m = 8;
+  p.splits = 1;
+  p.ad_w = p.ad_m = p.ad_v = nullptr; p.ad_wc = nullptr; p.ad_wd = 0.f; p.ad_keep = 0;
+  for (int i = 0; i < 8; ++i) p.ad_sc[i] = 0.f;
+  if (g.adam) {
+    p.epi = EPI_ADAMW;
+    p.ad_w = g.adam->w; p.ad_m = g.adam->m; p.ad_v = g.adam->v; p.ad_wc = (bf16*)g.adam->w_compute;
+    p.ad_wd = g.adam->weight_decay; p.ad_keep = g.adam->keep_grad ? 1 : 0;
+    for (int i = 0; i < 8; ++i) p.ad_sc[i] = g.adam->sc[i];
+  }
+}
+
+// Number of K slices the launchers use for a problem with `tiles` output tiles on `units`
+// tile-processing units (SMs, or SM pairs).
+static inline int gemm_split_count(const FaxGemm& g, int tiles, int units, int bk) {
+  const int kb_total = g.K / bk;
+  if (!(g.c_f32 && g.epi == EPI_NONE && g.alpha == 1.f && !g.adam && tiles * 2 <= units && kb_total >= 16)) return 1;
+  int sp = units / tiles;
+  if (sp > kb_total / 8) sp = kb_total / 8;
+  if (sp > 16) sp = 16;
+  if (sp <= 1) return 1;
+  const int kb_per = (kb_total + sp - 1) / sp;
+  return (kb_total + kb_per - 1) / kb_per;          // no empty slices
 }
 
 // One warp's share of a tile: NCH chunks of 32 columns starting at tensor-memory address

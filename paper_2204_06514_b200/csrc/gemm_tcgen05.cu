@@ -17,6 +17,8 @@
 // the context's status word, drains and returns.
 #include "gemm_common.cuh"
 
+#include <cstddef>
+
 namespace {
 
 using namespace tc;
@@ -193,11 +195,7 @@ fax_status launch(fax_ctx* ctx, const FaxGemm& g) {
                            : make_map(ctx, &mb, g.B, g.K, g.N, g.ldb, BK, BN));
   if (!ok) return FAX_ERR_INVALID_ARG;
   GemmParams p;
-  p.M = g.M; p.N = g.N; p.K = g.K; p.a_mn = g.a_mn_major; p.b_mn = g.b_mn_major;
-  p.C = g.C; p.ldc = g.ldc; p.c_f32 = g.c_f32; p.accumulate = g.accumulate; p.epi = g.epi;
-  p.bias = (const bf16*)g.bias; p.resid = (const bf16*)g.resid; p.ldr = g.ldr; p.aux = (bf16*)g.aux; p.ldaux = g.ldaux;
-  p.alpha = g.alpha; p.status = ctx->dev_status;
-  p.group_m = 8;
+  fill_gemm_params(p, g, ctx->dev_status);
   static bool attr_set = false;
   if (!attr_set) {
     FAX_CUDA_TRY(ctx, cudaFuncSetAttribute(gemm_tcgen05_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -207,18 +205,7 @@ fax_status launch(fax_ctx* ctx, const FaxGemm& g) {
   const int tiles = (g.M / BM) * (g.N / BN);
   // Few output tiles and a long K (the weight-gradient shapes of narrow models): slice K so that
   // the machine is filled; partial tiles are added into the float output with vector atomics.
-  p.splits = 1;
-  const int kb_total = g.K / BK;
-  if (g.c_f32 && g.epi == EPI_NONE && g.alpha == 1.f && tiles * 2 <= ctx->sm_count && kb_total >= 16) {
-    int sp = ctx->sm_count / tiles;
-    if (sp > kb_total / 8) sp = kb_total / 8;
-    if (sp > 16) sp = 16;
-    if (sp > 1) {
-      const int kb_per = (kb_total + sp - 1) / sp;
-      sp = (kb_total + kb_per - 1) / kb_per;          // no empty slices
-      p.splits = sp;
-    }
-  }
+  p.splits = gemm_split_count(g, tiles, ctx->sm_count, BK);
   if (p.splits > 1 && !g.accumulate)
     FAX_CUDA_TRY(ctx, cudaMemset2DAsync(g.C, (size_t)g.ldc * 4, 0, (size_t)g.N * 4, (size_t)g.M, ctx->stream));
   const int items = tiles * p.splits;
@@ -228,6 +215,26 @@ fax_status launch(fax_ctx* ctx, const FaxGemm& g) {
 }
 
 }  // namespace
+
+bool fax_gemm_patch_info_1cta(const void* func, const void* param, size_t* size, size_t* sc_offset) {
+  if (func != (const void*)gemm_tcgen05_kernel<256> && func != (const void*)gemm_tcgen05_kernel<128> &&
+      func != (const void*)gemm_tcgen05_kernel<64>)
+    return false;
+  if (((const GemmParams*)param)->epi != EPI_ADAMW) return false;
+  *size = sizeof(GemmParams);
+  *sc_offset = offsetof(GemmParams, ad_sc);
+  return true;
+}
+
+bool fax_gemm_can_fuse_adam(fax_ctx* ctx, const FaxGemm& g) {
+  if (!fax_gemm_tc_supported(g) || !g.c_f32 || g.epi != EPI_NONE || g.accumulate || g.alpha != 1.f) return false;
+  if (g.ldc != g.N) return false;                       // w, m, v share C's dense layout
+  FaxGemm plain = g;
+  plain.adam = nullptr;
+  if (ctx->use_2cta && fax_gemm_tc2_supported(g))
+    return gemm_split_count(plain, (g.M / 256) * (g.N / 256), ctx->sm_count / 2, BK) == 1;
+  return gemm_split_count(plain, (g.M / BM) * (g.N / pick_bn(g.N)), ctx->sm_count, BK) == 1;
+}
 
 bool fax_gemm_tc_supported(const FaxGemm& g) {
   if (g.M % BM || g.K % BK || pick_bn(g.N) == 0) return false;

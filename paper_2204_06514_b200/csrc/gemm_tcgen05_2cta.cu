@@ -15,6 +15,8 @@
 // No TMA load uses cluster multicast.  Every wait is bounded.
 #include "gemm_common.cuh"
 
+#include <cstddef>
+
 namespace {
 
 using namespace tc;
@@ -216,6 +218,14 @@ gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
 
 }  // namespace
 
+bool fax_gemm_patch_info_2cta(const void* func, const void* param, size_t* size, size_t* sc_offset) {
+  if (func != (const void*)gemm_tcgen05_2cta_kernel) return false;
+  if (((const GemmParams*)param)->epi != EPI_ADAMW) return false;
+  *size = sizeof(GemmParams);
+  *sc_offset = offsetof(GemmParams, ad_sc);
+  return true;
+}
+
 bool fax_gemm_tc2_supported(const FaxGemm& g) { return g.M % 256 == 0 && g.N % 256 == 0 && g.K % BK == 0; }
 
 // Caller has already checked fax_gemm_tc_supported (alignment, strides).
@@ -227,11 +237,7 @@ fax_status fax_gemm_tc2(fax_ctx* ctx, const FaxGemm& g) {
                            : make_map(ctx, &mb, g.B, g.K, g.N, g.ldb, BK, BNH));
   if (!ok) return FAX_ERR_INVALID_ARG;
   GemmParams p;
-  p.M = g.M; p.N = g.N; p.K = g.K; p.a_mn = g.a_mn_major; p.b_mn = g.b_mn_major;
-  p.C = g.C; p.ldc = g.ldc; p.c_f32 = g.c_f32; p.accumulate = g.accumulate; p.epi = g.epi;
-  p.bias = (const bf16*)g.bias; p.resid = (const bf16*)g.resid; p.ldr = g.ldr; p.aux = (bf16*)g.aux; p.ldaux = g.ldaux;
-  p.alpha = g.alpha; p.status = ctx->dev_status;
-  p.group_m = 8;
+  fill_gemm_params(p, g, ctx->dev_status);
   static bool attr_set = false;
   if (!attr_set) {
     FAX_CUDA_TRY(ctx, cudaFuncSetAttribute(gemm_tcgen05_2cta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
@@ -239,17 +245,7 @@ fax_status fax_gemm_tc2(fax_ctx* ctx, const FaxGemm& g) {
   }
   const int tiles = (g.M / 256) * (g.N / 256);
   const int max_pairs = ctx->sm_count / 2;
-  p.splits = 1;
-  const int kb_total = g.K / BK;
-  if (g.c_f32 && g.epi == EPI_NONE && g.alpha == 1.f && tiles * 2 <= max_pairs && kb_total >= 16) {
-    int sp = max_pairs / tiles;
-    if (sp > kb_total / 8) sp = kb_total / 8;
-    if (sp > 16) sp = 16;
-    if (sp > 1) {
-      const int kb_per = (kb_total + sp - 1) / sp;
-      p.splits = (kb_total + kb_per - 1) / kb_per;
-    }
-  }
+  p.splits = gemm_split_count(g, tiles, max_pairs, BK);
   if (p.splits > 1 && !g.accumulate)
     FAX_CUDA_TRY(ctx, cudaMemset2DAsync(g.C, (size_t)g.ldc * 4, 0, (size_t)g.N * 4, (size_t)g.M, ctx->stream));
   const int items = tiles * p.splits;

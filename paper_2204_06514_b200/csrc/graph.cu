@@ -30,6 +30,14 @@ static fax_status patch_and_launch(fax_ctx* ctx, FaxGraphEntry& e, const fax_ada
     np.kernelParams = args;
     FAX_CUDA_TRY(ctx, cudaGraphExecKernelNodeSetParams(e.exec, e.adam_nodes[i], &np));
   }
+  // weight-gradient GEMMs with AdamW in their epilogue carry the scalars inside their parameter struct
+  for (FaxGemmPatch& g : e.gemm_nodes) {
+    memcpy(g.blob.data() + g.sc_offset, sc, 6 * sizeof(float));
+    cudaKernelNodeParams np = g.params;
+    void* args[3] = {np.kernelParams[0], np.kernelParams[1], g.blob.data()};
+    np.kernelParams = args;
+    FAX_CUDA_TRY(ctx, cudaGraphExecKernelNodeSetParams(e.exec, g.node, &np));
+  }
   FAX_CUDA_TRY(ctx, cudaGraphLaunch(e.exec, ctx->stream));
   ctx->launches += e.launches;
   e.last_use = ++ctx->graph_clock;
@@ -78,7 +86,15 @@ fax_status fax_run_step(fax_ctx* ctx, uint64_t key, const fax_adamw_hparams* hp,
         if (cudaGraphNodeGetType(nd, &t) != cudaSuccess || t != cudaGraphNodeTypeKernel) continue;
         cudaKernelNodeParams np;
         if (cudaGraphKernelNodeGetParams(nd, &np) != cudaSuccess) continue;
-        if (fax_adamw_is_kernel(np.func)) { e.adam_nodes.push_back(nd); e.adam_params.push_back(np); }
+        if (fax_adamw_is_kernel(np.func)) { e.adam_nodes.push_back(nd); e.adam_params.push_back(np); continue; }
+        size_t psize = 0, sc_off = 0;
+        if (np.kernelParams && (fax_gemm_patch_info_2cta(np.func, np.kernelParams[2], &psize, &sc_off) ||
+                                fax_gemm_patch_info_1cta(np.func, np.kernelParams[2], &psize, &sc_off))) {
+          FaxGemmPatch gp;
+          gp.node = nd; gp.params = np; gp.sc_offset = sc_off;
+          gp.blob.assign((const unsigned char*)np.kernelParams[2], (const unsigned char*)np.kernelParams[2] + psize);
+          e.gemm_nodes.push_back(gp);
+        }
       }
       e.graph = graph; e.exec = exec; e.launches = n_launch;
       return patch_and_launch(ctx, e, hp);

@@ -106,6 +106,7 @@ fax_status lm_fwd_bwd(fax_ctx* ctx, const fax_lm_cfg* c, const fax_lm_state* st,
     const int R = (N - r0) < w.head_rows ? (N - r0) : w.head_rows;
     const char* xf_rows = (const char*)sv.xf + (size_t)r0 * d * es;
     FaxGemm g;
+    g.adam = nullptr;
     g.alpha = 1.f; g.epi = EPI_NONE; g.bias = nullptr; g.resid = nullptr; g.ldr = 0; g.aux = nullptr; g.ldaux = 0;
     // logits = xf wte^T
     g.M = R; g.N = V; g.K = d;

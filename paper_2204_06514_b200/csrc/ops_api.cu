@@ -19,6 +19,7 @@ extern "C" fax_status fax_op_gemm(fax_ctx* ctx, int32_t prec, const fax_gemm_des
   g.C = d->C; g.ldc = d->ldc; g.c_f32 = d->c_f32 != 0; g.accumulate = d->accumulate != 0;
   g.epi = d->epilogue; g.bias = d->bias; g.resid = d->resid; g.ldr = d->ldr; g.aux = d->aux; g.ldaux = d->ldaux;
   g.alpha = d->alpha;
+  g.adam = nullptr;
   if (d->force_simt) return fax_gemm_simt(ctx, prec, g);
   return fax_gemm(ctx, prec, g);
 }

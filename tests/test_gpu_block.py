@@ -198,6 +198,55 @@ def test_graph_replay_patches_the_adamw_scalars(sess):
     assert st == fx.FAX_OK, detail
 
 
+@pytest.mark.parametrize("name", ["C1", "C2"])
+def test_fused_update_matches_separate_update(sess, name):
+    """AdamW in the epilogue of the weight-gradient GEMMs gives the weights of the separate update."""
+    cfg = synth.CONFIGS[name]
+    params = perturbed_block_params(cfg)
+    x, dy = synth.block_inputs(cfg)
+    hp = dict(synth.ADAMW)
+    wd = hp.pop("weight_decay")
+    mats = ("w_qkv", "w_o", "w_fc1", "w_fc2")
+    try:
+        runs = {}
+        for mode in ("separate", "fused_keep", "fused"):
+            fx.fax_set_fused_update(sess.ctx, mode != "separate", mode == "fused_keep")
+            r = BlockRunner(sess, cfg, params, fx.FAX_PREC_BF16, weight_decay=wd)
+            tx, tdy = r.to_device(x), r.to_device(dy)
+            r.step(tx, tdy, hparams(step=1, **hp))
+            torch.cuda.synchronize()
+            runs[mode] = r
+        a, b, c = runs["separate"], runs["fused_keep"], runs["fused"]
+        for k in O.PARAM_NAMES:
+            ga = host(a.p[k].g)
+            assert relerr(host(b.p[k].g), ga) <= 1e-3, k                 # gradients kept
+            if k in mats and name == "C1":                               # (C2's narrow shapes slice K: not fused)
+                assert float(c.p[k].g.abs().max()) == 0.0, k             # not materialised
+            # the update itself: oracle AdamW on this run's own gradient
+            w0 = params[k].astype(np.float64)
+            gb = host(b.p[k].g).reshape(w0.shape)
+            cw, cm, cv = O.adamw(w0, 0 * w0, 0 * w0, gb, weight_decay=wd, step=1, **hp)
+            assert relerr(host(b.p[k].w).reshape(w0.shape), cw) <= TOL_ADAMW, k
+            assert relerr(host(b.p[k].m).reshape(w0.shape), cm) <= TOL_ADAMW, k
+            assert relerr(host(b.p[k].v).reshape(w0.shape), cv) <= 1e-5, k
+            assert torch.equal(b.p[k].wc, b.p[k].w.to(torch.bfloat16)), k
+            assert torch.equal(c.p[k].wc, c.p[k].w.to(torch.bfloat16)), k
+            # moments are linear / quadratic in the gradient: all three runs agree
+            assert relerr(host(c.p[k].m), host(a.p[k].m)) <= 1e-3, k
+        # graph replay patches the scalars inside the fused GEMMs too: a step with lr = 0 freezes the weights
+        c.step(c.to_device(x), c.to_device(dy), hparams(step=2, **hp))
+        torch.cuda.synchronize()
+        w2 = {k: c.p[k].w.clone() for k in O.PARAM_NAMES}
+        c.step(c.to_device(x), c.to_device(dy), hparams(step=3, **dict(hp, lr=0.0)))
+        torch.cuda.synchronize()
+        for k in O.PARAM_NAMES:
+            assert torch.equal(c.p[k].w, w2[k]), k
+    finally:
+        fx.fax_set_fused_update(sess.ctx, False, False)
+    st, detail = fx.fax_check_device_status(sess.ctx)
+    assert st == fx.FAX_OK, detail
+
+
 def test_block_error_paths(sess):
     cfg = synth.CONFIGS["C1"]
     r = BlockRunner(sess, cfg, synth.block_params(cfg), fx.FAX_PREC_BF16)
