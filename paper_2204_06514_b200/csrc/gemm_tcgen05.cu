@@ -247,10 +247,44 @@ bool fax_gemm_tc_supported(const FaxGemm& g) {
   return true;
 }
 
+// A dimension that is 128 past a multiple of 256 (the vocabulary of the LM head): the two-CTA
+// kernel takes the multiple-of-256 part, the one-CTA kernel the last 128 rows or columns.
+static bool split_for_two_cta(fax_ctx* ctx, const FaxGemm& g, FaxGemm* main_part, FaxGemm* tail) {
+  if (!ctx->use_2cta || g.adam || g.K % 64) return false;
+  const size_t es = 2, cs = g.c_f32 ? 4 : 2;
+  if (g.M % 256 == 0 && g.N % 256 == 128 && g.N > 1024) {
+    const int n1 = g.N - 128;
+    *main_part = g; *tail = g;
+    main_part->N = n1; tail->N = 128;
+    tail->B = (const char*)g.B + (g.b_mn_major ? (size_t)n1 : (size_t)n1 * g.ldb) * es;
+    tail->C = (char*)g.C + (size_t)n1 * cs;
+    if (g.bias) tail->bias = (const char*)g.bias + (size_t)n1 * es;
+    if (g.resid) tail->resid = (const char*)g.resid + (size_t)n1 * es;
+    if (g.aux) tail->aux = (char*)g.aux + (size_t)n1 * es;
+    return true;
+  }
+  if (g.N % 256 == 0 && g.M % 256 == 128 && g.M > 1024) {
+    const int m1 = g.M - 128;
+    *main_part = g; *tail = g;
+    main_part->M = m1; tail->M = 128;
+    tail->A = (const char*)g.A + (g.a_mn_major ? (size_t)m1 : (size_t)m1 * g.lda) * es;
+    tail->C = (char*)g.C + (size_t)m1 * g.ldc * cs;
+    if (g.resid) tail->resid = (const char*)g.resid + (size_t)m1 * g.ldr * es;
+    if (g.aux) tail->aux = (char*)g.aux + (size_t)m1 * g.ldaux * es;
+    return true;
+  }
+  return false;
+}
+
 fax_status fax_gemm_tc(fax_ctx* ctx, const FaxGemm& g) {
   if (!fax_gemm_tc_supported(g)) return FAX_ERR_UNSUPPORTED_SHAPE;
   FaxProfScope prof(ctx, KC_GEMM_TC, 2.0 * g.M * g.N * g.K, 0.0);
   if (ctx->use_2cta && fax_gemm_tc2_supported(g)) return fax_gemm_tc2(ctx, g);
+  FaxGemm part, tail;
+  if (split_for_two_cta(ctx, g, &part, &tail) && fax_gemm_tc_supported(part) && fax_gemm_tc_supported(tail)) {
+    FAX_TRY(fax_gemm_tc2(ctx, part));
+    return launch<128>(ctx, tail);
+  }
   switch (pick_bn(g.N)) {
     case 256: return launch<256>(ctx, g);
     case 128: return launch<128>(ctx, g);

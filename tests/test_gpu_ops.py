@@ -97,7 +97,8 @@ def test_layernorm_forward_backward(sess, prec, rows, d):
     assert relerr(host(dg), rdg) <= tolg and relerr(host(db), rdb) <= tolg
 
 
-GEMM_SHAPES = [(128, 128, 64), (256, 384, 192), (100, 36, 50), (512, 1024, 2048), (384, 128, 4096 + 64)]
+GEMM_SHAPES = [(128, 128, 64), (256, 384, 192), (100, 36, 50), (512, 1024, 2048), (384, 128, 4096 + 64),
+               (256, 1408, 128), (1408, 256, 128)]       # the last two: 256-multiple part + 128 tail
 
 
 @pytest.mark.parametrize("prec", [0, 1])
