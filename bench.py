@@ -154,7 +154,8 @@ def oracle_sample(cfg, n_tokens: int):
     return cfg.tokens / full, cores, what
 
 
-SAMPLE_TOKENS = {"C1": 128, "C2": 512, "C3": 128, "C4": 128, "C5": 32}
+SAMPLE_TOKENS = {"C1": 128, "C2": 512, "C3": 128, "C4": 128, "C5": 32, "P1": 128, "P2": 32, "P3": 16,
+                 "F3": 128, "F2": 128}
 
 
 def run_reference(args):
@@ -310,6 +311,21 @@ def run_ours(args):
     prof = fx.fax_profile_end(sess.ctx)
     fx.fax_set_adamw_overlap(sess.ctx, True)
 
+    # per-phase split (the paper's Fig. 3 reports forward, loss and backward separately): the phase
+    # entry points timed on their own, outside the step's timed region
+    ph_steps = max(1, min(args.steps, 5))
+    if cfg.is_lm:
+        fb = timed(lambda: runner.forward_backward(ids, tg), ph_steps) / ph_steps
+        phases = {"forward_loss_backward_ms": fb, "adamw_ms": max(ms / args.steps - fb, 0.0),
+                  "note": "forward + loss + backward through fax_lm_forward_backward; AdamW = step - that"}
+    else:
+        hp_ph = hparams(step=1, **hp0)
+        fwd = timed(lambda: runner.forward(x), ph_steps) / ph_steps
+        bwd = timed(lambda: runner.backward(dy), ph_steps) / ph_steps
+        adw = timed(lambda: runner.adamw(hp_ph), ph_steps) / ph_steps
+        phases = {"forward_ms": fwd, "backward_ms": bwd, "adamw_ms": adw,
+                  "note": "fax_block_forward, fax_block_backward, fax_adamw_step timed separately"}
+
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -355,7 +371,7 @@ def run_ours(args):
                 "vs_nominal_2250": achieved_tf / NOMINAL_BF16_TFLOPS,
                 "vs_measured_sustained": achieved_tf / peaks["bf16_tflops_sustained"],
                 "flops_convention": "6*matmul_params*tokens + causal-halved attention (6*B*T^2*d per layer)"},
-        "roofline": roofline, "kernels": kernels,
+        "roofline": roofline, "kernels": kernels, "phases": phases,
         "cpu_baseline": {"value": cpu_val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what},
         "e2e": {"value": dist_util.whole_job_rate(tokens, world, ms_e2e / e2e_steps), "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
@@ -372,7 +388,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--config", default="C3", choices=["C1", "C2", "C3", "C4", "C5"])
+    ap.add_argument("--config", default="C3", choices=["C1", "C2", "C3", "C4", "C5", "P1", "P2", "P3", "F3", "F2"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--fused-update", default="off", choices=["off", "keep", "nograd"],
                     help="AdamW of the weight matrices in the dW GEMM epilogue: off; on and the gradients still "

@@ -92,6 +92,19 @@ CONFIGS = {
     "C5": Config("C5", 4, batch=1, seq=2048, d_model=12288, n_heads=96, head_dim=128, d_ff=49152),
 }
 
+# Paper-shaped workloads beyond the five benchmark configs (same kernels): Table 1's hidden sizes at
+# batch 1 x seq 2048 (head_dim 128, FFN 4 d: the paper gives neither), Fig. 3's 124M model at
+# batch 32 x seq 2048, and a 350M-class 24-layer LM (the model size of Fig. 2).
+CONFIGS.update({
+    "P1": Config("P1", 5, batch=1, seq=2048, d_model=5120, n_heads=40, head_dim=128, d_ff=20480),
+    "P2": Config("P2", 6, batch=1, seq=2048, d_model=10240, n_heads=80, head_dim=128, d_ff=40960),
+    "P3": Config("P3", 7, batch=1, seq=2048, d_model=16384, n_heads=128, head_dim=128, d_ff=65536),
+    "F3": Config("F3", 8, batch=32, seq=2048, d_model=768, n_heads=12, head_dim=64, d_ff=3072,
+                 n_layers=12, vocab=50304),
+    "F2": Config("F2", 9, batch=16, seq=1024, d_model=1024, n_heads=16, head_dim=64, d_ff=4096,
+                 n_layers=24, vocab=50304),
+})
+
 ADAMW = dict(lr=1e-3, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.1)
 
 # fixed tensor-id enumeration
