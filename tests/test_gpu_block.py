@@ -314,3 +314,56 @@ def test_lm_bf16_c4_shape_reduced(sess):
     # C4's widths and full vocabulary (d 768, 12 x 64, FFN 3072, V 50304), 2 layers, 2 x 128 tokens
     cfg = synth.scaled(synth.CONFIGS["C4"], batch=2, seq=128, n_layers=2)
     lm_case(sess, cfg, fx.FAX_PREC_BF16, synth.lm_params(cfg))
+
+
+def test_lm_three_steps_and_resume_fp32(sess):
+    """Three consecutive LM steps in the float32 validation mode follow the oracle's trajectory (loss,
+    weights, moments), and a run resumed from copied-out state (w, m, v, step) continues identically."""
+    cfg = synth.Config("lm_multi", 10, batch=2, seq=6, d_model=16, n_heads=2, head_dim=8, d_ff=32, n_layers=2, vocab=13)
+    lm = synth.lm_params(cfg)
+    for l in range(cfg.n_layers):
+        lm["blocks"][l] = perturbed_block_params(cfg, l)
+    lm["wte"] *= 10; lm["wpe"] *= 10
+    ids, tg = synth.lm_tokens(cfg)
+    B, T, H, hd = cfg.batch, cfg.seq, cfg.n_heads, cfg.head_dim
+    hp = dict(synth.ADAMW)
+    wd = hp.pop("weight_decay")
+    names = [n for n, _ in O.lm_tensors(lm)]
+    # warm optimizer state keeps the update smooth in the gradient (no first-step sign function)
+    m0 = {n: synth.warm_state(cfg.seed, i, a.shape, 1e-2)[0] for i, (n, a) in enumerate(O.lm_tensors(lm))}
+    v0 = {n: synth.warm_state(cfg.seed, i, a.shape, 1e-2)[1] for i, (n, a) in enumerate(O.lm_tensors(lm))}
+
+    def unflatten(flat):
+        return dict(wte=flat["wte"], wpe=flat["wpe"], lnf_g=flat["lnf_g"], lnf_b=flat["lnf_b"],
+                    blocks=[{k: flat[f"blocks.{l}.{k}"] for k in O.PARAM_NAMES} for l in range(cfg.n_layers)])
+
+    def set_state(r, w, m, v):
+        for n, ps in r.named_params():
+            ps.w.copy_(torch.as_tensor(np.asarray(w[n], dtype=np.float32)))
+            ps.m.copy_(torch.as_tensor(np.asarray(m[n], dtype=np.float32)))
+            ps.v.copy_(torch.as_tensor(np.asarray(v[n], dtype=np.float32)))
+
+    w = {n: a.astype(np.float64) for n, a in O.lm_tensors(lm)}
+    m, v = dict(m0), dict(v0)
+    r = LmRunner(sess, cfg, lm, fx.FAX_PREC_FP32_VALIDATE, weight_decay=wd)
+    set_state(r, w, m, v)
+    tids, ttg = torch.as_tensor(ids).to(sess.device), torch.as_tensor(tg).to(sess.device)
+    snap = None
+    for step in (5, 6, 7):
+        loss_ref, _, w, m, v = O.lm_step(ids, tg, unflatten(w), m, v, B, T, H, hd,
+                                         dict(weight_decay=wd, step=step, **hp), cfg.ln_eps)
+        loss = r.step(tids, ttg, hparams(step=step, **hp), want_host_loss=True)
+        assert abs(loss - loss_ref) <= TOL_FP32 * abs(loss_ref), step
+        for n, ps in r.named_params():
+            assert relerr(host(ps.w).reshape(w[n].shape), w[n]) <= TOL_FP32, (step, n)
+            assert relerr(host(ps.m).reshape(w[n].shape), m[n]) <= TOL_FP32, (step, n)
+        if step == 6:
+            snap = {n: (ps.w.clone(), ps.m.clone(), ps.v.clone()) for n, ps in r.named_params()}
+    # resume: a fresh runner given the state after step 6 reproduces step 7 bit for bit
+    r2 = LmRunner(sess, cfg, lm, fx.FAX_PREC_FP32_VALIDATE, weight_decay=wd)
+    for n, ps in r2.named_params():
+        ps.w.copy_(snap[n][0]); ps.m.copy_(snap[n][1]); ps.v.copy_(snap[n][2])
+    loss2 = r2.step(tids, ttg, hparams(step=7, **hp), want_host_loss=True)
+    assert loss2 == loss
+    for (n, a), (_, b) in zip(r.named_params(), r2.named_params()):
+        assert torch.equal(a.w, b.w), n
