@@ -164,15 +164,21 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnFwdParams
       for (int c = 0; c < 4; ++c) tc_ld32(tmem + lane_base + (uint32_t)(sb * 128 + 32 * c), sv[c]);
       tc_wait_ld();
       const bool diag = (j == qi);
-      float mx = -INFINITY;
+      if (diag) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+#pragma unroll
+          for (int e = 0; e < 32; ++e)
+            if (32 * c + e > r) sv[c][e] = 0xff800000u;      // -inf
+      }
+      // three-input max, four independent chains (the two-input form is the slowest part of the tile)
+      float mxa[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
       for (int c = 0; c < 4; ++c)
 #pragma unroll
-        for (int e = 0; e < 32; ++e) {
-          float s = __uint_as_float(sv[c][e]);
-          if (diag && (32 * c + e > r)) { s = -INFINITY; sv[c][e] = __float_as_uint(s); }
-          mx = fmaxf(mx, s);
-        }
+        for (int e = 0; e < 32; e += 2)
+          mxa[(e >> 1) & 3] = max3(mxa[(e >> 1) & 3], __uint_as_float(sv[c][e]), __uint_as_float(sv[c][e + 1]));
+      const float mx = fmaxf(fmaxf(mxa[0], mxa[1]), fmaxf(mxa[2], mxa[3]));
       const float m_new = fmaxf(m_used, mx * p.scale_log2);
       bool odone_waited = false;
       if (__any_sync(0xffffffffu, m_new > m_used + 8.0f)) {
