@@ -366,4 +366,7 @@ def test_lm_three_steps_and_resume_fp32(sess):
     loss2 = r2.step(tids, ttg, hparams(step=7, **hp), want_host_loss=True)
     assert loss2 == loss
     for (n, a), (_, b) in zip(r.named_params(), r2.named_params()):
-        assert torch.equal(a.w, b.w), n
+        if n == "wte":        # its gradient includes the embedding scatter: float atomics, arrival order
+            assert relerr(host(b.w), host(a.w)) <= 1e-6
+        else:
+            assert torch.equal(a.w, b.w), n
