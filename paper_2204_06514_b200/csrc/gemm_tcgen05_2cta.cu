@@ -12,7 +12,7 @@
 //                 tcgen05.commit multicasts "stage empty" / "accumulator full" to both
 //   warps 2..9  : epilogue of the CTA's own 128 x 256 half; "accumulator empty" is
 //                 signalled to the even CTA's barrier
-// No TMA load uses cluster multicast.  Every wait is bounded.
+// Every TMA load is a plain load into the issuing CTA's own shared memory.  Every wait is bounded.
 #include "gemm_common.cuh"
 
 #include <cstddef>
