@@ -226,6 +226,75 @@ layernorm_bwd_dx_warp_kernel(int rows, int d, const T* __restrict__ da, const T*
   }
 }
 
+// Backward dx with G warps per row (rows of more than 256 vectors): a lane holds at most 8
+// vectors of da and of x, which keeps the kernel at 3 to 4 blocks per SM; the G partial sums of
+// a row meet in shared memory behind a barrier of just those warps.
+template <typename T, int VPT, int G>
+__global__ void __launch_bounds__(256)
+layernorm_bwd_dx_group_kernel(int rows, int d, const T* __restrict__ da, const T* __restrict__ x,
+                              const float* __restrict__ mu_in, const float* __restrict__ rstd_in,
+                              const T* __restrict__ gamma, const T* __restrict__ add, T* __restrict__ dx) {
+  constexpr int VN = Vec<T>::N;
+  constexpr int RG = 8 / G;
+  __shared__ float2 red[8];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int rg = warp / G, gw = warp % G;
+  const int nvec = d / VN;
+  const int row = blockIdx.x * RG + rg;
+  const bool live = row < rows;
+  uint4 rda[VPT], rx[VPT];
+  float mu = 0.f, rstd = 0.f, s1 = 0.f, s2 = 0.f;
+  if (live) {
+    const uint4* dar = reinterpret_cast<const uint4*>(da + (size_t)row * d);
+    const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)row * d);
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+      const int vi = lane + 32 * (i + VPT * gw);
+      if (vi < nvec) { rda[i] = dar[vi]; rx[i] = xr[vi]; }
+    }
+    mu = mu_in[row]; rstd = rstd_in[row];
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+      const int vi = lane + 32 * (i + VPT * gw);
+      if (vi < nvec) {
+        float fd[VN], fx[VN], g[VN];
+        unpack<T>(rda[i], fd); unpack<T>(rx[i], fx);
+        load_vec<T>(gamma + vi * VN, g);
+#pragma unroll
+        for (int j = 0; j < VN; ++j) { const float u = fd[j] * g[j]; s1 += u; s2 += u * (fx[j] - mu) * rstd; }
+      }
+    }
+    s1 = warp_sum(s1); s2 = warp_sum(s2);
+  }
+  if (G > 1) {
+    if (lane == 0) red[warp] = make_float2(s1, s2);
+    __syncthreads();
+    s1 = 0.f; s2 = 0.f;
+#pragma unroll
+    for (int k = 0; k < G; ++k) { s1 += red[rg * G + k].x; s2 += red[rg * G + k].y; }
+  }
+  if (!live) return;
+  const float c1 = s1 / (float)d, c2 = s2 / (float)d;
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) {
+    const int vi = lane + 32 * (i + VPT * gw);
+    if (vi < nvec) {
+      float fd[VN], fx[VN], g[VN], o[VN];
+      unpack<T>(rda[i], fd); unpack<T>(rx[i], fx);
+      load_vec<T>(gamma + vi * VN, g);
+#pragma unroll
+      for (int j = 0; j < VN; ++j) o[j] = rstd * (fd[j] * g[j] - c1 - (fx[j] - mu) * rstd * c2);
+      if (add) {
+        float av[VN];
+        load_vec<T>(add + (size_t)row * d + vi * VN, av);
+#pragma unroll
+        for (int j = 0; j < VN; ++j) o[j] += av[j];
+      }
+      store_vec<T>(dx + (size_t)row * d + vi * VN, o);
+    }
+  }
+}
+
 // Backward dx, one block per row (wide rows).
 template <typename T, int VPT>
 __global__ void __launch_bounds__(512)
@@ -399,6 +468,12 @@ template <typename T>
 fax_status ln_bwd_dx_t(fax_ctx* ctx, int rows, int d, const void* da, const void* x, const float* mu,
                        const float* rstd, const void* gamma, const void* add, void* dx) {
   const int nvec = d / Vec<T>::N;
+  if (nvec > 256 && nvec <= 512) {
+    // two warps per row, 8 vectors per lane
+    layernorm_bwd_dx_group_kernel<T, 8, 2><<<(rows + 3) / 4, 256, 0, ctx->stream>>>(
+        rows, d, (const T*)da, (const T*)x, mu, rstd, (const T*)gamma, (const T*)add, (T*)dx);
+    return fax_after_launch(ctx);
+  }
   if (nvec <= 512) {
     const int need = (nvec + 31) / 32;
 #define LN_BWDW(V)                                                                                      \
