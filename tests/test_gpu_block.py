@@ -370,3 +370,41 @@ def test_lm_three_steps_and_resume_fp32(sess):
             assert relerr(host(b.w), host(a.w)) <= 1e-6
         else:
             assert torch.equal(a.w, b.w), n
+
+
+def test_lm_and_adamw_error_paths(sess):
+    cfg = synth.Config("lm_err", 11, batch=2, seq=128, d_model=128, n_heads=2, head_dim=64, d_ff=256, n_layers=1, vocab=256)
+    lm = synth.lm_params(cfg)
+    r = LmRunner(sess, cfg, lm, fx.FAX_PREC_BF16)
+    ids, tg = synth.lm_tokens(cfg)
+    tids, ttg = torch.as_tensor(ids).to(sess.device), torch.as_tensor(tg).to(sess.device)
+    hp = dict(synth.ADAMW); hp.pop("weight_decay")
+    # step < 1
+    with pytest.raises(fx.FaxError) as e:
+        r.step(tids, ttg, hparams(step=0, **hp))
+    assert e.value.status == fx.FAX_ERR_INVALID_ARG
+    # scratch arena too small
+    import ctypes as C
+    small = fx.LmState.from_buffer_copy(r.state)
+    small.scratch_bytes = 1024
+    with pytest.raises(fx.FaxError) as e:
+        fx.fax_lm_forward_backward(sess.ctx, r.lcfg, small, ptr(tids), ptr(ttg), ptr(r.loss))
+    assert e.value.status == fx.FAX_ERR_WORKSPACE_TOO_SMALL
+    # vocabulary that the bf16 tiles do not divide
+    bad = fx.LmCfg(1, 250, 128, r.lcfg.block)
+    with pytest.raises(fx.FaxError) as e:
+        fx.fax_lm_sizes(bad)
+    assert e.value.status == fx.FAX_ERR_UNSUPPORTED_SHAPE
+    # AdamW: misaligned pointer, bad beta
+    w = torch.zeros(1024, device=sess.device)
+    t = fx.AdamwTensor(C.c_void_p(w.data_ptr() + 4), ptr(w), ptr(w), ptr(w), None, 8, 0.0)
+    with pytest.raises(fx.FaxError) as e:
+        fx.fax_adamw_step(sess.ctx, [t], hparams(step=1, **hp))
+    assert e.value.status == fx.FAX_ERR_INVALID_ARG
+    t = fx.AdamwTensor(ptr(w), ptr(w), ptr(w), ptr(w), None, 8, 0.0)
+    with pytest.raises(fx.FaxError):
+        fx.fax_adamw_step(sess.ctx, [t], hparams(step=1, **dict(hp, beta1=1.0)))
+    # the context is still usable afterwards
+    r.step(tids, ttg, hparams(step=1, **hp))
+    st, _ = fx.fax_check_device_status(sess.ctx)
+    assert st == fx.FAX_OK and torch.isfinite(r.loss).all()
