@@ -274,6 +274,20 @@ fax_status fax_lm_step(fax_ctx* ctx, const fax_lm_cfg* cfg, const fax_lm_state* 
 fax_status fax_lm_forward_backward(fax_ctx* ctx, const fax_lm_cfg* cfg, const fax_lm_state* st,
                                    const int32_t* ids, const int32_t* targets, float* loss_device);
 
+/* Gradient accumulation over micro-batches: forward + loss + backward of one
+ * micro-batch, its gradients scaled by grad_scale (normally 1 / number of
+ * micro-batches: the loss of each call is the mean over its own batch*seq
+ * tokens) and written (accumulate = 0) or added (accumulate != 0) to st->...g.
+ * loss_device receives this micro-batch's unscaled mean loss.  After the last
+ * micro-batch fax_lm_apply_adamw updates every tensor from the accumulated
+ * gradients.  k calls on k micro-batches followed by fax_lm_apply_adamw equal
+ * one fax_lm_step on the concatenated batch. */
+fax_status fax_lm_accumulate(fax_ctx* ctx, const fax_lm_cfg* cfg, const fax_lm_state* st,
+                             const int32_t* ids, const int32_t* targets, float* loss_device,
+                             int32_t accumulate, float grad_scale);
+fax_status fax_lm_apply_adamw(fax_ctx* ctx, const fax_lm_cfg* cfg, const fax_lm_state* st,
+                              const fax_adamw_hparams* hp);
+
 /* Same as fax_lm_step with HOST ids / targets (int32 [batch, seq], pinned
  * recommended): copies them into the head of the scratch arena, runs the
  * step, copies the loss back and synchronises. */

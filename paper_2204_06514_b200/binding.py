@@ -116,6 +116,8 @@ _SIGNATURES = {
     "fax_lm_step": (C.c_int32, [_P, C.POINTER(LmCfg), C.POINTER(LmState), _P, _P, C.POINTER(AdamwHparams),
                                 _P, C.POINTER(C.c_float)]),
     "fax_lm_forward_backward": (C.c_int32, [_P, C.POINTER(LmCfg), C.POINTER(LmState), _P, _P, _P]),
+    "fax_lm_accumulate": (C.c_int32, [_P, C.POINTER(LmCfg), C.POINTER(LmState), _P, _P, _P, C.c_int32, C.c_float]),
+    "fax_lm_apply_adamw": (C.c_int32, [_P, C.POINTER(LmCfg), C.POINTER(LmState), C.POINTER(AdamwHparams)]),
     "fax_lm_step_host": (C.c_int32, [_P, C.POINTER(LmCfg), C.POINTER(LmState), _P, _P,
                                      C.POINTER(AdamwHparams), _P, C.POINTER(C.c_float)]),
 }
@@ -294,6 +296,15 @@ def fax_lm_step(ctx, cfg, st, ids, targets, hp, loss_device, want_host_loss=Fals
 def fax_lm_forward_backward(ctx, cfg, st, ids, targets, loss_device):
     _check(load_library().fax_lm_forward_backward(ctx, C.byref(cfg), C.byref(st), ids, targets, loss_device),
            "fax_lm_forward_backward")
+
+
+def fax_lm_accumulate(ctx, cfg, st, ids, targets, loss_device, accumulate: bool, grad_scale: float):
+    _check(load_library().fax_lm_accumulate(ctx, C.byref(cfg), C.byref(st), ids, targets, loss_device,
+                                            int(bool(accumulate)), grad_scale), "fax_lm_accumulate")
+
+
+def fax_lm_apply_adamw(ctx, cfg, st, hp):
+    _check(load_library().fax_lm_apply_adamw(ctx, C.byref(cfg), C.byref(st), C.byref(hp)), "fax_lm_apply_adamw")
 
 
 def fax_lm_step_host(ctx, cfg, st, ids_host, targets_host, hp, loss_device) -> float:

@@ -234,7 +234,7 @@ fax_status fax_attention_bwd_simt(fax_ctx* ctx, int prec, int B, int T, int H, i
 fax_status fax_embed_fwd(fax_ctx* ctx, int prec, int B, int T, int d, int vocab, const int32_t* ids,
                          const void* wte, const void* wpe, void* x0);
 fax_status fax_embed_bwd(fax_ctx* ctx, int prec, int B, int T, int max_seq, int d, int vocab,
-                         const int32_t* ids, const void* dx0, float* dwte, float* dwpe);
+                         const int32_t* ids, const void* dx0, float* dwte, float* dwpe, bool accumulate_wpe);
 fax_status fax_xent(fax_ctx* ctx, int prec, int rows, int vocab, void* logits, int64_t ld,
                     const int32_t* targets, float inv_n, float* row_loss);
 fax_status fax_loss_mean(fax_ctx* ctx, int n, const float* row_loss, float* loss);

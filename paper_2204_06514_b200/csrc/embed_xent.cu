@@ -30,13 +30,13 @@ __global__ void embed_bwd_wte_kernel(int n_tok, int d, int vocab, const int32_t*
 // dwpe[t] = sum_b dx0[b, t]   (fixed order: deterministic); rows t >= Tn are zeroed
 template <typename T>
 __global__ void embed_bwd_wpe_kernel(int Bn, int Tn, int max_seq, int d, const T* __restrict__ dx0,
-                                     float* __restrict__ dwpe) {
+                                     float* __restrict__ dwpe, int accumulate) {
   int t = blockIdx.x;
   for (int c = threadIdx.x; c < d; c += blockDim.x) {
     float s = 0.f;
     if (t < Tn)
       for (int b = 0; b < Bn; ++b) s += to_f32(dx0[((size_t)b * Tn + t) * d + c]);
-    dwpe[(size_t)t * d + c] = s;
+    dwpe[(size_t)t * d + c] = accumulate ? dwpe[(size_t)t * d + c] + s : s;
   }
 }
 
@@ -176,17 +176,17 @@ fax_status fax_embed_fwd(fax_ctx* ctx, int prec, int B, int T, int d, int vocab,
 }
 
 fax_status fax_embed_bwd(fax_ctx* ctx, int prec, int B, int T, int max_seq, int d, int vocab,
-                         const int32_t* ids, const void* dx0, float* dwte, float* dwpe) {
+                         const int32_t* ids, const void* dx0, float* dwte, float* dwpe, bool accumulate_wpe) {
   int n = B * T;
   FaxProfScope prof(ctx, KC_EMBED, 0.0, (double)n * d * (2.0 * fax_elem_size(prec) + 8.0));
   if (prec == FAX_PREC_BF16) {
     embed_bwd_wte_kernel<bf16><<<n, 128, 0, ctx->stream>>>(n, d, vocab, ids, (const bf16*)dx0, dwte);
     FAX_TRY(fax_after_launch(ctx));
-    embed_bwd_wpe_kernel<bf16><<<max_seq, 128, 0, ctx->stream>>>(B, T, max_seq, d, (const bf16*)dx0, dwpe);
+    embed_bwd_wpe_kernel<bf16><<<max_seq, 128, 0, ctx->stream>>>(B, T, max_seq, d, (const bf16*)dx0, dwpe, accumulate_wpe ? 1 : 0);
   } else {
     embed_bwd_wte_kernel<float><<<n, 128, 0, ctx->stream>>>(n, d, vocab, ids, (const float*)dx0, dwte);
     FAX_TRY(fax_after_launch(ctx));
-    embed_bwd_wpe_kernel<float><<<max_seq, 128, 0, ctx->stream>>>(B, T, max_seq, d, (const float*)dx0, dwpe);
+    embed_bwd_wpe_kernel<float><<<max_seq, 128, 0, ctx->stream>>>(B, T, max_seq, d, (const float*)dx0, dwpe, accumulate_wpe ? 1 : 0);
   }
   return fax_after_launch(ctx);
 }

@@ -81,7 +81,7 @@ fax_status lm_check_state(const fax_lm_cfg* c, const fax_lm_state* st) {
 
 fax_status lm_fwd_bwd(fax_ctx* ctx, const fax_lm_cfg* c, const fax_lm_state* st, const int32_t* ids,
                       const int32_t* targets, float* loss_device, const LmSaved& sv, const LmScratch& w,
-                      const fax_adamw_hparams* hp) {
+                      const fax_adamw_hparams* hp, bool acc = false, float grad_scale = 1.f) {
   const fax_block_cfg* bc = &c->block;
   const int prec = bc->prec, L = c->n_layers;
   const int N = bc->batch * bc->seq, d = bc->d_model, V = c->vocab;
@@ -114,7 +114,7 @@ fax_status lm_fwd_bwd(fax_ctx* ctx, const fax_lm_cfg* c, const fax_lm_state* st,
     g.B = wte; g.ldb = d; g.b_mn_major = false;
     g.C = w.logits; g.ldc = V; g.c_f32 = false; g.accumulate = false;
     FAX_TRY(fax_gemm(ctx, prec, g));
-    FAX_TRY(fax_xent(ctx, prec, R, V, w.logits, V, targets + r0, 1.0f / (float)N, w.row_loss + r0));
+    FAX_TRY(fax_xent(ctx, prec, R, V, w.logits, V, targets + r0, grad_scale / (float)N, w.row_loss + r0));
     // dxf = dlogits wte
     g.M = R; g.N = d; g.K = V;
     g.A = w.logits; g.lda = V; g.a_mn_major = false;
@@ -125,7 +125,7 @@ fax_status lm_fwd_bwd(fax_ctx* ctx, const fax_lm_cfg* c, const fax_lm_state* st,
     g.M = V; g.N = d; g.K = R;
     g.A = w.logits; g.lda = V; g.a_mn_major = true;
     g.B = xf_rows; g.ldb = d; g.b_mn_major = true;
-    g.C = st->wte.g; g.ldc = d; g.c_f32 = true; g.accumulate = (r0 != 0);
+    g.C = st->wte.g; g.ldc = d; g.c_f32 = true; g.accumulate = acc || (r0 != 0);
     FAX_TRY(fax_gemm(ctx, prec, g));
   }
   FAX_TRY(fax_loss_mean(ctx, N, w.row_loss, loss_device));
@@ -133,7 +133,7 @@ fax_status lm_fwd_bwd(fax_ctx* ctx, const fax_lm_cfg* c, const fax_lm_state* st,
   // backward through the final LayerNorm and the blocks
   void* dcur = w.dxb;
   FAX_TRY(fax_layernorm_bwd(ctx, prec, N, d, dxf, sv.act[L], sv.muf, sv.rstdf, lnf_g, nullptr, dcur,
-                            st->lnf_g.g, st->lnf_b.g, false, w.blk.partial, w.blk.partial_floats));
+                            st->lnf_g.g, st->lnf_b.g, acc, w.blk.partial, w.blk.partial_floats));
   void* dnext = w.dxa;
   for (int l = L - 1; l >= 0; --l) {
     fax_block_params p; fax_block_grads g;
@@ -141,12 +141,12 @@ fax_status lm_fwd_bwd(fax_ctx* ctx, const fax_lm_cfg* c, const fax_lm_state* st,
     fax_adamw_tensor t12[12];
     FaxAdamHook hook = {t12, hp};
     if (hp) fax_layer_adamw_tensors(&st->layers[l], prec, t12);
-    FAX_TRY(fax_block_backward_impl(ctx, bc, &p, dcur, sv.blk[l], sv.act[l], dnext, &g, false, w.blk,
+    FAX_TRY(fax_block_backward_impl(ctx, bc, &p, dcur, sv.blk[l], sv.act[l], dnext, &g, acc, w.blk,
                                     hp ? &hook : nullptr));
     void* t = dcur; dcur = dnext; dnext = t;
   }
   // embedding gradients: scatter into the tied dwte, batch-sum into dwpe
-  return fax_embed_bwd(ctx, prec, bc->batch, bc->seq, c->max_seq, d, V, ids, dcur, st->wte.g, st->wpe.g);
+  return fax_embed_bwd(ctx, prec, bc->batch, bc->seq, c->max_seq, d, V, ids, dcur, st->wte.g, st->wpe.g, acc);
 }
 
 // AdamW of the tensors that are not inside a block (the blocks' tensors are updated under backward).
@@ -229,6 +229,36 @@ extern "C" fax_status fax_lm_forward_backward(fax_ctx* ctx, const fax_lm_cfg* cf
                                               const int32_t* ids, const int32_t* targets, float* loss_device) {
   if (!ctx || !ids || !targets) return FAX_ERR_INVALID_ARG;
   return lm_run(ctx, cfg, st, ids, targets, nullptr, loss_device, nullptr, nullptr);
+}
+
+extern "C" fax_status fax_lm_accumulate(fax_ctx* ctx, const fax_lm_cfg* cfg, const fax_lm_state* st,
+                                        const int32_t* ids, const int32_t* targets, float* loss_device,
+                                        int32_t accumulate, float grad_scale) {
+  if (!ctx || !ids || !targets || !loss_device) return FAX_ERR_INVALID_ARG;
+  FAX_TRY(lm_validate(cfg));
+  FAX_TRY(lm_check_state(cfg, st));
+  FaxArena ar(st->saved, st->saved_bytes), aw(st->scratch, st->scratch_bytes);
+  LmSaved sv; LmScratch w;
+  carve_saved(cfg, ar, &sv);
+  carve_scratch(cfg, aw, &w);
+  if (ar.used() > st->saved_bytes || aw.used() > st->scratch_bytes) return FAX_ERR_WORKSPACE_TOO_SMALL;
+  return lm_fwd_bwd(ctx, cfg, st, ids, targets, loss_device, sv, w, nullptr, accumulate != 0, grad_scale);
+}
+
+extern "C" fax_status fax_lm_apply_adamw(fax_ctx* ctx, const fax_lm_cfg* cfg, const fax_lm_state* st,
+                                         const fax_adamw_hparams* hp) {
+  if (!ctx || !hp || hp->step < 1) return FAX_ERR_INVALID_ARG;
+  FAX_TRY(lm_validate(cfg));
+  FAX_TRY(lm_check_state(cfg, st));
+  fax_adamw_hparams h = *hp;
+  h.grad_is_bf16 = 0;
+  const int prec = cfg->block.prec;
+  for (int l = 0; l < cfg->n_layers; ++l) {
+    fax_adamw_tensor t12[12];
+    fax_layer_adamw_tensors(&st->layers[l], prec, t12);
+    FAX_TRY(fax_adamw_launch(ctx, t12, 12, &h));
+  }
+  return lm_adamw(ctx, cfg, st, &h);
 }
 
 extern "C" fax_status fax_lm_step(fax_ctx* ctx, const fax_lm_cfg* cfg, const fax_lm_state* st,

@@ -153,6 +153,13 @@ class LmRunner:
         return fx.fax_lm_step(self.sess.ctx, self.lcfg, self.state, _ptr(ids), _ptr(targets), hp,
                               _ptr(self.loss), want_host_loss)
 
+    def accumulate(self, ids, targets, accumulate: bool, grad_scale: float):
+        fx.fax_lm_accumulate(self.sess.ctx, self.lcfg, self.state, _ptr(ids), _ptr(targets), _ptr(self.loss),
+                             accumulate, grad_scale)
+
+    def apply_adamw(self, hp):
+        fx.fax_lm_apply_adamw(self.sess.ctx, self.lcfg, self.state, hp)
+
     def step_host(self, ids_host, targets_host, hp) -> float:
         return fx.fax_lm_step_host(self.sess.ctx, self.lcfg, self.state, _ptr(ids_host), _ptr(targets_host),
                                    hp, _ptr(self.loss))

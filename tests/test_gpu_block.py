@@ -408,3 +408,42 @@ def test_lm_and_adamw_error_paths(sess):
     r.step(tids, ttg, hparams(step=1, **hp))
     st, _ = fx.fax_check_device_status(sess.ctx)
     assert st == fx.FAX_OK and torch.isfinite(r.loss).all()
+
+
+@pytest.mark.parametrize("prec", [fx.FAX_PREC_FP32_VALIDATE, fx.FAX_PREC_BF16])
+def test_lm_gradient_accumulation_equals_the_big_batch(sess, prec):
+    """Two micro-batches accumulated with grad_scale 1/2, then fax_lm_apply_adamw == one step on the whole batch."""
+    if prec == fx.FAX_PREC_BF16:
+        big = synth.Config("lm_acc", 12, batch=4, seq=128, d_model=128, n_heads=2, head_dim=64, d_ff=256, n_layers=2, vocab=256)
+    else:
+        big = synth.Config("lm_acc32", 13, batch=4, seq=6, d_model=16, n_heads=2, head_dim=8, d_ff=32, n_layers=2, vocab=13)
+    half = synth.scaled(big, batch=2)
+    lm = synth.lm_params(big)
+    ids, tg = synth.lm_tokens(big)
+    B, T, H, hd = big.batch, big.seq, big.n_heads, big.head_dim
+    rnd = (lambda a: synth.round_to_bf16(a).astype(np.float64)) if prec == 0 else (lambda a: a.astype(np.float64))
+    lmc = dict(wte=rnd(lm["wte"]), wpe=rnd(lm["wpe"]), lnf_g=rnd(lm["lnf_g"]), lnf_b=rnd(lm["lnf_b"]),
+               blocks=[{k: rnd(v) for k, v in p.items()} for p in lm["blocks"]])
+    rloss, rg = O.lm_forward_backward(ids, tg, lmc, B, T, H, hd, big.ln_eps)
+    rg = dict(O.lm_tensors(rg))
+    hp = dict(synth.ADAMW)
+    wd = hp.pop("weight_decay")
+    r = LmRunner(sess, half, lm, prec, weight_decay=wd)
+    dev = lambda a: torch.as_tensor(np.ascontiguousarray(a)).to(sess.device)
+    r.accumulate(dev(ids[:2]), dev(tg[:2]), False, 0.5)
+    l0 = float(r.loss.item())
+    r.accumulate(dev(ids[2:]), dev(tg[2:]), True, 0.5)
+    l1 = float(r.loss.item())
+    tol_f = TOL_FWD_BF16 if prec == 0 else TOL_FP32
+    tol_g = TOL_GRAD_BF16 if prec == 0 else TOL_FP32
+    assert abs(0.5 * (l0 + l1) - rloss) <= tol_f * abs(rloss)
+    for name, ps in r.named_params():
+        assert relerr(host(ps.g).reshape(rg[name].shape), rg[name]) <= tol_g, name
+    grads = {n: host(ps.g) for n, ps in r.named_params()}
+    r.apply_adamw(hparams(step=1, **hp))
+    for (name, ps), (_, w0) in zip(r.named_params(), O.lm_tensors(lm)):
+        w0 = w0.astype(np.float64)
+        cw, _, _ = O.adamw(w0, 0 * w0, 0 * w0, grads[name].reshape(w0.shape), weight_decay=wd, step=1, **hp)
+        assert relerr(host(ps.w).reshape(w0.shape), cw) <= TOL_ADAMW, name
+    st, detail = fx.fax_check_device_status(sess.ctx)
+    assert st == fx.FAX_OK, detail
