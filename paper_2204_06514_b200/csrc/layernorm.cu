@@ -1,6 +1,9 @@
 // LayerNorm forward / backward (block steps F1, F5, B3, B7 and the LM's final
-// LayerNorm).  HBM-bound: one block per row keeps the whole row in registers,
-// 128-bit loads and stores, warp-shuffle reductions, two-pass mean / variance.
+// LayerNorm).  HBM-bound: rows stay packed in registers between the reductions and the
+// output pass, 128-bit loads and stores, two-pass mean / variance.  Rows of up to 512
+// vectors: groups of warps walk rows with the next row in flight, and the backward pass
+// accumulates dgamma / dbeta in registers on the way; wider rows: one block per row and a
+// separate column reduction.
 #include "common.cuh"
 #include "../../include/fax_ops.h"
 
@@ -70,55 +73,95 @@ template <> __device__ __forceinline__ void unpack<bf16>(const uint4& u, float (
   for (int i = 0; i < 4; ++i) { float2 t = __bfloat1622float2(h[i]); f[2 * i] = t.x; f[2 * i + 1] = t.y; }
 }
 
-// Forward, one warp per row (rows of up to 32*VPT vectors): the row stays packed in
-// registers, reductions are warp shuffles only, no block barrier.
-template <typename T, int VPT>
-__global__ void __launch_bounds__(128)
-layernorm_fwd_warp_kernel(int rows, int d, const T* __restrict__ x, const T* __restrict__ gamma,
-                          const T* __restrict__ beta, float eps, T* __restrict__ out,
-                          float* __restrict__ mu_out, float* __restrict__ rstd_out, T* __restrict__ x_copy) {
+// Forward for rows of up to 512 vectors: a block of 512 threads holds 16 / WG row groups of WG
+// warps; a group walks rows, gamma and beta stay in registers, the next row is requested before
+// the current one is reduced (two-pass mean / variance, each a shuffle reduction plus, for
+// WG > 1, one barrier of the group's own).
+template <typename T, int VPT, int WG>
+__global__ void __launch_bounds__(512, 2)
+layernorm_fwd_group_kernel(int rows, int d, const T* __restrict__ x, const T* __restrict__ gamma,
+                           const T* __restrict__ beta, float eps, T* __restrict__ out,
+                           float* __restrict__ mu_out, float* __restrict__ rstd_out, T* __restrict__ x_copy) {
   constexpr int VN = Vec<T>::N;
-  const int lane = threadIdx.x & 31;
-  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (row >= rows) return;
+  constexpr int NG = 16 / WG, TG = 32 * WG;
+  __shared__ float red[2][16];
+  const int grp = threadIdx.x / TG, t = threadIdx.x % TG;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nvec = d / VN;
-  const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)row * d);
-  uint4 raw[VPT];
-  float s = 0.f;
+  const int stride = NG * gridDim.x;
+  const float inv_d = 1.f / (float)d;
+  uint4 gm[VPT], bt[VPT], nxt[VPT];
 #pragma unroll
   for (int i = 0; i < VPT; ++i) {
-    const int vi = lane + 32 * i;
-    if (vi < nvec) {
-      raw[i] = xr[vi];
-      float f[VN]; unpack<T>(raw[i], f);
-#pragma unroll
-      for (int j = 0; j < VN; ++j) s += f[j];
-    }
+    const int vi = t + TG * i;
+    const bool in = vi < nvec;
+    gm[i] = in ? reinterpret_cast<const uint4*>(gamma)[vi] : make_uint4(0, 0, 0, 0);
+    bt[i] = in ? reinterpret_cast<const uint4*>(beta)[vi] : make_uint4(0, 0, 0, 0);
+    nxt[i] = make_uint4(0, 0, 0, 0);
   }
-  const float mu = warp_sum(s) / (float)d;
-  float q = 0.f;
+  int row = NG * blockIdx.x + grp;
+  if (row < rows) {
+    const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)row * d);
 #pragma unroll
-  for (int i = 0; i < VPT; ++i) {
-    if (lane + 32 * i < nvec) {
-      float f[VN]; unpack<T>(raw[i], f);
-#pragma unroll
-      for (int j = 0; j < VN; ++j) { float t = f[j] - mu; q += t * t; }
-    }
+    for (int i = 0; i < VPT; ++i) if (t + TG * i < nvec) nxt[i] = xr[t + TG * i];
   }
-  const float rstd = rsqrtf(warp_sum(q) / (float)d + eps);
-  if (lane == 0) { mu_out[row] = mu; rstd_out[row] = rstd; }
+  for (; row < rows; row += stride) {
+    uint4 cur[VPT];
 #pragma unroll
-  for (int i = 0; i < VPT; ++i) {
-    const int vi = lane + 32 * i;
-    if (vi < nvec) {
-      float f[VN], g[VN], b[VN], o[VN];
-      unpack<T>(raw[i], f);
-      load_vec<T>(gamma + vi * VN, g);
-      load_vec<T>(beta + vi * VN, b);
+    for (int i = 0; i < VPT; ++i) cur[i] = nxt[i];
+    if (row + stride < rows) {
+      const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)(row + stride) * d);
 #pragma unroll
-      for (int j = 0; j < VN; ++j) o[j] = (f[j] - mu) * rstd * g[j] + b[j];
-      store_vec<T>(out + (size_t)row * d + vi * VN, o);
-      if (x_copy) reinterpret_cast<uint4*>(x_copy + (size_t)row * d)[vi] = raw[i];
+      for (int i = 0; i < VPT; ++i) if (t + TG * i < nvec) nxt[i] = xr[t + TG * i];
+    }
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+      if (t + TG * i < nvec) {
+        float f[VN]; unpack<T>(cur[i], f);
+#pragma unroll
+        for (int j = 0; j < VN; ++j) s += f[j];
+      }
+    }
+    s = warp_sum(s);
+    if (WG > 1) {
+      if (lane == 0) red[0][warp] = s;
+      asm volatile("bar.sync %0, %1;" ::"r"(1 + grp), "r"(TG) : "memory");
+      s = 0.f;
+#pragma unroll
+      for (int k = 0; k < WG; ++k) s += red[0][grp * WG + k];
+    }
+    const float mu = s * inv_d;
+    float q = 0.f;
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+      if (t + TG * i < nvec) {
+        float f[VN]; unpack<T>(cur[i], f);
+#pragma unroll
+        for (int j = 0; j < VN; ++j) { const float c = f[j] - mu; q += c * c; }
+      }
+    }
+    q = warp_sum(q);
+    if (WG > 1) {
+      if (lane == 0) red[1][warp] = q;
+      asm volatile("bar.sync %0, %1;" ::"r"(1 + grp), "r"(TG) : "memory");
+      q = 0.f;
+#pragma unroll
+      for (int k = 0; k < WG; ++k) q += red[1][grp * WG + k];
+    }
+    const float rstd = rsqrtf(q * inv_d + eps);
+    if (t == 0) { mu_out[row] = mu; rstd_out[row] = rstd; }
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+      const int vi = t + TG * i;
+      if (vi < nvec) {
+        float f[VN], g[VN], b[VN], o[VN];
+        unpack<T>(cur[i], f); unpack<T>(gm[i], g); unpack<T>(bt[i], b);
+#pragma unroll
+        for (int j = 0; j < VN; ++j) o[j] = (f[j] - mu) * rstd * g[j] + b[j];
+        store_vec<T>(out + (size_t)row * d + vi * VN, o);
+        if (x_copy) reinterpret_cast<uint4*>(x_copy + (size_t)row * d)[vi] = cur[i];
+      }
     }
   }
 }
@@ -172,127 +215,130 @@ layernorm_fwd_kernel(int rows, int d, const T* __restrict__ x, const T* __restri
   }
 }
 
-// Backward dx, one warp per row: da and x stay packed in registers.
-//   u = da*gamma; dx = rstd*(u - mean(u) - xhat*mean(u*xhat)) (+ add)
-template <typename T, int VPT>
-__global__ void __launch_bounds__(128)
-layernorm_bwd_dx_warp_kernel(int rows, int d, const T* __restrict__ da, const T* __restrict__ x,
-                             const float* __restrict__ mu_in, const float* __restrict__ rstd_in,
-                             const T* __restrict__ gamma, const T* __restrict__ add, T* __restrict__ dx) {
+// Backward, fused: dx and the per-block column sums for dgamma / dbeta in one pass over da and x.
+// A block of 512 threads holds 16 / WG row groups of WG warps; a group walks rows
+// (group index + k * groups in the grid), every thread owning the same VPT vector columns in all
+// of them, so the column sums accumulate in registers.  The next row's vectors are requested
+// before the current row is reduced.  At the end the groups of a block add their sums in shared
+// memory and the block writes one slab: partial[block][0][c] = sum da*xhat, partial[block][1][c] = sum da.
+template <typename T, int VPT, int WG>
+__global__ void __launch_bounds__(512, 1)
+layernorm_bwd_fused_kernel(int rows, int d, const T* __restrict__ da, const T* __restrict__ x,
+                           const float* __restrict__ mu_in, const float* __restrict__ rstd_in,
+                           const T* __restrict__ gamma, const T* __restrict__ add, T* __restrict__ dx,
+                           float* __restrict__ partial) {
   constexpr int VN = Vec<T>::N;
-  const int lane = threadIdx.x & 31;
-  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (row >= rows) return;
-  const int nvec = d / VN;
-  const float mu = mu_in[row], rstd = rstd_in[row];
-  const uint4* dar = reinterpret_cast<const uint4*>(da + (size_t)row * d);
-  const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)row * d);
-  uint4 rda[VPT], rx[VPT];
-  float s1 = 0.f, s2 = 0.f;
-#pragma unroll
-  for (int i = 0; i < VPT; ++i) {
-    const int vi = lane + 32 * i;
-    if (vi < nvec) { rda[i] = dar[vi]; rx[i] = xr[vi]; }
-  }
-#pragma unroll
-  for (int i = 0; i < VPT; ++i) {
-    const int vi = lane + 32 * i;
-    if (vi < nvec) {
-      float fd[VN], fx[VN], g[VN];
-      unpack<T>(rda[i], fd); unpack<T>(rx[i], fx);
-      load_vec<T>(gamma + vi * VN, g);
-#pragma unroll
-      for (int j = 0; j < VN; ++j) { float u = fd[j] * g[j]; s1 += u; s2 += u * (fx[j] - mu) * rstd; }
-    }
-  }
-  const float c1 = warp_sum(s1) / (float)d, c2 = warp_sum(s2) / (float)d;
-#pragma unroll
-  for (int i = 0; i < VPT; ++i) {
-    const int vi = lane + 32 * i;
-    if (vi < nvec) {
-      float fd[VN], fx[VN], g[VN], o[VN];
-      unpack<T>(rda[i], fd); unpack<T>(rx[i], fx);
-      load_vec<T>(gamma + vi * VN, g);
-#pragma unroll
-      for (int j = 0; j < VN; ++j) o[j] = rstd * (fd[j] * g[j] - c1 - (fx[j] - mu) * rstd * c2);
-      if (add) {
-        float av[VN];
-        load_vec<T>(add + (size_t)row * d + vi * VN, av);
-#pragma unroll
-        for (int j = 0; j < VN; ++j) o[j] += av[j];
-      }
-      store_vec<T>(dx + (size_t)row * d + vi * VN, o);
-    }
-  }
-}
-
-// Backward dx with G warps per row (rows of more than 256 vectors): a lane holds at most 8
-// vectors of da and of x, which keeps the kernel at 3 to 4 blocks per SM; the G partial sums of
-// a row meet in shared memory behind a barrier of just those warps.
-template <typename T, int VPT, int G>
-__global__ void __launch_bounds__(256)
-layernorm_bwd_dx_group_kernel(int rows, int d, const T* __restrict__ da, const T* __restrict__ x,
-                              const float* __restrict__ mu_in, const float* __restrict__ rstd_in,
-                              const T* __restrict__ gamma, const T* __restrict__ add, T* __restrict__ dx) {
-  constexpr int VN = Vec<T>::N;
-  constexpr int RG = 8 / G;
-  __shared__ float2 red[8];
+  constexpr int NG = 16 / WG, TG = 32 * WG;
+  extern __shared__ float fuse_sm[];                 // 2 * d floats
+  __shared__ float2 red[2][16];
+  const int grp = threadIdx.x / TG, t = threadIdx.x % TG;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int rg = warp / G, gw = warp % G;
   const int nvec = d / VN;
-  const int row = blockIdx.x * RG + rg;
-  const bool live = row < rows;
-  uint4 rda[VPT], rx[VPT];
-  float mu = 0.f, rstd = 0.f, s1 = 0.f, s2 = 0.f;
-  if (live) {
-    const uint4* dar = reinterpret_cast<const uint4*>(da + (size_t)row * d);
-    const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)row * d);
+  const int stride = NG * gridDim.x;
+  const float inv_d = 1.f / (float)d;
+  float ag[VPT][VN], ab[VPT][VN];
+  uint4 gm[VPT], nda[VPT], nx[VPT], nad[VPT];
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) {
+#pragma unroll
+    for (int j = 0; j < VN; ++j) { ag[i][j] = 0.f; ab[i][j] = 0.f; }
+    const int vi = t + TG * i;
+    gm[i] = (vi < nvec) ? reinterpret_cast<const uint4*>(gamma)[vi] : make_uint4(0, 0, 0, 0);
+    nda[i] = nx[i] = nad[i] = make_uint4(0, 0, 0, 0);
+  }
+  int row = NG * blockIdx.x + grp;
+  float nmu = 0.f, nrs = 0.f;
+#define LN_FETCH(r)                                                                      \
+  {                                                                                      \
+    const uint4* dar = reinterpret_cast<const uint4*>(da + (size_t)(r) * d);             \
+    const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)(r) * d);               \
+    const uint4* adr = reinterpret_cast<const uint4*>(add + (size_t)(r) * d);            \
+    _Pragma("unroll") for (int i = 0; i < VPT; ++i) {                                    \
+      const int vi = t + TG * i;                                                         \
+      if (vi < nvec) { nda[i] = dar[vi]; nx[i] = xr[vi]; if (add) nad[i] = adr[vi]; }    \
+    }                                                                                    \
+    nmu = mu_in[r]; nrs = rstd_in[r];                                                    \
+  }
+  if (row < rows) LN_FETCH(row)
+  for (int it = 0; row < rows; row += stride, ++it) {
+    uint4 cda[VPT], cx[VPT], cad[VPT];
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) { cda[i] = nda[i]; cx[i] = nx[i]; cad[i] = nad[i]; }
+    const float mu = nmu, rstd = nrs;
+    const int nr = row + stride;
+    if (nr < rows) LN_FETCH(nr)
+    float s1 = 0.f, s2 = 0.f;
 #pragma unroll
     for (int i = 0; i < VPT; ++i) {
-      const int vi = lane + 32 * (i + VPT * gw);
-      if (vi < nvec) { rda[i] = dar[vi]; rx[i] = xr[vi]; }
-    }
-    mu = mu_in[row]; rstd = rstd_in[row];
-#pragma unroll
-    for (int i = 0; i < VPT; ++i) {
-      const int vi = lane + 32 * (i + VPT * gw);
-      if (vi < nvec) {
+      if (t + TG * i < nvec) {
         float fd[VN], fx[VN], g[VN];
-        unpack<T>(rda[i], fd); unpack<T>(rx[i], fx);
-        load_vec<T>(gamma + vi * VN, g);
+        unpack<T>(cda[i], fd); unpack<T>(cx[i], fx); unpack<T>(gm[i], g);
 #pragma unroll
         for (int j = 0; j < VN; ++j) { const float u = fd[j] * g[j]; s1 += u; s2 += u * (fx[j] - mu) * rstd; }
       }
     }
     s1 = warp_sum(s1); s2 = warp_sum(s2);
-  }
-  if (G > 1) {
-    if (lane == 0) red[warp] = make_float2(s1, s2);
-    __syncthreads();
-    s1 = 0.f; s2 = 0.f;
+    if (WG > 1) {
+      // the WG warps of this row meet at a barrier of their own; red is double-buffered by
+      // iteration parity, so one barrier per row is enough
+      if (lane == 0) red[it & 1][warp] = make_float2(s1, s2);
+      asm volatile("bar.sync %0, %1;" ::"r"(1 + grp), "r"(TG) : "memory");
+      s1 = 0.f; s2 = 0.f;
 #pragma unroll
-    for (int k = 0; k < G; ++k) { s1 += red[rg * G + k].x; s2 += red[rg * G + k].y; }
-  }
-  if (!live) return;
-  const float c1 = s1 / (float)d, c2 = s2 / (float)d;
+      for (int k = 0; k < WG; ++k) { const float2 v = red[it & 1][grp * WG + k]; s1 += v.x; s2 += v.y; }
+    }
+    const float c1 = s1 * inv_d, c2 = s2 * inv_d;
 #pragma unroll
-  for (int i = 0; i < VPT; ++i) {
-    const int vi = lane + 32 * (i + VPT * gw);
-    if (vi < nvec) {
-      float fd[VN], fx[VN], g[VN], o[VN];
-      unpack<T>(rda[i], fd); unpack<T>(rx[i], fx);
-      load_vec<T>(gamma + vi * VN, g);
+    for (int i = 0; i < VPT; ++i) {
+      const int vi = t + TG * i;
+      if (vi < nvec) {
+        float fd[VN], fx[VN], g[VN], o[VN];
+        unpack<T>(cda[i], fd); unpack<T>(cx[i], fx); unpack<T>(gm[i], g);
 #pragma unroll
-      for (int j = 0; j < VN; ++j) o[j] = rstd * (fd[j] * g[j] - c1 - (fx[j] - mu) * rstd * c2);
-      if (add) {
-        float av[VN];
-        load_vec<T>(add + (size_t)row * d + vi * VN, av);
+        for (int j = 0; j < VN; ++j) {
+          const float xh = (fx[j] - mu) * rstd;
+          o[j] = rstd * (fd[j] * g[j] - c1 - xh * c2);
+          ag[i][j] += fd[j] * xh;
+          ab[i][j] += fd[j];
+        }
+        if (add) {
+          float av[VN];
+          unpack<T>(cad[i], av);
 #pragma unroll
-        for (int j = 0; j < VN; ++j) o[j] += av[j];
+          for (int j = 0; j < VN; ++j) o[j] += av[j];
+        }
+        store_vec<T>(dx + (size_t)row * d + vi * VN, o);
       }
-      store_vec<T>(dx + (size_t)row * d + vi * VN, o);
     }
   }
+#undef LN_FETCH
+  // the groups add their column sums one after the other (fixed order: deterministic)
+  for (int g = 0; g < NG; ++g) {
+    if (grp == g) {
+#pragma unroll
+      for (int i = 0; i < VPT; ++i) {
+        const int vi = t + TG * i;
+        if (vi < nvec) {
+#pragma unroll
+          for (int j = 0; j < VN; j += 4) {
+            float4* pg = reinterpret_cast<float4*>(fuse_sm + vi * VN + j);
+            float4* pb = reinterpret_cast<float4*>(fuse_sm + d + vi * VN + j);
+            float4 vg = make_float4(ag[i][j], ag[i][j + 1], ag[i][j + 2], ag[i][j + 3]);
+            float4 vb = make_float4(ab[i][j], ab[i][j + 1], ab[i][j + 2], ab[i][j + 3]);
+            if (g > 0) {
+              const float4 og = *pg, ob = *pb;
+              vg.x += og.x; vg.y += og.y; vg.z += og.z; vg.w += og.w;
+              vb.x += ob.x; vb.y += ob.y; vb.z += ob.z; vb.w += ob.w;
+            }
+            *pg = vg; *pb = vb;
+          }
+        }
+      }
+    }
+    __syncthreads();
+  }
+  float4* dst = reinterpret_cast<float4*>(partial + (size_t)blockIdx.x * 2 * d);
+  for (int c = threadIdx.x; c < 2 * d / 4; c += blockDim.x) dst[c] = reinterpret_cast<const float4*>(fuse_sm)[c];
 }
 
 // Backward dx, one block per row (wide rows).
@@ -401,15 +447,28 @@ colreduce_kernel(int rows, int cols, const T* __restrict__ in, int64_t ld, const
   }
 }
 
-// out[c] (+)= sum_s partial[s][c] for c < width (width = cols, or 2*cols with out split in two)
-__global__ void colreduce_fold_kernel(int slabs, int width, int cols, const float* __restrict__ partial,
-                                      float* __restrict__ out0, float* __restrict__ out1, int accumulate) {
-  int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= width) return;
+// out[c] (+)= sum_s partial[s][c] for c < width (width = cols, or 2*cols with out split in two).
+// Block = 32 columns x 8 slab phases, summed in a fixed order.
+__global__ void __launch_bounds__(256)
+colreduce_fold_kernel(int slabs, int width, int cols, const float* __restrict__ partial,
+                      float* __restrict__ out0, float* __restrict__ out1, int accumulate) {
+  __shared__ float sm[8][33];
+  const int lane = threadIdx.x & 31, ph = threadIdx.x >> 5;
+  const int c = blockIdx.x * 32 + lane;
   float s = 0.f;
-  for (int i = 0; i < slabs; ++i) s += partial[(size_t)i * width + c];
-  float* dst = (c < cols) ? (out0 + c) : (out1 + (c - cols));
-  *dst = accumulate ? (*dst + s) : s;
+  if (c < width) {
+#pragma unroll 4
+    for (int i = ph; i < slabs; i += 8) s += partial[(size_t)i * width + c];
+  }
+  sm[ph][lane] = s;
+  __syncthreads();
+  if (ph == 0 && c < width) {
+    s = 0.f;
+#pragma unroll
+    for (int k = 0; k < 8; ++k) s += sm[k][lane];
+    float* dst = (c < cols) ? (out0 + c) : (out1 + (c - cols));
+    *dst = accumulate ? (*dst + s) : s;
+  }
 }
 
 int pick_vpt(int nvec, int max_threads, int* threads) {
@@ -422,18 +481,33 @@ int pick_vpt(int nvec, int max_threads, int* threads) {
   return 0;
 }
 
-// Row slabs of the column reductions: enough blocks to fill the machine, at most 256 slabs.
-int colreduce_slabs(fax_ctx* ctx, int rows, int nvec) {
+// Row slabs of the column reductions: as many blocks as are resident at once (a grid a little
+// larger than that would leave a second, nearly empty wave), at most 256 slabs.
+int colreduce_slabs(fax_ctx* ctx, int rows, int nvec, int blocks_per_sm) {
   const int gx = (nvec + 31) / 32;
-  int slabs = (8 * ctx->sm_count + gx - 1) / gx;
+  int slabs = blocks_per_sm * ctx->sm_count / gx;
   const int max_by_rows = (rows + 31) / 32;
   if (slabs > max_by_rows) slabs = max_by_rows;
   if (slabs > 256) slabs = 256;
   if (slabs < 1) slabs = 1;
   return slabs;
 }
+// Resident 256-thread blocks per SM: 8 for the plain column sum (32 registers), 5 for the
+// LayerNorm variant (48 registers).
+constexpr int kColsumBlocksPerSm = 8, kLnColBlocksPerSm = 5;
+// The fused backward covers rows of up to 512 vectors; one slab per block, one block per SM.
+bool ln_bwd_is_fused(int nvec) { return nvec <= 512; }
+int ln_row_groups(int nvec) { return nvec <= 64 ? 16 : nvec <= 128 ? 8 : nvec <= 256 ? 4 : 2; }
+int ln_bwd_fused_grid(fax_ctx* ctx, int rows, int nvec) {
+  const int ng = ln_row_groups(nvec);
+  int grid = (rows + ng - 1) / ng;
+  if (grid > ctx->sm_count) grid = ctx->sm_count;
+  if (grid > 256) grid = 256;
+  return grid < 1 ? 1 : grid;
+}
 int ln_bwd_slabs(fax_ctx* ctx, int rows, int d, int prec) {
-  return colreduce_slabs(ctx, rows, d / (prec == FAX_PREC_BF16 ? 8 : 4));
+  const int nvec = d / (prec == FAX_PREC_BF16 ? 8 : 4);
+  return ln_bwd_is_fused(nvec) ? ln_bwd_fused_grid(ctx, rows, nvec) : colreduce_slabs(ctx, rows, nvec, kLnColBlocksPerSm);
 }
 
 template <typename T>
@@ -441,15 +515,19 @@ fax_status ln_fwd_t(fax_ctx* ctx, int rows, int d, const void* x, const void* ga
                     float eps, void* out, float* mu, float* rstd, void* x_copy) {
   const int nvec = d / Vec<T>::N;
   if (nvec <= 512) {
-    const int need = (nvec + 31) / 32;
-#define LN_FWDW(V)                                                                                      \
-    if (need <= V) {                                                                                    \
-      layernorm_fwd_warp_kernel<T, V><<<(rows + 3) / 4, 128, 0, ctx->stream>>>(                         \
-          rows, d, (const T*)x, (const T*)gamma, (const T*)beta, eps, (T*)out, mu, rstd, (T*)x_copy);   \
-      return fax_after_launch(ctx);                                                                     \
-    }
-    LN_FWDW(1) LN_FWDW(2) LN_FWDW(3) LN_FWDW(4) LN_FWDW(6) LN_FWDW(8) LN_FWDW(12) LN_FWDW(16)
-#undef LN_FWDW
+    const int ng = ln_row_groups(nvec);
+    int grid = (rows + ng - 1) / ng;
+    if (grid > 2 * ctx->sm_count) grid = 2 * ctx->sm_count;
+#define LN_FWDG(V, W)                                                                                   \
+    layernorm_fwd_group_kernel<T, V, W><<<grid, 512, 0, ctx->stream>>>(                                 \
+        rows, d, (const T*)x, (const T*)gamma, (const T*)beta, eps, (T*)out, mu, rstd, (T*)x_copy)
+    if (nvec <= 32) LN_FWDG(1, 1);
+    else if (nvec <= 64) LN_FWDG(2, 1);
+    else if (nvec <= 128) LN_FWDG(2, 2);
+    else if (nvec <= 256) LN_FWDG(2, 4);
+    else LN_FWDG(2, 8);
+#undef LN_FWDG
+    return fax_after_launch(ctx);
   }
   int threads = 0;
   int vpt = pick_vpt(nvec, 512, &threads);
@@ -468,23 +546,6 @@ template <typename T>
 fax_status ln_bwd_dx_t(fax_ctx* ctx, int rows, int d, const void* da, const void* x, const float* mu,
                        const float* rstd, const void* gamma, const void* add, void* dx) {
   const int nvec = d / Vec<T>::N;
-  if (nvec > 256 && nvec <= 512) {
-    // two warps per row, 8 vectors per lane
-    layernorm_bwd_dx_group_kernel<T, 8, 2><<<(rows + 3) / 4, 256, 0, ctx->stream>>>(
-        rows, d, (const T*)da, (const T*)x, mu, rstd, (const T*)gamma, (const T*)add, (T*)dx);
-    return fax_after_launch(ctx);
-  }
-  if (nvec <= 512) {
-    const int need = (nvec + 31) / 32;
-#define LN_BWDW(V)                                                                                      \
-    if (need <= V) {                                                                                    \
-      layernorm_bwd_dx_warp_kernel<T, V><<<(rows + 3) / 4, 128, 0, ctx->stream>>>(                      \
-          rows, d, (const T*)da, (const T*)x, mu, rstd, (const T*)gamma, (const T*)add, (T*)dx);        \
-      return fax_after_launch(ctx);                                                                     \
-    }
-    LN_BWDW(1) LN_BWDW(2) LN_BWDW(3) LN_BWDW(4) LN_BWDW(6) LN_BWDW(8) LN_BWDW(12) LN_BWDW(16)
-#undef LN_BWDW
-  }
   int threads = 0;
   int vpt = pick_vpt(nvec, 512, &threads);
   if (!vpt || vpt > 8) return FAX_ERR_UNSUPPORTED_SHAPE;
@@ -498,18 +559,40 @@ fax_status ln_bwd_dx_t(fax_ctx* ctx, int rows, int d, const void* da, const void
   return fax_after_launch(ctx);
 }
 
+template <typename T>
+fax_status ln_bwd_fused_t(fax_ctx* ctx, int rows, int d, const void* da, const void* x, const float* mu,
+                          const float* rstd, const void* gamma, const void* add, void* dx, float* dgamma,
+                          float* dbeta, bool accumulate, float* partial) {
+  const int nvec = d / Vec<T>::N;
+  const int grid = ln_bwd_fused_grid(ctx, rows, nvec);
+  const size_t smem = (size_t)2 * d * sizeof(float);
+#define LN_FUSED(V, W)                                                                                 \
+  layernorm_bwd_fused_kernel<T, V, W><<<grid, 512, smem, ctx->stream>>>(                               \
+      rows, d, (const T*)da, (const T*)x, mu, rstd, (const T*)gamma, (const T*)add, (T*)dx, partial)
+  if (nvec <= 32) LN_FUSED(1, 1);
+  else if (nvec <= 64) LN_FUSED(2, 1);
+  else if (nvec <= 128) LN_FUSED(2, 2);
+  else if (nvec <= 256) LN_FUSED(2, 4);
+  else LN_FUSED(2, 8);
+#undef LN_FUSED
+  FAX_TRY(fax_after_launch(ctx));
+  colreduce_fold_kernel<<<(2 * d + 31) / 32, 256, 0, ctx->stream>>>(grid, 2 * d, d, partial, dgamma, dbeta,
+                                                                   accumulate ? 1 : 0);
+  return fax_after_launch(ctx);
+}
+
 template <typename T, bool LN>
 fax_status colreduce_t(fax_ctx* ctx, int rows, int cols, const void* in, int64_t ld, const void* x,
                        const float* mu, const float* rstd, float* out0, float* out1, bool accumulate,
                        float* partial) {
   const int nvec = cols / Vec<T>::N;
-  const int slabs = colreduce_slabs(ctx, rows, nvec);
+  const int slabs = colreduce_slabs(ctx, rows, nvec, LN ? kLnColBlocksPerSm : kColsumBlocksPerSm);
   dim3 grid((nvec + 31) / 32, slabs);
   colreduce_kernel<T, LN><<<grid, 256, 0, ctx->stream>>>(rows, cols, (const T*)in, ld, (const T*)x, mu, rstd, partial);
   FAX_TRY(fax_after_launch(ctx));
   const int width = LN ? 2 * cols : cols;
-  colreduce_fold_kernel<<<(width + 255) / 256, 256, 0, ctx->stream>>>(slabs, width, cols, partial, out0, out1,
-                                                                      accumulate ? 1 : 0);
+  colreduce_fold_kernel<<<(width + 31) / 32, 256, 0, ctx->stream>>>(slabs, width, cols, partial, out0, out1,
+                                                                    accumulate ? 1 : 0);
   return fax_after_launch(ctx);
 }
 
@@ -540,6 +623,11 @@ fax_status fax_layernorm_bwd(fax_ctx* ctx, int prec, int rows, int d, const void
   if (partial_floats < (size_t)2 * ln_bwd_slabs(ctx, rows, d, prec) * d) return FAX_ERR_WORKSPACE_TOO_SMALL;
   // dx pass reads da, x (and add) and writes dx; the dgamma/dbeta pass reads da and x again
   FaxProfScope prof(ctx, KC_LN_BWD, 0.0, (double)rows * d * fax_elem_size(prec) * (add ? 4 : 3));
+  if (ln_bwd_is_fused(d / (prec == FAX_PREC_BF16 ? 8 : 4))) {
+    if (prec == FAX_PREC_BF16)
+      return ln_bwd_fused_t<bf16>(ctx, rows, d, da, x, mu, rstd, gamma, add, dx, dgamma, dbeta, accumulate, partial);
+    return ln_bwd_fused_t<float>(ctx, rows, d, da, x, mu, rstd, gamma, add, dx, dgamma, dbeta, accumulate, partial);
+  }
   if (prec == FAX_PREC_BF16) {
     FAX_TRY(ln_bwd_dx_t<bf16>(ctx, rows, d, da, x, mu, rstd, gamma, add, dx));
     return colreduce_t<bf16, true>(ctx, rows, d, da, d, x, mu, rstd, dgamma, dbeta, accumulate, partial);
@@ -557,7 +645,7 @@ fax_status fax_colsum(fax_ctx* ctx, int prec, int rows, int cols, const void* in
                       bool accumulate, float* partial, size_t partial_floats) {
   const int vn = prec == FAX_PREC_BF16 ? 8 : 4;
   if (cols % vn || ld % vn) return FAX_ERR_UNSUPPORTED_SHAPE;
-  if (partial_floats < (size_t)colreduce_slabs(ctx, rows, cols / vn) * cols) return FAX_ERR_WORKSPACE_TOO_SMALL;
+  if (partial_floats < (size_t)colreduce_slabs(ctx, rows, cols / vn, kColsumBlocksPerSm) * cols) return FAX_ERR_WORKSPACE_TOO_SMALL;
   FaxProfScope prof(ctx, KC_COLSUM, 0.0, (double)rows * cols * fax_elem_size(prec));
   if (prec == FAX_PREC_BF16)
     return colreduce_t<bf16, false>(ctx, rows, cols, in, ld, nullptr, nullptr, nullptr, out, out, accumulate, partial);
