@@ -290,13 +290,16 @@ fax_status launch_fwd(fax_ctx* ctx, int B, int T, int H, const void* qkv, void* 
 // bf16 operand tiles; the elected thread then issues dV_j += P^T dO_i and
 // dK_j += dS^T Q_i (accumulating in tensor memory over the whole walk) and
 // dQ_i = dS K_j, which the row threads stage in shared memory and one thread adds
-// into a float32 dQ buffer with a bulk tensor reduction.  The P / dS / Q / dO / K tiles are each used both as a K-major and as
+// into a float32 dQ buffer with a bulk tensor reduction (per-thread vector reductions
+// from registers into global memory were measured a third slower).  Eight row warps:
+// nothing in the backward pass reduces along a row, so two warps share each quarter
+// of the tensor-memory lanes and take one half of the columns each.  The P / dS / Q / dO / K tiles are each used both as a K-major and as
 // an MN-major operand: the bytes are the same, only the descriptor differs.
 // Tensor memory: [0,128) S, [128,256) dP then dQ, [256,256+HD) dV, [384,384+HD) dK.  P is signalled
 // before dS so that dV runs while the row threads still work on dS; dK is issued before dQ so the Q
 // tile can be reloaded while dQ is computed and read out.
 // ---------------------------------------------------------------------------
-constexpr int BWD_THREADS = 192;   // 4 row warps + MMA warp + TMA warp
+constexpr int BWD_THREADS = 320;   // 8 row warps (4 lane quarters x 2 column halves) + MMA warp + TMA warp
 
 struct AttnBwdParams {
   int B, T, H;
@@ -330,7 +333,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_co
   uint8_t* gbase = smem_raw + (base - raw);
   const uint32_t bars = base + C_::BAR_OFF;
   // barriers: 0 K/V full | 1,2 Q full | 3,4 dO full | 5,6 Q free | 7,8 dO free | 9 S full | 10 dP full |
-  //           11 P ready (4) | 12 dS ready (4) | 13 dQ full | 14 dQ read out (4)
+  //           11 P ready (8) | 12 dS ready (8) | 13 dQ full | 14 dQ read out (8)
   auto bar = [&](int i) { return bars + 8u * i; };
   volatile uint32_t* tmem_slot = (volatile uint32_t*)(gbase + C_::BAR_OFF + 128);
   volatile int* abort_flag = (volatile int*)(gbase + C_::BAR_OFF + 132);
@@ -347,13 +350,13 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_co
   const int nsteps = nq - kj;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < 15; ++i) mbar_init(bar(i), (i == 11 || i == 12 || i == 14) ? 4u : 1u);
+    for (int i = 0; i < 15; ++i) mbar_init(bar(i), (i == 11 || i == 12 || i == 14) ? 8u : 1u);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_qkv) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_do) : "memory");
   }
-  if (warp == 4) tmem_alloc(smem_u32((const void*)tmem_slot), C_::TMEM_COLS);
+  if (warp == 8) tmem_alloc(smem_u32((const void*)tmem_slot), C_::TMEM_COLS);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -364,7 +367,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_co
   auto q_s = [&](int i) { return base + C_::Q_OFF + i * C_::TILE_BYTES; };
   auto do_s = [&](int i) { return base + C_::DO_OFF + i * C_::TILE_BYTES; };
 
-  if (warp == 5) {
+  if (warp == 9) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
       mbar_expect_tx(bar(0), 2 * C_::TILE_BYTES);
@@ -389,7 +392,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_co
       }
       if (!ok) { const long long t0 = clock64(); while (clock64() - t0 < 2000000LL) { } }
     }
-  } else if (warp == 4) {
+  } else if (warp == 8) {
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
       const uint32_t idesc_s = idesc_bf16(128, false, false);
@@ -439,8 +442,12 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_co
       }
     }
   } else {
-    const int r = 32 * warp + lane;
-    const uint32_t lane_base = (uint32_t)(32 * warp) << 16;
+    // Row threads: warp w serves query rows 32*(w&3).. (its quarter of the tensor-memory lanes) and
+    // the column half w>>2 of every tile: nothing here reduces along a row, so the halves are
+    // independent and each scheduler has two warps to interleave.
+    const int hc = warp >> 2;
+    const int r = 32 * (warp & 3) + lane;
+    const uint32_t lane_base = (uint32_t)(32 * (warp & 3)) << 16;
     uint8_t* p_row = gbase + C_::P_OFF + r * 128;
     uint8_t* ds_row = gbase + C_::DS_OFF + r * 128;
     bool ok = true;
@@ -451,22 +458,22 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_co
       const float lse2 = p.lse[stat] * 1.4426950408889634f;
       const float Dr = p.Dv[stat];
       const bool diag = (it == 0);
-      uint32_t pp[64];
+      uint32_t pp[32];
       // P = exp(S / sqrt(hd) - LSE): the P tile is also needed (as bf16) by dS below
       if (!mbar_wait_warp(bar(9), ph, abort_flag, p.status, 309)) { ok = false; break; }
       tc_fence_after();
       {
-        uint32_t sv[4][32];
+        uint32_t sv[2][32];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) tc_ld32(tm_s + lane_base + 32 * c, sv[c]);
+        for (int c = 0; c < 2; ++c) tc_ld32(tm_s + lane_base + 64 * hc + 32 * c, sv[c]);
         tc_wait_ld();
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
+        for (int c = 0; c < 2; ++c)
 #pragma unroll
           for (int e = 0; e < 32; e += 2) {
             float p0 = ex2_approx(__uint_as_float(sv[c][e]) * p.scale_log2 - lse2);
             float p1 = ex2_approx(__uint_as_float(sv[c][e + 1]) * p.scale_log2 - lse2);
-            if (diag) { if (32 * c + e > r) p0 = 0.f; if (32 * c + e + 1 > r) p1 = 0.f; }
+            if (diag) { if (64 * hc + 32 * c + e > r) p0 = 0.f; if (64 * hc + 32 * c + e + 1 > r) p1 = 0.f; }
             __nv_bfloat162 hp = __floats2bfloat162_rn(p0, p1);
             pp[16 * c + (e >> 1)] = *reinterpret_cast<uint32_t*>(&hp);
           }
@@ -474,13 +481,13 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_co
       if (it > 0) {
         // the P / dS buffers staged the previous dQ tile: its bulk reduction must have read them
         if (threadIdx.x == 0) bulk_wait_read_all();
-        named_barrier_sync(1, 128);
+        named_barrier_sync(1, 256);
       }
 #pragma unroll
-      for (int c = 0; c < 4; ++c)
+      for (int c = 0; c < 2; ++c)
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-          const int off = (c >> 1) * 16384 + (((((c & 1) << 2) + k) ^ (r & 7)) << 4);
+          const int off = hc * 16384 + ((((c << 2) + k) ^ (r & 7)) << 4);
           *reinterpret_cast<uint4*>(p_row + off) =
               make_uint4(pp[16 * c + 4 * k], pp[16 * c + 4 * k + 1], pp[16 * c + 4 * k + 2], pp[16 * c + 4 * k + 3]);
         }
@@ -491,15 +498,14 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_co
       // dS = P * (dP - D), from the bf16 P that the products use
       if (!mbar_wait_warp(bar(10), ph, abort_flag, p.status, 310)) { ok = false; break; }
       tc_fence_after();
-#pragma unroll
-      for (int half = 0; half < 2; ++half) {
+      {
         uint32_t dv[2][32];
-        tc_ld32(tm_dp + lane_base + 64 * half, dv[0]);
-        tc_ld32(tm_dp + lane_base + 64 * half + 32, dv[1]);
+        tc_ld32(tm_dp + lane_base + 64 * hc, dv[0]);
+        tc_ld32(tm_dp + lane_base + 64 * hc + 32, dv[1]);
         tc_wait_ld();
 #pragma unroll
         for (int cc = 0; cc < 2; ++cc) {
-          const int c = 2 * half + cc;
+          const int c = cc;
           uint32_t dd[16];
 #pragma unroll
           for (int e = 0; e < 32; e += 2) {
@@ -510,7 +516,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_co
           }
 #pragma unroll
           for (int k = 0; k < 4; ++k) {
-            const int off = (c >> 1) * 16384 + (((((c & 1) << 2) + k) ^ (r & 7)) << 4);
+            const int off = hc * 16384 + ((((c << 2) + k) ^ (r & 7)) << 4);
             *reinterpret_cast<uint4*>(ds_row + off) = make_uint4(dd[4 * k], dd[4 * k + 1], dd[4 * k + 2], dd[4 * k + 3]);
           }
         }
@@ -524,14 +530,16 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_co
       // float32 dQ accumulator in global memory
       if (!mbar_wait_warp(bar(13), ph, abort_flag, p.status, 311)) { ok = false; break; }
       tc_fence_after();
+      {
+        // this warp's half of the head's columns: HD/2 = 64 (two boxes) or 32 (one box)
+        constexpr int NB = HD / 64;
+        const int c0 = hc * (HD / 2);
+        uint32_t v[NB][32];
 #pragma unroll
-      for (int c0 = 0; c0 < HD; c0 += 64) {
-        uint32_t v[2][32];
-        tc_ld32(tm_dp + lane_base + c0, v[0]);
-        tc_ld32(tm_dp + lane_base + c0 + 32, v[1]);
+        for (int cc = 0; cc < NB; ++cc) tc_ld32(tm_dp + lane_base + c0 + 32 * cc, v[cc]);
         tc_wait_ld();
 #pragma unroll
-        for (int cc = 0; cc < 2; ++cc) {
+        for (int cc = 0; cc < NB; ++cc) {
           uint8_t* box = gbase + C_::P_OFF + ((c0 >> 5) + cc) * 16384 + r * 128;
 #pragma unroll
           for (int k = 0; k < 8; ++k)
@@ -543,7 +551,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_co
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(14));
       fence_proxy_async();
-      named_barrier_sync(1, 128);
+      named_barrier_sync(1, 256);
       if (threadIdx.x == 0) {
 #pragma unroll
         for (int i = 0; i < HD / 32; ++i)
@@ -558,7 +566,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_co
       bf16* dk_row = p.dqkv + tok * 3 * d + d + h * HD;
       bf16* dv_row = p.dqkv + tok * 3 * d + 2 * d + h * HD;
 #pragma unroll 1
-      for (int c0 = 0; c0 < HD; c0 += 32) {
+      for (int c0 = hc * (HD / 2); c0 < (hc + 1) * (HD / 2); c0 += 32) {
         uint32_t kv[32], vv[32];
         tc_ld32(tm_dk + lane_base + c0, kv);
         tc_ld32(tm_dv + lane_base + c0, vv);
@@ -581,7 +589,7 @@ attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_co
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 4) { tc_fence_after(); tmem_dealloc(tmem, C_::TMEM_COLS); }
+  if (warp == 8) { tc_fence_after(); tmem_dealloc(tmem, C_::TMEM_COLS); }
 }
 
 // D[b,h,t] = sum_c dO[t,c] * O[t,c] over the head's columns; one warp per (token, head)
