@@ -671,6 +671,8 @@ bool fax_attention_tc_supported(int B, int T, int H, int hd) {
 fax_status fax_attention_fwd_tc(fax_ctx* ctx, int B, int T, int H, int hd, const void* qkv, void* o, float* lse) {
   if (!fax_attention_tc_supported(B, T, H, hd) || !fax_aligned(qkv, 16) || !fax_aligned(o, 16))
     return FAX_ERR_UNSUPPORTED_SHAPE;
+  // sequences of a whole number of query-tile pairs take the two-tile persistent kernel
+  if (fax_attention_fwd2_supported(B, T, H, hd)) return fax_attention_fwd2_tc(ctx, B, T, H, hd, qkv, o, lse);
   return hd == 64 ? launch_fwd<64>(ctx, B, T, H, qkv, o, lse) : launch_fwd<128>(ctx, B, T, H, qkv, o, lse);
 }
 

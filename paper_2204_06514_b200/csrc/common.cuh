@@ -241,6 +241,8 @@ fax_status fax_loss_mean(fax_ctx* ctx, int n, const float* row_loss, float* loss
 
 bool fax_attention_tc_supported(int B, int T, int H, int hd);
 fax_status fax_attention_fwd_tc(fax_ctx* ctx, int B, int T, int H, int hd, const void* qkv, void* o, float* lse);
+bool fax_attention_fwd2_supported(int B, int T, int H, int hd);
+fax_status fax_attention_fwd2_tc(fax_ctx* ctx, int B, int T, int H, int hd, const void* qkv, void* o, float* lse);
 size_t fax_attention_bwd_tc_scratch_bytes(int B, int T, int H, int hd);
 fax_status fax_attention_bwd_tc(fax_ctx* ctx, int B, int T, int H, int hd, const void* qkv, const void* o,
                                 const float* lse, const void* d_o, void* dqkv, void* scratch, size_t scratch_bytes);
