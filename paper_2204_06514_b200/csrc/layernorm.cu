@@ -78,7 +78,7 @@ template <> __device__ __forceinline__ void unpack<bf16>(const uint4& u, float (
 // the current one is reduced (two-pass mean / variance, each a shuffle reduction plus, for
 // WG > 1, one barrier of the group's own).
 template <typename T, int VPT, int WG>
-__global__ void __launch_bounds__(512, 2)
+__global__ void __launch_bounds__(512, (VPT <= 2) ? 2 : 1)
 layernorm_fwd_group_kernel(int rows, int d, const T* __restrict__ x, const T* __restrict__ gamma,
                            const T* __restrict__ beta, float eps, T* __restrict__ out,
                            float* __restrict__ mu_out, float* __restrict__ rstd_out, T* __restrict__ x_copy) {
@@ -515,15 +515,19 @@ fax_status ln_fwd_t(fax_ctx* ctx, int rows, int d, const void* x, const void* ga
                     float eps, void* out, float* mu, float* rstd, void* x_copy) {
   const int nvec = d / Vec<T>::N;
   if (nvec <= 512) {
-    const int ng = ln_row_groups(nvec);
+    // narrow rows: one warp per row with 3 or 4 vectors per lane (more bytes in flight per thread)
+    const bool wide_lane = nvec > 64 && nvec <= 128;
+    const int ng = wide_lane ? 16 : ln_row_groups(nvec);
     int grid = (rows + ng - 1) / ng;
-    if (grid > 2 * ctx->sm_count) grid = 2 * ctx->sm_count;
+    const int cap = (wide_lane ? 1 : 2) * ctx->sm_count;
+    if (grid > cap) grid = cap;
 #define LN_FWDG(V, W)                                                                                   \
     layernorm_fwd_group_kernel<T, V, W><<<grid, 512, 0, ctx->stream>>>(                                 \
         rows, d, (const T*)x, (const T*)gamma, (const T*)beta, eps, (T*)out, mu, rstd, (T*)x_copy)
     if (nvec <= 32) LN_FWDG(1, 1);
     else if (nvec <= 64) LN_FWDG(2, 1);
-    else if (nvec <= 128) LN_FWDG(2, 2);
+    else if (nvec <= 96) LN_FWDG(3, 1);
+    else if (nvec <= 128) LN_FWDG(4, 1);
     else if (nvec <= 256) LN_FWDG(2, 4);
     else LN_FWDG(2, 8);
 #undef LN_FWDG
