@@ -1,6 +1,7 @@
 // Causal multi-head attention on the tcgen05 tensor cores (steps F3 / B5).
 //
-// Forward: one CTA per (batch, head, 128-query tile).  Q stays in shared memory;
+// Forward (sequence lengths that are not a multiple of 256; the others take the two-tile kernel
+// of attention_fwd2_tc.cu): one CTA per (batch, head, 128-query tile).  Q stays in shared memory;
 // K and V tiles of 128 keys stream through a double-buffered TMA ring.  One
 // elected thread issues S = Q K^T into tensor memory; four warps (one query row
 // per thread) run the online softmax on S read from tensor memory, write
@@ -282,23 +283,6 @@ fax_status launch_fwd(fax_ctx* ctx, int B, int T, int H, const void* qkv, void* 
 }
 
 
-// ---------------------------------------------------------------------------
-// Backward.  One CTA per (batch, head, 128-key tile j); it keeps K_j and V_j in
-// shared memory and walks the query tiles i >= j.  Per step the elected thread
-// issues S = Q_i K_j^T and dP = dO_i V_j^T; the row threads (one query row
-// each) form P = exp(S/sqrt(hd) - LSE) and dS = P * (dP - D) and write both as
-// bf16 operand tiles; the elected thread then issues dV_j += P^T dO_i and
-// dK_j += dS^T Q_i (accumulating in tensor memory over the whole walk) and
-// dQ_i = dS K_j, which the row threads stage in shared memory and one thread adds
-// into a float32 dQ buffer with a bulk tensor reduction (per-thread vector reductions
-// from registers into global memory were measured a third slower).  Eight row warps:
-// nothing in the backward pass reduces along a row, so two warps share each quarter
-// of the tensor-memory lanes and take one half of the columns each.  The P / dS / Q / dO / K tiles are each used both as a K-major and as
-// an MN-major operand: the bytes are the same, only the descriptor differs.
-// Tensor memory: [0,128) S, [128,256) dP then dQ, [256,256+HD) dV, [384,384+HD) dK.  P is signalled
-// before dS so that dV runs while the row threads still work on dS; dK is issued before dQ so the Q
-// tile can be reloaded while dQ is computed and read out.
-// ---------------------------------------------------------------------------
 constexpr int BWD_THREADS = 320;   // 8 row warps (4 lane quarters x 2 column halves) + MMA warp + TMA warp
 
 struct AttnBwdParams {
@@ -309,283 +293,375 @@ struct AttnBwdParams {
   int32_t* status;
 };
 
-template <int HD> struct BwdCfg {
-  static constexpr int NQ = (HD == 64) ? 2 : 1;          // Q / dO stages (shared memory allows 2 only at hd 64)
+// ---------------------------------------------------------------------------
+// Backward (step B5), persistent.  A CTA owns a 128-key tile j (K_j, V_j resident in shared memory) and
+// walks the query tiles i >= j; the score tiles are formed transposed (keys in the tensor-memory lanes):
+//   S^T = K_j Q_i^T, dP^T = V_j dO_i^T, so P^T and dS^T (bf16, written back over their own
+// accumulators by the row threads) are the A operands of dV_j += P^T dO_i and dK_j += dS^T Q_i
+// straight from tensor memory; only dS also goes to shared memory, as the MN-major A operand of
+// dQ_i = dS K_j.  After dS the MMA thread issues dQ first, then dK and (Q is double-buffered) S^T of
+// the next step, so these run while the row threads read dQ out.  A row thread owns one key row and
+// one half of the tile's 128 queries; the per-query statistics (LSE, D) of the tile sit in shared
+// memory.  A CTA loops over its share of the (batch, head, key tile) list, longest walks first;
+// the next tile's K, V, Q, dO loads overlap the read-out of dK and dV.
+// Tensor memory: [0,128) S^T, then P^T at +64h+[0,32) and dS^T at +64h+[32,64) | [128,256) dP^T, then dQ |
+// [256,256+HD) dV | [384,384+HD) dK.
+// ---------------------------------------------------------------------------
+template <int HD> struct Bwd2Cfg {
+  static constexpr int NQ = 2;                             // Q stages
+  static constexpr int NDO = (HD == 64) ? 2 : 1;           // dO stages
   static constexpr int TILE_BYTES = 128 * HD * 2;
-  static constexpr int PS_BYTES = 128 * 128 * 2;
   static constexpr int K_OFF = 0, V_OFF = TILE_BYTES;
   static constexpr int Q_OFF = 2 * TILE_BYTES, DO_OFF = Q_OFF + NQ * TILE_BYTES;
-  static constexpr int P_OFF = DO_OFF + NQ * TILE_BYTES, DS_OFF = P_OFF + PS_BYTES;
-  static constexpr int BAR_OFF = DS_OFF + PS_BYTES;
-  static constexpr int SMEM_BYTES = BAR_OFF + 256 + 1024;
-  static constexpr int TMEM_COLS = 512;                  // S [0,128) | dP then dQ [128,256) | dV [256,..) | dK [384,..)
+  static constexpr int DS_OFF = DO_OFF + NDO * TILE_BYTES;  // dS tile (32 KB); the dQ staging boxes start here too
+  static constexpr int STG_BYTES = 128 * HD * 4;            // dQ tile in float32
+  static constexpr int DS_BYTES = (STG_BYTES > 32768) ? STG_BYTES : 32768;
+  static constexpr int STAT_OFF = DS_OFF + DS_BYTES;        // [2][2][128] floats: log2e*LSE and D of the query tile
+  static constexpr int BAR_OFF = STAT_OFF + 2048;
+  static constexpr int LAYOUT_BYTES = BAR_OFF + 256;
+  // 768 bytes of slack for aligning the tiles to 1024 bytes (at hd 128 this is exactly the 227 KB a CTA
+  // may have); the kernel checks that the aligned layout fits before it touches anything
+  static constexpr int SMEM_BYTES = LAYOUT_BYTES + 768;
+  static constexpr int TMEM_COLS = 512;
+  // barriers
+  static constexpr int KVFULL = 0, KVFREE = 1, QFULL = 2, QFREE = 4, DOFULL = 6, DOFREE = 8, SFULL = 10, DPFULL = 11,
+                       PREADY = 12, DSREADY = 13, DQFULL = 14, DQREAD = 15, DKVREAD = 16, STGFREE = 17, STGFULL = 18,
+                       STATFULL = 19, ALLDONE = 20, STGFREE2 = 21, NBARS = 22;
 };
 
 template <int HD>
 __global__ void __launch_bounds__(BWD_THREADS, 1)
-attn_bwd_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_constant__ CUtensorMap tmap_do,
-                   const __grid_constant__ CUtensorMap tmap_dq, const AttnBwdParams p) {
-  using C_ = BwdCfg<HD>;
-  constexpr int NQ = C_::NQ;
+attn_bwd2_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_constant__ CUtensorMap tmap_do,
+                    const __grid_constant__ CUtensorMap tmap_dq, const AttnBwdParams p) {
+  using C_ = Bwd2Cfg<HD>;
+  constexpr int NQ = C_::NQ, NDO = C_::NDO;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* gbase = smem_raw + (base - raw);
   const uint32_t bars = base + C_::BAR_OFF;
-  // barriers: 0 K/V full | 1,2 Q full | 3,4 dO full | 5,6 Q free | 7,8 dO free | 9 S full | 10 dP full |
-  //           11 P ready (8) | 12 dS ready (8) | 13 dQ full | 14 dQ read out (8)
   auto bar = [&](int i) { return bars + 8u * i; };
-  volatile uint32_t* tmem_slot = (volatile uint32_t*)(gbase + C_::BAR_OFF + 128);
-  volatile int* abort_flag = (volatile int*)(gbase + C_::BAR_OFF + 132);
+  volatile uint32_t* tmem_slot = (volatile uint32_t*)(gbase + C_::BAR_OFF + 192);
+  volatile int* abort_flag = (volatile int*)(gbase + C_::BAR_OFF + 196);
+  if ((base - raw) + (uint32_t)C_::LAYOUT_BYTES > (uint32_t)C_::SMEM_BYTES) {
+    // the dynamic shared memory window starts less aligned than assumed: report, touch nothing
+    if (threadIdx.x == 0 && atomicCAS(p.status, 0, 1) == 0) p.status[1] = 320;
+    return;
+  }
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nq = p.T / 128;
   const int bh_count = p.B * p.H;
-  const int kj = (int)(blockIdx.x / bh_count);             // heaviest key tiles (small j) first
-  const int bh = blockIdx.x % bh_count;
-  const int b = bh / p.H, h = bh % p.H;
+  const int n_items = nq * bh_count;
   const int d = p.H * HD;
-  const int row0 = b * p.T;
-  const int qcol = h * HD, kcol = d + h * HD, vcol = 2 * d + h * HD;
-  const int nsteps = nq - kj;
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < 15; ++i) mbar_init(bar(i), (i == 11 || i == 12 || i == 14) ? 8u : 1u);
+    for (int i = 0; i < C_::NBARS; ++i) {
+      const bool eight = (i == C_::PREADY || i == C_::DSREADY || i == C_::DQREAD || i == C_::DKVREAD ||
+                          i == C_::STGFULL || i == C_::STATFULL);
+      mbar_init(bar(i), eight ? 8u : 1u);
+    }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_qkv) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_do) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_dq) : "memory");
   }
   if (warp == 8) tmem_alloc(smem_u32((const void*)tmem_slot), C_::TMEM_COLS);
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t tm_s = tmem, tm_dp = tmem + 128, tm_dv = tmem + 256, tm_dk = tmem + 384;
-  const uint32_t k_s = base + C_::K_OFF, v_s = base + C_::V_OFF;
-  const uint32_t p_s = base + C_::P_OFF, ds_s = base + C_::DS_OFF;
+  const uint32_t tm_st = tmem, tm_dp = tmem + 128, tm_dv = tmem + 256, tm_dk = tmem + 384;
+  const uint32_t k_s = base + C_::K_OFF, v_s = base + C_::V_OFF, ds_s = base + C_::DS_OFF;
   auto q_s = [&](int i) { return base + C_::Q_OFF + i * C_::TILE_BYTES; };
   auto do_s = [&](int i) { return base + C_::DO_OFF + i * C_::TILE_BYTES; };
 
   if (warp == 9) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
-      mbar_expect_tx(bar(0), 2 * C_::TILE_BYTES);
-#pragma unroll
-      for (int i = 0; i < HD / 64; ++i) {
-        tma_load_2d(k_s + i * 16384, &tmap_qkv, bar(0), kcol + 64 * i, row0 + kj * 128);
-        tma_load_2d(v_s + i * 16384, &tmap_qkv, bar(0), vcol + 64 * i, row0 + kj * 128);
-      }
+      uint32_t gs = 0;              // steps requested so far (all items)
       bool ok = true;
-      for (int it = 0; it < nsteps && ok; ++it) {
-        const int st = it % NQ;
-        const uint32_t ph = (uint32_t)((it / NQ) & 1);
-        const int qrow = row0 + (kj + it) * 128;
-        if (!mbar_wait(bar(5 + st), ph ^ 1u, abort_flag, p.status, 301)) { ok = false; break; }
-        mbar_expect_tx(bar(1 + st), C_::TILE_BYTES);
+      int it_n = 0;
+      for (int t = blockIdx.x; t < n_items && ok; t += gridDim.x, ++it_n) {
+        const int kj = t / bh_count, bh = t % bh_count;
+        const int b = bh / p.H, h = bh % p.H;
+        const int row0 = b * p.T;
+        const int qcol = h * HD, kcol = d + h * HD, vcol = 2 * d + h * HD;
+        if (!mbar_wait(bar(C_::KVFREE), (uint32_t)(it_n & 1) ^ 1u, abort_flag, p.status, 321)) { ok = false; break; }
+        mbar_expect_tx(bar(C_::KVFULL), 2 * C_::TILE_BYTES);
 #pragma unroll
-        for (int i = 0; i < HD / 64; ++i) tma_load_2d(q_s(st) + i * 16384, &tmap_qkv, bar(1 + st), qcol + 64 * i, qrow);
-        if (!mbar_wait(bar(7 + st), ph ^ 1u, abort_flag, p.status, 302)) { ok = false; break; }
-        mbar_expect_tx(bar(3 + st), C_::TILE_BYTES);
+        for (int i = 0; i < HD / 64; ++i) {
+          tma_load_2d(k_s + i * 16384, &tmap_qkv, bar(C_::KVFULL), kcol + 64 * i, row0 + kj * 128);
+          tma_load_2d(v_s + i * 16384, &tmap_qkv, bar(C_::KVFULL), vcol + 64 * i, row0 + kj * 128);
+        }
+        const int nsteps = nq - kj;
+        for (int it = 0; it < nsteps && ok; ++it, ++gs) {
+          const int qrow = row0 + (kj + it) * 128;
+          const int sq = (int)(gs % NQ), sd = (int)(gs % NDO);
+          if (!mbar_wait(bar(C_::QFREE + sq), ((gs / NQ) & 1u) ^ 1u, abort_flag, p.status, 322)) { ok = false; break; }
+          mbar_expect_tx(bar(C_::QFULL + sq), C_::TILE_BYTES);
 #pragma unroll
-        for (int i = 0; i < HD / 64; ++i) tma_load_2d(do_s(st) + i * 16384, &tmap_do, bar(3 + st), qcol + 64 * i, qrow);
+          for (int i = 0; i < HD / 64; ++i) tma_load_2d(q_s(sq) + i * 16384, &tmap_qkv, bar(C_::QFULL + sq), qcol + 64 * i, qrow);
+          if (!mbar_wait(bar(C_::DOFREE + sd), ((gs / NDO) & 1u) ^ 1u, abort_flag, p.status, 323)) { ok = false; break; }
+          mbar_expect_tx(bar(C_::DOFULL + sd), C_::TILE_BYTES);
+#pragma unroll
+          for (int i = 0; i < HD / 64; ++i) tma_load_2d(do_s(sd) + i * 16384, &tmap_do, bar(C_::DOFULL + sd), qcol + 64 * i, qrow);
+        }
       }
       if (!ok) { const long long t0 = clock64(); while (clock64() - t0 < 2000000LL) { } }
     }
   } else if (warp == 8) {
     // ---------------- MMA issuer ----------------
     if (lane == 0) {
-      const uint32_t idesc_s = idesc_bf16(128, false, false);
-      const uint32_t idesc_kv = idesc_bf16(HD, true, true);
-      const uint32_t idesc_q = idesc_bf16(HD, false, true);
+      const uint32_t idesc_s = idesc_bf16(128, false, false);     // S^T, dP^T: both operands K-major
+      const uint32_t idesc_acc = idesc_bf16(HD, false, true);      // dV, dK: A in tensor memory, B MN-major
+      const uint32_t idesc_dq = idesc_bf16(HD, true, true);        // dQ: dS and K both MN-major
       auto koff = [](int s) { return (uint32_t)((s / 4) * 16384 + (s % 4) * 32); };   // K-major k-step
-      bool ok = mbar_wait(bar(0), 0, abort_flag, p.status, 303);
-      for (int it = 0; it < nsteps && ok; ++it) {
-        const int st = it % NQ;
-        const uint32_t sph = (uint32_t)((it / NQ) & 1), ph = (uint32_t)(it & 1);
-        // S = Q K^T  (the S columns were read out before P of the previous step was signalled)
-        if (!mbar_wait(bar(1 + st), sph, abort_flag, p.status, 304)) { ok = false; break; }
+      auto acol = [](int k) { return (uint32_t)(64 * (k / 4) + 8 * (k % 4)); };       // A k-step in tensor memory
+      uint32_t gs = 0;
+      bool ok = true;
+      int it_n = 0;
+      auto issue_s = [&](uint32_t g) -> bool {
+        const int sq = (int)(g % NQ);
+        if (!mbar_wait(bar(C_::QFULL + sq), (g / NQ) & 1u, abort_flag, p.status, 324)) return false;
         tc_fence_after();
 #pragma unroll
         for (int s = 0; s < HD / 16; ++s)
-          tc_mma_bf16(tm_s, smem_desc(q_s(st) + koff(s), 16, 1024), smem_desc(k_s + koff(s), 16, 1024), idesc_s, s ? 1u : 0u);
-        tc_commit(bar(9));
-        // dP = dO V^T  (its columns double as dQ: wait until the previous dQ has been read out)
-        if (!mbar_wait(bar(3 + st), sph, abort_flag, p.status, 305)) { ok = false; break; }
-        if (it > 0 && !mbar_wait(bar(14), ph ^ 1u, abort_flag, p.status, 306)) { ok = false; break; }
-        tc_fence_after();
+          tc_mma_bf16(tm_st, smem_desc(k_s + koff(s), 16, 1024), smem_desc(q_s(sq) + koff(s), 16, 1024), idesc_s, s ? 1u : 0u);
+        tc_commit(bar(C_::SFULL));
+        return true;
+      };
+      for (int t = blockIdx.x; t < n_items && ok; t += gridDim.x, ++it_n) {
+        const int kj = t / bh_count;
+        const int nsteps = nq - kj;
+        if (!mbar_wait(bar(C_::KVFULL), (uint32_t)(it_n & 1), abort_flag, p.status, 325)) { ok = false; break; }
+        if (!issue_s(gs)) { ok = false; break; }
+        for (int it = 0; it < nsteps && ok; ++it, ++gs) {
+          const int sq = (int)(gs % NQ), sd = (int)(gs % NDO);
+          // dP^T = V dO^T (its columns held the previous step's dQ: wait until that was read out)
+          if (!mbar_wait(bar(C_::DOFULL + sd), (gs / NDO) & 1u, abort_flag, p.status, 326)) { ok = false; break; }
+          if (gs > 0 && !mbar_wait(bar(C_::DQREAD), (gs - 1) & 1u, abort_flag, p.status, 327)) { ok = false; break; }
+          tc_fence_after();
 #pragma unroll
-        for (int s = 0; s < HD / 16; ++s)
-          tc_mma_bf16(tm_dp, smem_desc(do_s(st) + koff(s), 16, 1024), smem_desc(v_s + koff(s), 16, 1024), idesc_s, s ? 1u : 0u);
-        tc_commit(bar(10));
-        // dV += P^T dO
-        if (!mbar_wait(bar(11), ph, abort_flag, p.status, 307)) { ok = false; break; }
-        tc_fence_after();
+          for (int s = 0; s < HD / 16; ++s)
+            tc_mma_bf16(tm_dp, smem_desc(v_s + koff(s), 16, 1024), smem_desc(do_s(sd) + koff(s), 16, 1024), idesc_s, s ? 1u : 0u);
+          tc_commit(bar(C_::DPFULL));
+          // dV += P^T dO (the first one of a key tile overwrites: dV and dK of the tile before must have been read out)
+          if (!mbar_wait(bar(C_::PREADY), gs & 1u, abort_flag, p.status, 328)) { ok = false; break; }
+          if (it == 0 && !mbar_wait(bar(C_::DKVREAD), (uint32_t)(it_n & 1) ^ 1u, abort_flag, p.status, 329)) { ok = false; break; }
+          tc_fence_after();
 #pragma unroll
-        for (int s = 0; s < 8; ++s)
-          tc_mma_bf16(tm_dv, smem_desc(p_s + s * 2048, 16384, 1024), smem_desc(do_s(st) + s * 2048, 16384, 1024),
-                      idesc_kv, (it | s) ? 1u : 0u);
-        tc_commit(bar(7 + st));          // dO stage free
-        // dK += dS^T Q, then dQ = dS K
-        if (!mbar_wait(bar(12), ph, abort_flag, p.status, 308)) { ok = false; break; }
-        tc_fence_after();
+          for (int k = 0; k < 8; ++k)
+            tc_mma_bf16_ts(tm_dv, tm_st + acol(k), smem_desc(do_s(sd) + k * 2048, 16384, 1024), idesc_acc, (it | k) ? 1u : 0u);
+          tc_commit(bar(C_::DOFREE + sd));
+          // dQ = dS K over the dP^T columns (all read by now), then dK += dS^T Q with dS^T from the spare
+          // columns of the S^T accumulator, then S^T of the next step over that accumulator
+          if (!mbar_wait(bar(C_::DSREADY), gs & 1u, abort_flag, p.status, 330)) { ok = false; break; }
+          tc_fence_after();
 #pragma unroll
-        for (int s = 0; s < 8; ++s)
-          tc_mma_bf16(tm_dk, smem_desc(ds_s + s * 2048, 16384, 1024), smem_desc(q_s(st) + s * 2048, 16384, 1024),
-                      idesc_kv, (it | s) ? 1u : 0u);
-        tc_commit(bar(5 + st));          // Q stage free
+          for (int k = 0; k < 8; ++k)
+            tc_mma_bf16(tm_dp, smem_desc(ds_s + k * 2048, 16384, 1024), smem_desc(k_s + k * 2048, 16384, 1024), idesc_dq,
+                        k ? 1u : 0u);
+          tc_commit(bar(C_::DQFULL));
 #pragma unroll
-        for (int s = 0; s < 8; ++s)
-          tc_mma_bf16(tm_dp, smem_desc(ds_s + koff(s), 16, 1024), smem_desc(k_s + s * 2048, 16384, 1024),
-                      idesc_q, s ? 1u : 0u);
-        tc_commit(bar(13));              // dQ ready; also: every MMA issued so far is complete
+          for (int k = 0; k < 8; ++k)
+            tc_mma_bf16_ts(tm_dk, tm_st + 32u + acol(k), smem_desc(q_s(sq) + k * 2048, 16384, 1024), idesc_acc, (it | k) ? 1u : 0u);
+          tc_commit(bar(C_::QFREE + sq));
+          if (it + 1 == nsteps) {
+            tc_commit(bar(C_::KVFREE));
+            tc_commit(bar(C_::ALLDONE));         // every MMA of this key tile is complete: dV and dK are final
+          } else if (!issue_s(gs + 1)) { ok = false; break; }
+        }
       }
     }
   } else {
-    // Row threads: warp w serves query rows 32*(w&3).. (its quarter of the tensor-memory lanes) and
-    // the column half w>>2 of every tile: nothing here reduces along a row, so the halves are
-    // independent and each scheduler has two warps to interleave.
+    // ---- row threads: key row kr (dQ read-out: query row kr), query / column half hc ----
     const int hc = warp >> 2;
-    const int r = 32 * (warp & 3) + lane;
+    const int kr = 32 * (warp & 3) + lane;
     const uint32_t lane_base = (uint32_t)(32 * (warp & 3)) << 16;
-    uint8_t* p_row = gbase + C_::P_OFF + r * 128;
-    uint8_t* ds_row = gbase + C_::DS_OFF + r * 128;
+    uint8_t* ds_row = gbase + C_::DS_OFF + hc * 16384 + kr * 128;
+    float* stat = reinterpret_cast<float*>(gbase + C_::STAT_OFF);      // [buf][0: lse2, 1: D][128]
+    const int tid = threadIdx.x;                                       // 0..255
+    uint32_t gs = 0;
     bool ok = true;
-    for (int it = 0; it < nsteps; ++it) {
-      const uint32_t ph = (uint32_t)(it & 1);
-      const int qi = kj + it;
-      const long long stat = ((long long)b * p.H + h) * p.T + qi * 128 + r;
-      const float lse2 = p.lse[stat] * 1.4426950408889634f;
-      const float Dr = p.Dv[stat];
-      const bool diag = (it == 0);
-      uint32_t pp[32];
-      // P = exp(S / sqrt(hd) - LSE): the P tile is also needed (as bf16) by dS below
-      if (!mbar_wait_warp(bar(9), ph, abort_flag, p.status, 309)) { ok = false; break; }
+    int it_n = 0;
+    for (int t = blockIdx.x; t < n_items && ok; t += gridDim.x, ++it_n) {
+      const int kj = t / bh_count, bh = t % bh_count;
+      const int b = bh / p.H, h = bh % p.H;
+      const int row0 = b * p.T;
+      const int nsteps = nq - kj;
+      const long long stat0 = ((long long)b * p.H + h) * p.T;
+      auto load_stats = [&](int qi, uint32_t buf) {
+        const long long idx = stat0 + qi * 128 + (tid & 127);
+        stat[buf * 256 + tid] = (tid < 128) ? p.lse[idx] * 1.4426950408889634f : p.Dv[idx];
+      };
+      // statistics of a step are published through a barrier of eight warp arrivals: one phase per step
+      load_stats(kj, gs & 1u);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar(C_::STATFULL));
+      for (int it = 0; it < nsteps; ++it, ++gs) {
+        const uint32_t ph = gs & 1u;
+        const int qi = kj + it;
+        const float* st_l = stat + ph * 256 + 64 * hc;
+        const float* st_d = st_l + 128;
+        if (!mbar_wait_warp(bar(C_::STATFULL), ph, abort_flag, p.status, 335)) { ok = false; break; }
+        if (it + 1 < nsteps) {
+          // the other buffer was last read in the step before this one, which every warp has left
+          // (this step's S^T needed the previous dS of all of them)
+          load_stats(qi + 1, ph ^ 1u);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar(C_::STATFULL));
+        }
+        uint32_t pp[32];
+        // P^T = exp(S^T / sqrt(hd) - LSE[q])
+        if (!mbar_wait_warp(bar(C_::SFULL), ph, abort_flag, p.status, 331)) { ok = false; break; }
+        tc_fence_after();
+        {
+          uint32_t sv[2][32];
+          tc_ld32(tm_st + lane_base + 64 * hc, sv[0]);
+          tc_ld32(tm_st + lane_base + 64 * hc + 32, sv[1]);
+          tc_wait_ld();
+#pragma unroll
+          for (int c = 0; c < 2; ++c)
+#pragma unroll
+            for (int e = 0; e < 32; e += 4) {
+              const float4 l4 = *reinterpret_cast<const float4*>(st_l + 32 * c + e);
+              float p0 = ex2_approx(__uint_as_float(sv[c][e]) * p.scale_log2 - l4.x);
+              float p1 = ex2_approx(__uint_as_float(sv[c][e + 1]) * p.scale_log2 - l4.y);
+              float p2 = ex2_approx(__uint_as_float(sv[c][e + 2]) * p.scale_log2 - l4.z);
+              float p3 = ex2_approx(__uint_as_float(sv[c][e + 3]) * p.scale_log2 - l4.w);
+              if (it == 0) {        // diagonal tile: query index below key index is masked
+                const int q0 = 64 * hc + 32 * c + e;
+                if (q0 < kr) p0 = 0.f;
+                if (q0 + 1 < kr) p1 = 0.f;
+                if (q0 + 2 < kr) p2 = 0.f;
+                if (q0 + 3 < kr) p3 = 0.f;
+              }
+              __nv_bfloat162 h0 = __floats2bfloat162_rn(p0, p1), h1 = __floats2bfloat162_rn(p2, p3);
+              pp[16 * c + (e >> 1)] = *reinterpret_cast<uint32_t*>(&h0);
+              pp[16 * c + (e >> 1) + 1] = *reinterpret_cast<uint32_t*>(&h1);
+            }
+        }
+        tc_st32(tm_st + lane_base + 64 * hc, pp);
+        tc_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(C_::PREADY));
+        // dS^T = P^T * (dP^T - D[q]), from the bf16 P that the products use
+        if (!mbar_wait_warp(bar(C_::DPFULL), ph, abort_flag, p.status, 332)) { ok = false; break; }
+        tc_fence_after();
+        uint32_t dd[32];
+        {
+          uint32_t dv[2][32];
+          tc_ld32(tm_dp + lane_base + 64 * hc, dv[0]);
+          tc_ld32(tm_dp + lane_base + 64 * hc + 32, dv[1]);
+          tc_wait_ld();
+#pragma unroll
+          for (int c = 0; c < 2; ++c)
+#pragma unroll
+            for (int e = 0; e < 32; e += 4) {
+              const float4 d4 = *reinterpret_cast<const float4*>(st_d + 32 * c + e);
+              const float2 pa = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pp[16 * c + (e >> 1)]));
+              const float2 pb = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pp[16 * c + (e >> 1) + 1]));
+              __nv_bfloat162 h0 = __floats2bfloat162_rn(pa.x * (__uint_as_float(dv[c][e]) - d4.x),
+                                                        pa.y * (__uint_as_float(dv[c][e + 1]) - d4.y));
+              __nv_bfloat162 h1 = __floats2bfloat162_rn(pb.x * (__uint_as_float(dv[c][e + 2]) - d4.z),
+                                                        pb.y * (__uint_as_float(dv[c][e + 3]) - d4.w));
+              dd[16 * c + (e >> 1)] = *reinterpret_cast<uint32_t*>(&h0);
+              dd[16 * c + (e >> 1) + 1] = *reinterpret_cast<uint32_t*>(&h1);
+            }
+        }
+        tc_st32(tm_st + lane_base + 64 * hc + 32, dd);
+        if (gs > 0) {
+          // the dS buffer staged the first 32 KB of the previous dQ tile: the bulk reductions of those
+          // boxes (the older of the two groups at hd 128, the only group at hd 64) must have read it
+          if (tid == 0) {
+            if (HD == 128) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+            else bulk_wait_read_all();
+            mbar_arrive(bar(C_::STGFREE));
+          }
+          if (!mbar_wait_warp(bar(C_::STGFREE), (gs - 1) & 1u, abort_flag, p.status, 333)) { ok = false; break; }
+        }
+#pragma unroll
+        for (int k = 0; k < 8; ++k)
+          *reinterpret_cast<uint4*>(ds_row + ((k ^ (kr & 7)) << 4)) = make_uint4(dd[4 * k], dd[4 * k + 1], dd[4 * k + 2], dd[4 * k + 3]);
+        fence_proxy_async();
+        tc_wait_st();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(C_::DSREADY));
+        // dQ tile: tensor memory -> shared memory (32-column float boxes, 128-byte swizzled) -> one bulk
+        // add-reduction per box into the float32 dQ accumulator
+        if (!mbar_wait_warp(bar(C_::DQFULL), ph, abort_flag, p.status, 334)) { ok = false; break; }
+        tc_fence_after();
+        if (HD == 128 && gs > 0) {
+          // boxes 2 and 3 (the column half of warps 4..7) lie behind the dS tile: their reductions of the step before
+          if (tid == 0) { bulk_wait_read_all(); mbar_arrive(bar(C_::STGFREE2)); }
+          if (hc == 1 && !mbar_wait_warp(bar(C_::STGFREE2), (gs - 1) & 1u, abort_flag, p.status, 337)) { ok = false; break; }
+        }
+        {
+          constexpr int NB = HD / 64;          // this warp's half of the head's columns: two boxes or one
+          const int c0 = hc * (HD / 2);
+          uint32_t v[NB][32];
+#pragma unroll
+          for (int cc = 0; cc < NB; ++cc) tc_ld32(tm_dp + lane_base + c0 + 32 * cc, v[cc]);
+          tc_wait_ld();
+#pragma unroll
+          for (int cc = 0; cc < NB; ++cc) {
+            uint8_t* box = gbase + C_::DS_OFF + ((c0 >> 5) + cc) * 16384 + kr * 128;
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+              *reinterpret_cast<uint4*>(box + ((k ^ (kr & 7)) << 4)) =
+                  make_uint4(v[cc][4 * k], v[cc][4 * k + 1], v[cc][4 * k + 2], v[cc][4 * k + 3]);
+          }
+        }
+        tc_fence_before();
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) { mbar_arrive(bar(C_::DQREAD)); mbar_arrive(bar(C_::STGFULL)); }
+        if (tid == 0 && mbar_wait(bar(C_::STGFULL), ph, abort_flag, p.status, 336)) {
+#pragma unroll
+          for (int i = 0; i < HD / 32; ++i) {
+            tma_reduce_add_2d(&tmap_dq, base + C_::DS_OFF + i * 16384, h * HD + 32 * i, (int)(row0 + qi * 128));
+            if (HD == 128 && i == 1) bulk_commit_group();     // boxes 0, 1 (the dS tile's bytes) as a group of their own
+          }
+          bulk_commit_group();
+        }
+      }
+      if (!ok) break;
+      if (!mbar_wait_warp(bar(C_::ALLDONE), (uint32_t)(it_n & 1), abort_flag, p.status, 338)) { ok = false; break; }
       tc_fence_after();
       {
-        uint32_t sv[2][32];
-#pragma unroll
-        for (int c = 0; c < 2; ++c) tc_ld32(tm_s + lane_base + 64 * hc + 32 * c, sv[c]);
-        tc_wait_ld();
-#pragma unroll
-        for (int c = 0; c < 2; ++c)
-#pragma unroll
-          for (int e = 0; e < 32; e += 2) {
-            float p0 = ex2_approx(__uint_as_float(sv[c][e]) * p.scale_log2 - lse2);
-            float p1 = ex2_approx(__uint_as_float(sv[c][e + 1]) * p.scale_log2 - lse2);
-            if (diag) { if (64 * hc + 32 * c + e > r) p0 = 0.f; if (64 * hc + 32 * c + e + 1 > r) p1 = 0.f; }
-            __nv_bfloat162 hp = __floats2bfloat162_rn(p0, p1);
-            pp[16 * c + (e >> 1)] = *reinterpret_cast<uint32_t*>(&hp);
-          }
-      }
-      if (it > 0) {
-        // the P / dS buffers staged the previous dQ tile: its bulk reduction must have read them
-        if (threadIdx.x == 0) bulk_wait_read_all();
-        named_barrier_sync(1, 256);
-      }
-#pragma unroll
-      for (int c = 0; c < 2; ++c)
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const int off = hc * 16384 + ((((c << 2) + k) ^ (r & 7)) << 4);
-          *reinterpret_cast<uint4*>(p_row + off) =
-              make_uint4(pp[16 * c + 4 * k], pp[16 * c + 4 * k + 1], pp[16 * c + 4 * k + 2], pp[16 * c + 4 * k + 3]);
-        }
-      fence_proxy_async();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(11));
-      // dS = P * (dP - D), from the bf16 P that the products use
-      if (!mbar_wait_warp(bar(10), ph, abort_flag, p.status, 310)) { ok = false; break; }
-      tc_fence_after();
-      {
-        uint32_t dv[2][32];
-        tc_ld32(tm_dp + lane_base + 64 * hc, dv[0]);
-        tc_ld32(tm_dp + lane_base + 64 * hc + 32, dv[1]);
-        tc_wait_ld();
-#pragma unroll
-        for (int cc = 0; cc < 2; ++cc) {
-          const int c = cc;
-          uint32_t dd[16];
-#pragma unroll
-          for (int e = 0; e < 32; e += 2) {
-            const float2 pf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&pp[16 * c + (e >> 1)]));
-            __nv_bfloat162 hd2 = __floats2bfloat162_rn(pf.x * (__uint_as_float(dv[cc][e]) - Dr),
-                                                       pf.y * (__uint_as_float(dv[cc][e + 1]) - Dr));
-            dd[e >> 1] = *reinterpret_cast<uint32_t*>(&hd2);
-          }
-#pragma unroll
-          for (int k = 0; k < 4; ++k) {
-            const int off = hc * 16384 + ((((c << 2) + k) ^ (r & 7)) << 4);
-            *reinterpret_cast<uint4*>(ds_row + off) = make_uint4(dd[4 * k], dd[4 * k + 1], dd[4 * k + 2], dd[4 * k + 3]);
-          }
-        }
-      }
-      fence_proxy_async();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(12));
-      // dQ tile of this step: tensor memory -> shared memory (the P / dS buffers, free by now, as
-      // 32-column boxes in the 128-byte-swizzled layout) -> one bulk add-reduction into the
-      // float32 dQ accumulator in global memory
-      if (!mbar_wait_warp(bar(13), ph, abort_flag, p.status, 311)) { ok = false; break; }
-      tc_fence_after();
-      {
-        // this warp's half of the head's columns: HD/2 = 64 (two boxes) or 32 (one box)
-        constexpr int NB = HD / 64;
-        const int c0 = hc * (HD / 2);
-        uint32_t v[NB][32];
-#pragma unroll
-        for (int cc = 0; cc < NB; ++cc) tc_ld32(tm_dp + lane_base + c0 + 32 * cc, v[cc]);
-        tc_wait_ld();
-#pragma unroll
-        for (int cc = 0; cc < NB; ++cc) {
-          uint8_t* box = gbase + C_::P_OFF + ((c0 >> 5) + cc) * 16384 + r * 128;
-#pragma unroll
-          for (int k = 0; k < 8; ++k)
-            *reinterpret_cast<uint4*>(box + ((k ^ (r & 7)) << 4)) =
-                make_uint4(v[cc][4 * k], v[cc][4 * k + 1], v[cc][4 * k + 2], v[cc][4 * k + 3]);
-        }
-      }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar(14));
-      fence_proxy_async();
-      named_barrier_sync(1, 256);
-      if (threadIdx.x == 0) {
-#pragma unroll
-        for (int i = 0; i < HD / 32; ++i)
-          tma_reduce_add_2d(&tmap_dq, base + C_::P_OFF + i * 16384, h * HD + 32 * i, (int)(row0 + qi * 128));
-        bulk_commit_group();
-      }
-    }
-    if (threadIdx.x == 0) bulk_wait_all();
-    if (ok) {
-      // the last wait on the dQ barrier covered every MMA: dV and dK of this key tile are final
-      const long long tok = (long long)row0 + kj * 128 + r;
-      bf16* dk_row = p.dqkv + tok * 3 * d + d + h * HD;
-      bf16* dv_row = p.dqkv + tok * 3 * d + 2 * d + h * HD;
+        const long long tok = (long long)row0 + kj * 128 + kr;
+        bf16* dk_row = p.dqkv + tok * 3 * d + d + h * HD;
+        bf16* dv_row = p.dqkv + tok * 3 * d + 2 * d + h * HD;
 #pragma unroll 1
-      for (int c0 = hc * (HD / 2); c0 < (hc + 1) * (HD / 2); c0 += 32) {
-        uint32_t kv[32], vv[32];
-        tc_ld32(tm_dk + lane_base + c0, kv);
-        tc_ld32(tm_dv + lane_base + c0, vv);
-        tc_wait_ld();
+        for (int c0 = hc * (HD / 2); c0 < (hc + 1) * (HD / 2); c0 += 32) {
+          uint32_t kv[32], vv[32];
+          tc_ld32(tm_dk + lane_base + c0, kv);
+          tc_ld32(tm_dv + lane_base + c0, vv);
+          tc_wait_ld();
 #pragma unroll
-        for (int c = 0; c < 32; c += 8) {
-          uint4 uk, uv;
-          __nv_bfloat162* hk = reinterpret_cast<__nv_bfloat162*>(&uk);
-          __nv_bfloat162* hv = reinterpret_cast<__nv_bfloat162*>(&uv);
+          for (int c = 0; c < 32; c += 8) {
+            uint4 uk, uv;
+            __nv_bfloat162* hk = reinterpret_cast<__nv_bfloat162*>(&uk);
+            __nv_bfloat162* hv = reinterpret_cast<__nv_bfloat162*>(&uv);
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            hk[e] = __floats2bfloat162_rn(__uint_as_float(kv[c + 2 * e]) * p.scale, __uint_as_float(kv[c + 2 * e + 1]) * p.scale);
-            hv[e] = __floats2bfloat162_rn(__uint_as_float(vv[c + 2 * e]), __uint_as_float(vv[c + 2 * e + 1]));
+            for (int e = 0; e < 4; ++e) {
+              hk[e] = __floats2bfloat162_rn(__uint_as_float(kv[c + 2 * e]) * p.scale, __uint_as_float(kv[c + 2 * e + 1]) * p.scale);
+              hv[e] = __floats2bfloat162_rn(__uint_as_float(vv[c + 2 * e]), __uint_as_float(vv[c + 2 * e + 1]));
+            }
+            *reinterpret_cast<uint4*>(dk_row + c0 + c) = uk;
+            *reinterpret_cast<uint4*>(dv_row + c0 + c) = uv;
           }
-          *reinterpret_cast<uint4*>(dk_row + c0 + c) = uk;
-          *reinterpret_cast<uint4*>(dv_row + c0 + c) = uv;
         }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar(C_::DKVREAD));
       }
     }
+    if (tid == 0) bulk_wait_all();
   }
   tc_fence_before();
   __syncthreads();
@@ -649,12 +725,13 @@ fax_status launch_bwd(fax_ctx* ctx, int B, int T, int H, const void* qkv, const 
   p.status = ctx->dev_status;
   static bool attr_set = false;
   if (!attr_set) {
-    FAX_CUDA_TRY(ctx, cudaFuncSetAttribute(attn_bwd_tc_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           BwdCfg<HD>::SMEM_BYTES));
+    FAX_CUDA_TRY(ctx, cudaFuncSetAttribute(attn_bwd2_tc_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           Bwd2Cfg<HD>::SMEM_BYTES));
     attr_set = true;
   }
-  const int grid = B * H * (T / 128);
-  attn_bwd_tc_kernel<HD><<<grid, BWD_THREADS, BwdCfg<HD>::SMEM_BYTES, ctx->stream>>>(mq, md, mdq, p);
+  const long long items = (long long)B * H * (T / 128);
+  const int grid = (int)(items < ctx->sm_count ? items : ctx->sm_count);
+  attn_bwd2_tc_kernel<HD><<<grid, BWD_THREADS, Bwd2Cfg<HD>::SMEM_BYTES, ctx->stream>>>(mq, md, mdq, p);
   FAX_TRY(fax_after_launch(ctx));
   const long long quads = n_tok * (long long)d / 4;
   attn_dq_convert_kernel<<<(unsigned)((quads + 255) / 256), 256, 0, ctx->stream>>>(n_tok, (int)d, dq_acc, p.scale,
