@@ -235,7 +235,7 @@ def run_ours(args):
         lm = dict(wte=rand((cfg.vocab, cfg.d_model), 0.02), wpe=rand((cfg.seq, cfg.d_model), 0.02),
                   blocks=[block_params() for _ in range(cfg.n_layers)],
                   lnf_g=torch.ones(cfg.d_model), lnf_b=torch.zeros(cfg.d_model))
-        runner = LmRunner(sess, cfg, lm, fx.FAX_PREC_BF16, weight_decay=wd)
+        runner = LmRunner(sess, cfg, lm, fx.FAX_PREC_BF16, weight_decay=wd, recompute=args.recompute)
         raw = torch.randint(0, cfg.vocab, (cfg.batch, cfg.seq + 1), generator=gen, device=dev, dtype=torch.int32)
         ids, tg = raw[:, :-1].contiguous(), raw[:, 1:].contiguous()
         ids_h, tg_h = ids.cpu().pin_memory(), tg.cpu().pin_memory()
@@ -249,7 +249,8 @@ def run_ours(args):
             step_no[0] += 1
             runner.step_host(ids_h, tg_h, hparams(step=step_no[0], **hp0))
     else:
-        runner = BlockRunner(sess, cfg, block_params(), fx.FAX_PREC_BF16, weight_decay=wd, host_io=True)
+        runner = BlockRunner(sess, cfg, block_params(), fx.FAX_PREC_BF16, weight_decay=wd, host_io=True,
+                             recompute=args.recompute)
         x = torch.randn((cfg.tokens, cfg.d_model), generator=gen, device=dev).to(torch.bfloat16)
         dy = torch.randn((cfg.tokens, cfg.d_model), generator=gen, device=dev).to(torch.bfloat16)
         x_h, dy_h = x.cpu().pin_memory(), dy.cpu().pin_memory()
@@ -365,7 +366,7 @@ def run_ours(args):
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": workload_name(cfg), "tokens_per_step": tokens, "params": cfg.n_params,
-                   "replicas": world, "fused_update": args.fused_update, "l2": "working set per step far exceeds the 126 MB L2"
+                   "replicas": world, "fused_update": args.fused_update, "recompute": bool(args.recompute), "l2": "working set per step far exceeds the 126 MB L2"
                    if cfg.n_params * 2 > 200e6 else "working set is L2-resident (small parity config)"},
         "mfu": {"step_flops": flops, "achieved_tflops": achieved_tf,
                 "vs_nominal_2250": achieved_tf / NOMINAL_BF16_TFLOPS,
@@ -390,6 +391,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", default="C3", choices=["C1", "C2", "C3", "C4", "C5", "P1", "P2", "P3", "F3", "F2"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--recompute", action="store_true",
+                    help="backward recomputes the LayerNorm outputs and GELU(h) instead of reading saved copies")
     ap.add_argument("--fused-update", default="off", choices=["off", "keep", "nograd"],
                     help="AdamW of the weight matrices in the dW GEMM epilogue: off; on and the gradients still "
                          "stored (default: every output of the step as documented); on without storing them")

@@ -96,6 +96,11 @@ typedef struct {
   int32_t batch, seq, d_model, n_heads, head_dim, d_ff;
   float ln_eps;
   int32_t prec; /* fax_precision */
+  /* 0: forward keeps both LayerNorm outputs and GELU(h) in the saved arena.  1: it keeps them only in the
+   * scratch arena for its own use and backward recomputes them (two LayerNorm passes and one GELU pass
+   * more per block) with the same kernels, so the gradients are the same: the saved arena shrinks by
+   * N*(2d + f) elements per block.  Forward then needs the scratch arena too. */
+  int32_t recompute;
 } fax_block_cfg;
 
 /* Compute-precision parameters (type T), in this order everywhere. */
@@ -116,7 +121,8 @@ fax_status fax_block_sizes(const fax_block_cfg* cfg, size_t* saved_bytes, size_t
 
 /* Where the pieces live inside the two block arenas (byte offsets from the
  * arena base), for inspection, checkpointing and tests.  saved_off[13]: x, a
- * (LN1 out), qkv, o, x1, m (LN2 out), h, g, mu1, rstd1, mu2, rstd2, lse.
+ * (LN1 out), qkv, o, x1, m (LN2 out), h, g, mu1, rstd1, mu2, rstd2, lse
+ * ((size_t)-1 for a, m, g when cfg->recompute is set: they are not saved).
  * scratch_off[4], valid after fax_block_backward: dh [N,f], dqkv [N,3d],
  * da [N,d] (gradient at LN1's output), dx1 [N,d].  Host pointers. */
 fax_status fax_block_arena_layout(const fax_block_cfg* cfg, size_t* saved_off, size_t* scratch_off);
@@ -127,7 +133,8 @@ fax_status fax_block_arena_layout(const fax_block_cfg* cfg, size_t* saved_off, s
  *   x1 = x + o Wo + bo        m = LN(x1; ln2)
  *   h = m W1 + b1             g = GELU_tanh(h)          y = x1 + g W2 + b2
  * x [N,d] T in; y [N,d] T out; `saved` receives what backward needs
- * (x, LN statistics, a, qkv, o, log-sum-exp, x1, m, h, g).  y may not alias x. */
+ * (x, LN statistics, a, qkv, o, log-sum-exp, x1, m, h, g).  y may not alias x.
+ * `scratch` is used (and must hold fax_block_sizes' scratch bytes) only when cfg->recompute is set. */
 fax_status fax_block_forward(fax_ctx* ctx, const fax_block_cfg* cfg, const fax_block_params* params,
                              const void* x, void* y, void* saved, size_t saved_bytes,
                              void* scratch, size_t scratch_bytes);

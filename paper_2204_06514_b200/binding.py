@@ -38,7 +38,8 @@ class ProfileEntry(C.Structure):
 
 class BlockCfg(C.Structure):
     _fields_ = [("batch", C.c_int32), ("seq", C.c_int32), ("d_model", C.c_int32), ("n_heads", C.c_int32),
-                ("head_dim", C.c_int32), ("d_ff", C.c_int32), ("ln_eps", C.c_float), ("prec", C.c_int32)]
+                ("head_dim", C.c_int32), ("d_ff", C.c_int32), ("ln_eps", C.c_float), ("prec", C.c_int32),
+                ("recompute", C.c_int32)]
 
 
 class BlockParams(C.Structure):

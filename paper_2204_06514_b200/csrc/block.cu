@@ -11,6 +11,7 @@ fax_status fax_block_validate(const fax_block_cfg* c) {
   if ((int64_t)c->n_heads * c->head_dim != c->d_model) return FAX_ERR_INVALID_ARG;
   if (c->prec != FAX_PREC_BF16 && c->prec != FAX_PREC_FP32_VALIDATE) return FAX_ERR_INVALID_ARG;
   if (!(c->ln_eps > 0.f)) return FAX_ERR_INVALID_ARG;
+  if (c->recompute != 0 && c->recompute != 1) return FAX_ERR_INVALID_ARG;
   if ((int64_t)c->batch * c->seq > (1 << 30)) return FAX_ERR_UNSUPPORTED_SHAPE;
   if (c->head_dim > 128) return FAX_ERR_UNSUPPORTED_SHAPE;
   if (c->prec == FAX_PREC_BF16) {
@@ -26,13 +27,14 @@ void fax_block_carve_saved(const fax_block_cfg* c, FaxArena& ar, bool with_x, Bl
   const size_t es = fax_elem_size(c->prec);
   const size_t N = (size_t)c->batch * c->seq, d = c->d_model, f = c->d_ff;
   s->x = with_x ? ar.take(N * d * es) : nullptr;
-  s->a = ar.take(N * d * es);
+  const bool keep = !c->recompute;       // LayerNorm outputs and GELU(h) are saved unless backward recomputes them
+  s->a = keep ? ar.take(N * d * es) : nullptr;
   s->qkv = ar.take(N * 3 * d * es);
   s->o = ar.take(N * d * es);
   s->x1 = ar.take(N * d * es);
-  s->m = ar.take(N * d * es);
+  s->m = keep ? ar.take(N * d * es) : nullptr;
   s->h = ar.take(N * f * es);
-  s->g = ar.take(N * f * es);
+  s->g = keep ? ar.take(N * f * es) : nullptr;
   s->mu1 = (float*)ar.take(N * 4);
   s->rstd1 = (float*)ar.take(N * 4);
   s->mu2 = (float*)ar.take(N * 4);
@@ -146,16 +148,21 @@ static fax_status linear_bwd_weight(fax_ctx* ctx, int prec, int N, int K, int No
 }
 
 fax_status fax_block_forward_impl(fax_ctx* ctx, const fax_block_cfg* c, const fax_block_params* p,
-                                  const void* x, void* y, const BlockSaved& s, bool copy_x) {
+                                  const void* x, void* y, const BlockSaved& s, bool copy_x, const BlockScratch* w) {
   const int N = c->batch * c->seq, d = c->d_model, f = c->d_ff, prec = c->prec;
-  FAX_TRY(fax_layernorm_fwd(ctx, prec, N, d, x, p->ln1_g, p->ln1_b, c->ln_eps, s.a, s.mu1, s.rstd1,
+  if (c->recompute && !w) return FAX_ERR_INVALID_ARG;
+  // with recomputation the LayerNorm outputs and GELU(h) only live until their consumer has run
+  void* a = c->recompute ? w->bufA : s.a;
+  void* m = c->recompute ? w->bufB : s.m;
+  void* g = c->recompute ? w->bufF : s.g;
+  FAX_TRY(fax_layernorm_fwd(ctx, prec, N, d, x, p->ln1_g, p->ln1_b, c->ln_eps, a, s.mu1, s.rstd1,
                             copy_x ? s.x : nullptr));
-  FAX_TRY(linear_fwd(ctx, prec, N, d, 3 * d, s.a, p->w_qkv, p->b_qkv, EPI_BIAS, nullptr, nullptr, s.qkv));
+  FAX_TRY(linear_fwd(ctx, prec, N, d, 3 * d, a, p->w_qkv, p->b_qkv, EPI_BIAS, nullptr, nullptr, s.qkv));
   FAX_TRY(fax_attention_fwd(ctx, prec, c->batch, c->seq, c->n_heads, c->head_dim, s.qkv, s.o, s.lse));
   FAX_TRY(linear_fwd(ctx, prec, N, d, d, s.o, p->w_o, p->b_o, EPI_BIAS_RESID, x, nullptr, s.x1));
-  FAX_TRY(fax_layernorm_fwd(ctx, prec, N, d, s.x1, p->ln2_g, p->ln2_b, c->ln_eps, s.m, s.mu2, s.rstd2, nullptr));
-  FAX_TRY(linear_fwd(ctx, prec, N, d, f, s.m, p->w_fc1, p->b_fc1, EPI_BIAS_GELU, nullptr, s.g, s.h));
-  FAX_TRY(linear_fwd(ctx, prec, N, f, d, s.g, p->w_fc2, p->b_fc2, EPI_BIAS_RESID, s.x1, nullptr, y));
+  FAX_TRY(fax_layernorm_fwd(ctx, prec, N, d, s.x1, p->ln2_g, p->ln2_b, c->ln_eps, m, s.mu2, s.rstd2, nullptr));
+  FAX_TRY(linear_fwd(ctx, prec, N, d, f, m, p->w_fc1, p->b_fc1, EPI_BIAS_GELU, nullptr, g, s.h));
+  FAX_TRY(linear_fwd(ctx, prec, N, f, d, g, p->w_fc2, p->b_fc2, EPI_BIAS_RESID, s.x1, nullptr, y));
   return FAX_OK;
 }
 
@@ -166,7 +173,13 @@ fax_status fax_block_backward_impl(fax_ctx* ctx, const fax_block_cfg* c, const f
   const int N = c->batch * c->seq, d = c->d_model, f = c->d_ff, prec = c->prec;
   // once both gradients of a linear layer (or LayerNorm) exist and the data-gradient GEMM has
   // consumed the old weight, its AdamW update runs on the optimizer stream under the rest of backward
-  const bool try_fuse = hook && ctx->fused_update && prec == FAX_PREC_BF16 && !acc;
+  const bool rc = c->recompute != 0;
+  // (the fused update rewrites a weight inside its dW GEMM, so the dX GEMM must come first: not with
+  // recomputation, where FC2's dW runs before its dX to free the GELU buffer)
+  const bool try_fuse = hook && ctx->fused_update && prec == FAX_PREC_BF16 && !acc && !rc;
+  // recomputed LayerNorm outputs need throw-away statistics: the head of the column-sum scratch
+  if (rc && w.partial_floats < (size_t)2 * N) return FAX_ERR_WORKSPACE_TOO_SMALL;
+  float* tmp_mu = w.partial; float* tmp_rstd = w.partial + N;
   auto update = [&](int first, bool matrix_done = false) -> fax_status {
     if (!hook) return FAX_OK;
     return matrix_done ? fax_adamw_async(ctx, hook->t + first + 1, 1, hook->hp)      // only the bias is left
@@ -174,14 +187,26 @@ fax_status fax_block_backward_impl(fax_ctx* ctx, const fax_block_cfg* c, const f
   };
   bool fz = false;
   // B1: through FC2 and GELU
-  FAX_TRY(linear_bwd_data(ctx, prec, N, f, d, dy, p->w_fc2, EPI_DGELU, s.h, w.bufF));          // dh
-  FAX_TRY(linear_bwd_weight(ctx, prec, N, f, d, s.g, dy, gr->w_fc2, acc, try_fuse ? hook->t + 10 : nullptr,
-                            try_fuse ? hook->hp : nullptr, &fz));
+  if (rc) {
+    // g = GELU(h) again, into the buffer that receives dh afterwards: dW2 first, then dh over it
+    FAX_TRY(fax_gelu_fwd(ctx, prec, (size_t)N * f, s.h, w.bufF));
+    FAX_TRY(linear_bwd_weight(ctx, prec, N, f, d, w.bufF, dy, gr->w_fc2, acc, nullptr, nullptr, &fz));
+    FAX_TRY(linear_bwd_data(ctx, prec, N, f, d, dy, p->w_fc2, EPI_DGELU, s.h, w.bufF));        // dh
+  } else {
+    FAX_TRY(linear_bwd_data(ctx, prec, N, f, d, dy, p->w_fc2, EPI_DGELU, s.h, w.bufF));        // dh
+    FAX_TRY(linear_bwd_weight(ctx, prec, N, f, d, s.g, dy, gr->w_fc2, acc, try_fuse ? hook->t + 10 : nullptr,
+                              try_fuse ? hook->hp : nullptr, &fz));
+  }
   FAX_TRY(fax_colsum(ctx, prec, N, d, dy, d, gr->b_fc2, acc, w.partial, w.partial_floats));
   FAX_TRY(update(10, fz));
   // B2: through FC1
   FAX_TRY(linear_bwd_data(ctx, prec, N, d, f, w.bufF, p->w_fc1, EPI_NONE, nullptr, w.bufA));    // dm
-  FAX_TRY(linear_bwd_weight(ctx, prec, N, d, f, s.m, w.bufF, gr->w_fc1, acc, try_fuse ? hook->t + 8 : nullptr,
+  const void* m_in = s.m;
+  if (rc) {   // m = LN2(x1) again, into the buffer that receives dx1 in B3
+    FAX_TRY(fax_layernorm_fwd(ctx, prec, N, d, s.x1, p->ln2_g, p->ln2_b, c->ln_eps, w.bufB, tmp_mu, tmp_rstd, nullptr));
+    m_in = w.bufB;
+  }
+  FAX_TRY(linear_bwd_weight(ctx, prec, N, d, f, m_in, w.bufF, gr->w_fc1, acc, try_fuse ? hook->t + 8 : nullptr,
                             try_fuse ? hook->hp : nullptr, &fz));
   FAX_TRY(fax_colsum(ctx, prec, N, f, w.bufF, f, gr->b_fc1, acc, w.partial, w.partial_floats));
   FAX_TRY(update(8, fz));
@@ -200,7 +225,12 @@ fax_status fax_block_backward_impl(fax_ctx* ctx, const fax_block_cfg* c, const f
                             w.bufA, w.bufQ, w.attn, w.attn_bytes));                             // dqkv
   // B6: through the QKV projection
   FAX_TRY(linear_bwd_data(ctx, prec, N, d, 3 * d, w.bufQ, p->w_qkv, EPI_NONE, nullptr, w.bufA)); // da
-  FAX_TRY(linear_bwd_weight(ctx, prec, N, d, 3 * d, s.a, w.bufQ, gr->w_qkv, acc, try_fuse ? hook->t + 2 : nullptr,
+  const void* a_in = s.a;
+  if (rc) {   // a = LN1(x) again, into the (by now free) dh buffer
+    FAX_TRY(fax_layernorm_fwd(ctx, prec, N, d, x, p->ln1_g, p->ln1_b, c->ln_eps, w.bufF, tmp_mu, tmp_rstd, nullptr));
+    a_in = w.bufF;
+  }
+  FAX_TRY(linear_bwd_weight(ctx, prec, N, d, 3 * d, a_in, w.bufQ, gr->w_qkv, acc, try_fuse ? hook->t + 2 : nullptr,
                             try_fuse ? hook->hp : nullptr, &fz));
   FAX_TRY(fax_colsum(ctx, prec, N, 3 * d, w.bufQ, 3 * d, gr->b_qkv, acc, w.partial, w.partial_floats));
   FAX_TRY(update(2, fz));
@@ -225,12 +255,17 @@ extern "C" fax_status fax_block_forward(fax_ctx* ctx, const fax_block_cfg* cfg, 
   FAX_TRY(fax_block_validate(cfg));
   FAX_TRY(check_params(params));
   if (!fax_aligned(x, 16) || !fax_aligned(y, 16) || !fax_aligned(saved, 256)) return FAX_ERR_INVALID_ARG;
-  (void)scratch; (void)scratch_bytes;
   FaxArena ar(saved, saved_bytes);
   BlockSaved s;
   fax_block_carve_saved(cfg, ar, true, &s);
   if (ar.used() > saved_bytes) return FAX_ERR_WORKSPACE_TOO_SMALL;
-  return fax_block_forward_impl(ctx, cfg, params, x, y, s, true);
+  if (!cfg->recompute) return fax_block_forward_impl(ctx, cfg, params, x, y, s, true);
+  if (!scratch || !fax_aligned(scratch, 256)) return FAX_ERR_INVALID_ARG;
+  FaxArena aw(scratch, scratch_bytes);
+  BlockScratch w;
+  fax_block_carve_scratch(cfg, aw, &w);
+  if (aw.used() > scratch_bytes) return FAX_ERR_WORKSPACE_TOO_SMALL;
+  return fax_block_forward_impl(ctx, cfg, params, x, y, s, true, &w);
 }
 
 extern "C" fax_status fax_block_backward(fax_ctx* ctx, const fax_block_cfg* cfg, const fax_block_params* params,
@@ -312,7 +347,7 @@ static fax_status block_step_impl(fax_ctx* ctx, const fax_block_cfg* cfg, const 
     FAX_CUDA_TRY(ctx, cudaMemcpyAsync(io->dy_dev, io->dy_host, io->bytes, cudaMemcpyHostToDevice, ctx->copy));
     FAX_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_copy_b, ctx->copy));
   }
-  FAX_TRY(fax_block_forward_impl(ctx, cfg, &p, x, y, s, true));
+  FAX_TRY(fax_block_forward_impl(ctx, cfg, &p, x, y, s, true, &w));
   if (io) {
     FAX_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_copy_a, ctx->stream));              // y is complete
     FAX_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->copy, ctx->ev_copy_a, 0));

@@ -15,7 +15,8 @@ struct BlockScratch {
 void fax_block_carve_saved(const fax_block_cfg* c, FaxArena& ar, bool with_x, BlockSaved* s);
 void fax_block_carve_scratch(const fax_block_cfg* c, FaxArena& ar, BlockScratch* s);
 fax_status fax_block_forward_impl(fax_ctx* ctx, const fax_block_cfg* c, const fax_block_params* p,
-                                  const void* x, void* y, const BlockSaved& s, bool copy_x);
+                                  const void* x, void* y, const BlockSaved& s, bool copy_x,
+                                  const BlockScratch* w = nullptr);
 fax_status fax_block_backward_impl(fax_ctx* ctx, const fax_block_cfg* c, const fax_block_params* p,
                                    const void* dy, const BlockSaved& s, const void* x, void* dx,
                                    const fax_block_grads* gr, bool acc, const BlockScratch& w,

@@ -241,6 +241,8 @@ fax_status fax_loss_mean(fax_ctx* ctx, int n, const float* row_loss, float* loss
 
 bool fax_attention_tc_supported(int B, int T, int H, int hd);
 fax_status fax_attention_fwd_tc(fax_ctx* ctx, int B, int T, int H, int hd, const void* qkv, void* o, float* lse);
+// g = GELU_tanh(h) element-wise with the function the FC1 epilogue uses (n elements of the precision's type)
+fax_status fax_gelu_fwd(fax_ctx* ctx, int prec, size_t n, const void* h, void* g);
 bool fax_attention_fwd2_supported(int B, int T, int H, int hd);
 fax_status fax_attention_fwd2_tc(fax_ctx* ctx, int B, int T, int H, int hd, const void* qkv, void* o, float* lse);
 size_t fax_attention_bwd_tc_scratch_bytes(int B, int T, int H, int hd);

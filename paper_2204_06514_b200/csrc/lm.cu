@@ -96,7 +96,7 @@ fax_status lm_fwd_bwd(fax_ctx* ctx, const fax_lm_cfg* c, const fax_lm_state* st,
   for (int l = 0; l < L; ++l) {
     fax_block_params p; fax_block_grads g;
     fax_layer_views(&st->layers[l], prec, &p, &g);
-    FAX_TRY(fax_block_forward_impl(ctx, bc, &p, sv.act[l], sv.act[l + 1], sv.blk[l], false));
+    FAX_TRY(fax_block_forward_impl(ctx, bc, &p, sv.act[l], sv.act[l + 1], sv.blk[l], false, &w.blk));
   }
   FAX_TRY(fax_layernorm_fwd(ctx, prec, N, d, sv.act[L], lnf_g, lnf_b, bc->ln_eps, sv.xf, sv.muf, sv.rstdf, nullptr));
 

@@ -18,8 +18,9 @@ def _ptr(t: torch.Tensor | None):
     return C.c_void_p(0 if t is None else t.data_ptr())
 
 
-def block_cfg(cfg: Config, prec: int) -> fx.BlockCfg:
-    return fx.BlockCfg(cfg.batch, cfg.seq, cfg.d_model, cfg.n_heads, cfg.head_dim, cfg.d_ff, cfg.ln_eps, prec)
+def block_cfg(cfg: Config, prec: int, recompute: int = 0) -> fx.BlockCfg:
+    return fx.BlockCfg(cfg.batch, cfg.seq, cfg.d_model, cfg.n_heads, cfg.head_dim, cfg.d_ff, cfg.ln_eps, prec,
+                       recompute)
 
 
 def hparams(lr, beta1, beta2, eps, step, grad_is_bf16=0, **_) -> fx.AdamwHparams:
@@ -75,9 +76,9 @@ class BlockRunner:
     """One decoder block with its training state resident on the device."""
 
     def __init__(self, sess: Session, cfg: Config, params: dict, prec: int = fx.FAX_PREC_BF16,
-                 weight_decay: float = 0.1, host_io: bool = False):
+                 weight_decay: float = 0.1, host_io: bool = False, recompute: bool = False):
         self.sess, self.cfg, self.prec = sess, cfg, prec
-        self.bcfg = block_cfg(cfg, prec)
+        self.bcfg = block_cfg(cfg, prec, int(recompute))
         self.dtype = torch.bfloat16 if prec == fx.FAX_PREC_BF16 else torch.float32
         self.p = {k: ParamSet(params[k], prec, sess.device, weight_decay) for k in PARAM_NAMES}
         self.saved_bytes, self.scratch_bytes = fx.fax_block_sizes(self.bcfg)
@@ -122,9 +123,9 @@ class LmRunner:
     """N-layer LM with its training state resident on the device."""
 
     def __init__(self, sess: Session, cfg: Config, lm: dict, prec: int = fx.FAX_PREC_BF16,
-                 weight_decay: float = 0.1):
+                 weight_decay: float = 0.1, recompute: bool = False):
         self.sess, self.cfg, self.prec = sess, cfg, prec
-        self.lcfg = fx.LmCfg(cfg.n_layers, cfg.vocab, lm["wpe"].shape[0], block_cfg(cfg, prec))
+        self.lcfg = fx.LmCfg(cfg.n_layers, cfg.vocab, lm["wpe"].shape[0], block_cfg(cfg, prec, int(recompute)))
         mk = lambda a: ParamSet(a, prec, sess.device, weight_decay)
         self.wte, self.wpe = mk(lm["wte"]), mk(lm["wpe"])
         self.lnf_g, self.lnf_b = mk(lm["lnf_g"]), mk(lm["lnf_b"])
