@@ -52,11 +52,18 @@ __device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, 
 }
 
 // Epilogue of one 32-column chunk held in registers: row `row`, columns col .. col+31.
-__device__ __forceinline__ void gemm_epilogue_chunk(const GemmParams& p, const uint32_t (&r)[32], long long row, int col) {
+// EPI >= 0: the epilogue mode is a compile-time constant and the output is bf16 (the kernels
+// are instantiated per mode, which keeps each one's epilogue code short and branch-free);
+// EPI < 0: mode, output type, accumulation and K-slicing are read from the parameters.
+template <int EPI>
+__device__ __forceinline__ void gemm_epilogue_chunk(const GemmParams& pr, const uint32_t (&r)[32], long long row, int col) {
+        const GemmParams& p = pr;
+        const int p_epi = EPI >= 0 ? EPI : pr.epi;
+        const bool p_c_f32 = EPI >= 0 ? false : (pr.c_f32 != 0);
         float v[32];
 #pragma unroll
         for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) * p.alpha;
-        if (p.epi == EPI_BIAS || p.epi == EPI_BIAS_GELU || p.epi == EPI_BIAS_RESID) {
+        if (p_epi == EPI_BIAS || p_epi == EPI_BIAS_GELU || p_epi == EPI_BIAS_RESID) {
           const uint4* bp = reinterpret_cast<const uint4*>(p.bias + col);
 #pragma unroll
           for (int j4 = 0; j4 < 4; ++j4) {
@@ -66,7 +73,7 @@ __device__ __forceinline__ void gemm_epilogue_chunk(const GemmParams& p, const u
             for (int e = 0; e < 4; ++e) { float2 f = __bfloat1622float2(h[e]); v[8 * j4 + 2 * e] += f.x; v[8 * j4 + 2 * e + 1] += f.y; }
           }
         }
-        if (p.epi == EPI_BIAS_RESID) {
+        if (p_epi == EPI_BIAS_RESID) {
           const bf16* rp = p.resid + row * p.ldr + col;
 #pragma unroll
           for (int j8 = 0; j8 < 2; ++j8) {
@@ -78,7 +85,7 @@ __device__ __forceinline__ void gemm_epilogue_chunk(const GemmParams& p, const u
             }
           }
         }
-        if (p.epi == EPI_DGELU) {
+        if (p_epi == EPI_DGELU) {
           const bf16* ap = p.aux + row * p.ldaux + col;
 #pragma unroll
           for (int j8 = 0; j8 < 2; ++j8) {
@@ -91,7 +98,7 @@ __device__ __forceinline__ void gemm_epilogue_chunk(const GemmParams& p, const u
             }
           }
         }
-        if (p.epi == EPI_ADAMW) {
+        if (p_epi == EPI_ADAMW) {
           // the accumulator is the gradient of w[row, col..]: AdamW here, w / m / v in place
           const long long off = row * p.ldc + col;
           const float lr = p.ad_sc[0], b1 = p.ad_sc[1], b2 = p.ad_sc[2], eps = p.ad_sc[3];
@@ -128,7 +135,7 @@ __device__ __forceinline__ void gemm_epilogue_chunk(const GemmParams& p, const u
               st_global_v8((float*)p.C + off + 8 * j8, g8);
             }
           }
-        } else if (p.c_f32) {
+        } else if (p_c_f32) {
           float* cp = (float*)p.C + row * p.ldc + col;
           if (p.splits > 1) {
 #pragma unroll
@@ -150,7 +157,7 @@ __device__ __forceinline__ void gemm_epilogue_chunk(const GemmParams& p, const u
           }
         } else {
           bf16* cp = (bf16*)p.C + row * p.ldc + col;
-          bf16* gp = (p.epi == EPI_BIAS_GELU) ? (p.aux + row * p.ldaux + col) : nullptr;
+          bf16* gp = (p_epi == EPI_BIAS_GELU) ? (p.aux + row * p.ldaux + col) : nullptr;
 #pragma unroll
           for (int j8 = 0; j8 < 2; ++j8) {
             U8 u;
@@ -173,6 +180,11 @@ __device__ __forceinline__ void gemm_epilogue_chunk(const GemmParams& p, const u
             }
           }
         }
+}
+
+// The compile-time epilogue mode a problem runs with (see gemm_epilogue_chunk).
+static inline int gemm_static_epi(const FaxGemm& g) {
+  return (!g.c_f32 && !g.adam && g.epi >= EPI_NONE && g.epi <= EPI_DGELU) ? g.epi : -1;
 }
 
 // Fills the kernel parameters that do not depend on the tile shape.
@@ -208,20 +220,23 @@ static inline int gemm_split_count(const FaxGemm& g, int tiles, int units, int b
 
 // One warp's share of a tile: NCH chunks of 32 columns starting at tensor-memory address
 // t_base / global column col0.  Two register buffers keep the load of the next chunk in
-// flight while the current one is stored.
-template <int NCH>
-__device__ __forceinline__ void gemm_epilogue_warp(const GemmParams& p, uint32_t t_base, long long row, int col0) {
+// flight while the current one is stored.  `drained` runs as soon as the last chunk has been
+// read out of tensor memory (before its stores): the accumulator can be handed back to the MMA
+// issuer while this warp is still writing to global memory.
+template <int NCH, int EPI, typename Drained>
+__device__ __forceinline__ void gemm_epilogue_warp(const GemmParams& p, uint32_t t_base, long long row, int col0,
+                                                   Drained drained) {
   uint32_t ra[32], rb[32];
   tc_ld32(t_base, ra);
 #pragma unroll
   for (int i = 0; i < NCH; i += 2) {
     tc_wait_ld();
-    if (i + 1 < NCH) tc_ld32(t_base + 32 * (i + 1), rb);
-    gemm_epilogue_chunk(p, ra, row, col0 + 32 * i);
+    if (i + 1 < NCH) tc_ld32(t_base + 32 * (i + 1), rb); else drained();
+    gemm_epilogue_chunk<EPI>(p, ra, row, col0 + 32 * i);
     if (i + 1 < NCH) {
       tc_wait_ld();
-      if (i + 2 < NCH) tc_ld32(t_base + 32 * (i + 2), ra);
-      gemm_epilogue_chunk(p, rb, row, col0 + 32 * (i + 1));
+      if (i + 2 < NCH) tc_ld32(t_base + 32 * (i + 2), ra); else drained();
+      gemm_epilogue_chunk<EPI>(p, rb, row, col0 + 32 * (i + 1));
     }
   }
 }

@@ -168,10 +168,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       tc_fence_after();
       const long long row = m0 + 32 * q + lane;
       const uint32_t t_base = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(acc * BN + half * (BN / 2));
-      gemm_epilogue_warp<NCH>(p, t_base, row, n0 + half * (BN / 2));
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(tempty_bar(acc));
+      gemm_epilogue_warp<NCH, -1>(p, t_base, row, n0 + half * (BN / 2), [&]() {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_relaxed(tempty_bar(acc));
+      });
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
   }

@@ -53,8 +53,11 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
       "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1) : "memory");
 }
+// Arrival on a barrier of the pair's even CTA.  Relaxed: what it orders is this warp's
+// tensor-memory reads, which tcgen05.wait::ld and the tcgen05 fence have already completed; a
+// release at cluster scope would also wait until the warp's global stores have drained.
 __device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
+  asm volatile("mbarrier.arrive.relaxed.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
@@ -69,6 +72,7 @@ __device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t adesc
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
 
+template <int EPI>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                          const GemmParams p) {
@@ -199,10 +203,11 @@ gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
       tc_fence_after();
       const long long row = m0 + 32 * q + lane;
       const uint32_t t_base = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(acc * BN + half * (BN / 2));
-      gemm_epilogue_warp<NCH>(p, t_base, row, n0 + half * (BN / 2));
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(leader_addr(tempty_bar(acc)));
+      gemm_epilogue_warp<NCH, EPI>(p, t_base, row, n0 + half * (BN / 2), [&]() {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_cluster(leader_addr(tempty_bar(acc)));
+      });
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
   }
@@ -219,7 +224,7 @@ gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
 }  // namespace
 
 bool fax_gemm_patch_info_2cta(const void* func, const void* param, size_t* size, size_t* sc_offset) {
-  if (func != (const void*)gemm_tcgen05_2cta_kernel) return false;
+  if (func != (const void*)gemm_tcgen05_2cta_kernel<-1>) return false;
   if (((const GemmParams*)param)->epi != EPI_ADAMW) return false;
   *size = sizeof(GemmParams);
   *sc_offset = offsetof(GemmParams, ad_sc);
@@ -240,7 +245,9 @@ fax_status fax_gemm_tc2(fax_ctx* ctx, const FaxGemm& g) {
   fill_gemm_params(p, g, ctx->dev_status);
   static bool attr_set = false;
   if (!attr_set) {
-    FAX_CUDA_TRY(ctx, cudaFuncSetAttribute(gemm_tcgen05_2cta_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+#define FAX_SET_SMEM(E) FAX_CUDA_TRY(ctx, cudaFuncSetAttribute(gemm_tcgen05_2cta_kernel<E>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))
+    FAX_SET_SMEM(-1); FAX_SET_SMEM(0); FAX_SET_SMEM(1); FAX_SET_SMEM(2); FAX_SET_SMEM(3); FAX_SET_SMEM(4);
+#undef FAX_SET_SMEM
     attr_set = true;
   }
   const int tiles = (g.M / 256) * (g.N / 256);
@@ -250,6 +257,11 @@ fax_status fax_gemm_tc2(fax_ctx* ctx, const FaxGemm& g) {
     FAX_CUDA_TRY(ctx, cudaMemset2DAsync(g.C, (size_t)g.ldc * 4, 0, (size_t)g.N * 4, (size_t)g.M, ctx->stream));
   const int items = tiles * p.splits;
   const int pairs = items < max_pairs ? items : max_pairs;
-  gemm_tcgen05_2cta_kernel<<<2 * pairs, NUM_THREADS, SMEM_BYTES, ctx->stream>>>(ma, mb, p);
+  switch (gemm_static_epi(g)) {
+#define FAX_LAUNCH(E) case E: gemm_tcgen05_2cta_kernel<E><<<2 * pairs, NUM_THREADS, SMEM_BYTES, ctx->stream>>>(ma, mb, p); break
+    FAX_LAUNCH(0); FAX_LAUNCH(1); FAX_LAUNCH(2); FAX_LAUNCH(3); FAX_LAUNCH(4);
+    default: gemm_tcgen05_2cta_kernel<-1><<<2 * pairs, NUM_THREADS, SMEM_BYTES, ctx->stream>>>(ma, mb, p); break;
+#undef FAX_LAUNCH
+  }
   return fax_after_launch(ctx);
 }
