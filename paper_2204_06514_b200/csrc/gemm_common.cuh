@@ -55,11 +55,32 @@ __device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, 
 // EPI >= 0: the epilogue mode is a compile-time constant and the output is bf16 (the kernels
 // are instantiated per mode, which keeps each one's epilogue code short and branch-free);
 // EPI < 0: mode, output type, accumulation and K-slicing are read from the parameters.
+// The residual / pre-activation values one chunk needs (32 bf16 of row `row` from column col),
+// requested ahead of the chunk's turn so that their latency hides under the previous chunk.
+// (Only the kernels with a compile-time mode fetch ahead; the run-time-mode epilogue loads the
+// values when it needs them, which keeps it within its register budget.)
+template <int EPI, bool NOW = false>
+__device__ __forceinline__ void gemm_epilogue_fetch(const GemmParams& p, long long row, int col, U8 (&x)[2]) {
+  if (EPI < 0 && !NOW) return;
+  const int epi = EPI >= 0 ? EPI : p.epi;
+  if (epi == EPI_BIAS_RESID) {
+    const bf16* rp = p.resid + row * p.ldr + col;
+    x[0] = ld_global_v8(rp); x[1] = ld_global_v8(rp + 16);
+  } else if (epi == EPI_DGELU) {
+    const bf16* ap = p.aux + row * p.ldaux + col;
+    x[0] = ld_global_v8(ap); x[1] = ld_global_v8(ap + 16);
+  }
+}
+
 template <int EPI>
-__device__ __forceinline__ void gemm_epilogue_chunk(const GemmParams& pr, const uint32_t (&r)[32], long long row, int col) {
+__device__ __forceinline__ void gemm_epilogue_chunk(const GemmParams& pr, const uint32_t (&r)[32], const U8 (&x)[2],
+                                                    long long row, int col) {
         const GemmParams& p = pr;
         const int p_epi = EPI >= 0 ? EPI : pr.epi;
         const bool p_c_f32 = EPI >= 0 ? false : (pr.c_f32 != 0);
+        U8 xn[2];
+        if (EPI < 0) gemm_epilogue_fetch<EPI, true>(pr, row, col, xn);
+        const U8* xv = EPI < 0 ? xn : x;
         float v[32];
 #pragma unroll
         for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) * p.alpha;
@@ -74,10 +95,9 @@ __device__ __forceinline__ void gemm_epilogue_chunk(const GemmParams& pr, const 
           }
         }
         if (p_epi == EPI_BIAS_RESID) {
-          const bf16* rp = p.resid + row * p.ldr + col;
 #pragma unroll
           for (int j8 = 0; j8 < 2; ++j8) {
-            const U8 u = ld_global_v8(rp + 16 * j8);
+            const U8& u = xv[j8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
               float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u.w[e]));
@@ -86,10 +106,9 @@ __device__ __forceinline__ void gemm_epilogue_chunk(const GemmParams& pr, const 
           }
         }
         if (p_epi == EPI_DGELU) {
-          const bf16* ap = p.aux + row * p.ldaux + col;
 #pragma unroll
           for (int j8 = 0; j8 < 2; ++j8) {
-            const U8 u = ld_global_v8(ap + 16 * j8);
+            const U8& u = xv[j8];
 #pragma unroll
             for (int e = 0; e < 8; ++e) {
               float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&u.w[e]));
@@ -220,23 +239,28 @@ static inline int gemm_split_count(const FaxGemm& g, int tiles, int units, int b
 
 // One warp's share of a tile: NCH chunks of 32 columns starting at tensor-memory address
 // t_base / global column col0.  Two register buffers keep the load of the next chunk in
-// flight while the current one is stored.  `drained` runs as soon as the last chunk has been
+// flight while the current one is stored; x0 holds the first chunk's residual / pre-activation
+// values (gemm_epilogue_fetch, issued by the caller before it waits for the accumulator).  `drained` runs as soon as the last chunk has been
 // read out of tensor memory (before its stores): the accumulator can be handed back to the MMA
 // issuer while this warp is still writing to global memory.
 template <int NCH, int EPI, typename Drained>
 __device__ __forceinline__ void gemm_epilogue_warp(const GemmParams& p, uint32_t t_base, long long row, int col0,
-                                                   Drained drained) {
+                                                   const U8 (&x0)[2], Drained drained) {
   uint32_t ra[32], rb[32];
+  U8 xa[2], xb[2];
+  xa[0] = x0[0]; xa[1] = x0[1];
   tc_ld32(t_base, ra);
 #pragma unroll
   for (int i = 0; i < NCH; i += 2) {
+    if (i + 1 < NCH) gemm_epilogue_fetch<EPI>(p, row, col0 + 32 * (i + 1), xb);
     tc_wait_ld();
     if (i + 1 < NCH) tc_ld32(t_base + 32 * (i + 1), rb); else drained();
-    gemm_epilogue_chunk<EPI>(p, ra, row, col0 + 32 * i);
+    gemm_epilogue_chunk<EPI>(p, ra, xa, row, col0 + 32 * i);
     if (i + 1 < NCH) {
+      if (i + 2 < NCH) gemm_epilogue_fetch<EPI>(p, row, col0 + 32 * (i + 2), xa);
       tc_wait_ld();
       if (i + 2 < NCH) tc_ld32(t_base + 32 * (i + 2), ra); else drained();
-      gemm_epilogue_chunk<EPI>(p, rb, row, col0 + 32 * (i + 1));
+      gemm_epilogue_chunk<EPI>(p, rb, xb, row, col0 + 32 * (i + 1));
     }
   }
 }

@@ -199,11 +199,13 @@ gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
       int tm, tn;
       tile_coords(tile % out_tiles, tiles_m, tiles_n, p.group_m, tm, tn);
       const int m0 = tm * 2 * BM + (int)rank * BM, n0 = tn * BN;
+      const long long row = m0 + 32 * q + lane;
+      U8 x0[2];
+      gemm_epilogue_fetch<EPI>(p, row, n0 + half * (BN / 2), x0);     // in flight while the accumulator fills
       if (!mbar_wait_warp(tfull_bar(acc), acc_phase, abort_flag, p.status, 114)) { ok = false; break; }
       tc_fence_after();
-      const long long row = m0 + 32 * q + lane;
       const uint32_t t_base = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(acc * BN + half * (BN / 2));
-      gemm_epilogue_warp<NCH, EPI>(p, t_base, row, n0 + half * (BN / 2), [&]() {
+      gemm_epilogue_warp<NCH, EPI>(p, t_base, row, n0 + half * (BN / 2), x0, [&]() {
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster(leader_addr(tempty_bar(acc)));

@@ -9,7 +9,17 @@
 
 namespace {
 
-constexpr int HEAD_ROWS = 8192;     // logits rows per chunk
+// Logits rows per chunk of the head: as many as fit a 4 GiB logits buffer (at least 8192).  Large
+// chunks matter for the dxf GEMM, whose output is only d wide: with 8192 rows and d = 768 it has 96
+// tiles for 74 SM pairs (two waves, the second a third full); all 16384 rows at once need three
+// waves instead of four.
+constexpr int HEAD_ROWS_MIN = 8192;
+constexpr size_t HEAD_LOGITS_BYTES = (size_t)4 << 30;
+int head_rows_for(size_t N, size_t V, size_t es) {
+  size_t rows = HEAD_LOGITS_BYTES / (V * es) / 256 * 256;
+  if (rows < (size_t)HEAD_ROWS_MIN) rows = HEAD_ROWS_MIN;
+  return (int)(N < rows ? N : rows);
+}
 
 struct LmSaved {
   std::vector<void*> act;           // act[l]: input of block l; act[L]: output of the last block
@@ -52,7 +62,7 @@ void carve_scratch(const fax_lm_cfg* c, FaxArena& ar, LmScratch* s) {
   fax_block_carve_scratch(&c->block, ar, &s->blk);
   s->dxa = ar.take(N * d * es);
   s->dxb = ar.take(N * d * es);
-  s->head_rows = N < (size_t)HEAD_ROWS ? (int)N : HEAD_ROWS;
+  s->head_rows = head_rows_for(N, (size_t)c->vocab, es);
   s->logits = ar.take((size_t)s->head_rows * c->vocab * es);
   s->row_loss = (float*)ar.take(N * 4);
 }
