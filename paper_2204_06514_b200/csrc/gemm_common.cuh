@@ -52,9 +52,12 @@ __device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, 
 }
 
 // Epilogue of one 32-column chunk held in registers: row `row`, columns col .. col+31.
-// EPI >= 0: the epilogue mode is a compile-time constant and the output is bf16 (the kernels
-// are instantiated per mode, which keeps each one's epilogue code short and branch-free);
+// EPI >= 0: the epilogue mode is a compile-time constant (the kernels are instantiated per mode,
+// which keeps each one's epilogue code short and branch-free): EPI_NONE .. EPI_DGELU with bf16
+// output, EPI_STATIC_F32 = plain float output (stored, accumulated or added by K slices);
 // EPI < 0: mode, output type, accumulation and K-slicing are read from the parameters.
+constexpr int EPI_STATIC_F32 = 6;
+
 // The residual / pre-activation values one chunk needs (32 bf16 of row `row` from column col),
 // requested ahead of the chunk's turn so that their latency hides under the previous chunk.
 // (Only the kernels with a compile-time mode fetch ahead; the run-time-mode epilogue loads the
@@ -62,7 +65,7 @@ __device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, 
 template <int EPI, bool NOW = false>
 __device__ __forceinline__ void gemm_epilogue_fetch(const GemmParams& p, long long row, int col, U8 (&x)[2]) {
   if (EPI < 0 && !NOW) return;
-  const int epi = EPI >= 0 ? EPI : p.epi;
+  const int epi = EPI == EPI_STATIC_F32 ? (int)EPI_NONE : (EPI >= 0 ? EPI : p.epi);
   if (epi == EPI_BIAS_RESID) {
     const bf16* rp = p.resid + row * p.ldr + col;
     x[0] = ld_global_v8(rp); x[1] = ld_global_v8(rp + 16);
@@ -76,8 +79,8 @@ template <int EPI>
 __device__ __forceinline__ void gemm_epilogue_chunk(const GemmParams& pr, const uint32_t (&r)[32], const U8 (&x)[2],
                                                     long long row, int col) {
         const GemmParams& p = pr;
-        const int p_epi = EPI >= 0 ? EPI : pr.epi;
-        const bool p_c_f32 = EPI >= 0 ? false : (pr.c_f32 != 0);
+        const int p_epi = EPI == EPI_STATIC_F32 ? (int)EPI_NONE : (EPI >= 0 ? EPI : pr.epi);
+        const bool p_c_f32 = EPI == EPI_STATIC_F32 ? true : (EPI >= 0 ? false : (pr.c_f32 != 0));
         U8 xn[2];
         if (EPI < 0) gemm_epilogue_fetch<EPI, true>(pr, row, col, xn);
         const U8* xv = EPI < 0 ? xn : x;
@@ -203,7 +206,9 @@ __device__ __forceinline__ void gemm_epilogue_chunk(const GemmParams& pr, const 
 
 // The compile-time epilogue mode a problem runs with (see gemm_epilogue_chunk).
 static inline int gemm_static_epi(const FaxGemm& g) {
-  return (!g.c_f32 && !g.adam && g.epi >= EPI_NONE && g.epi <= EPI_DGELU) ? g.epi : -1;
+  if (g.adam) return -1;
+  if (g.c_f32) return g.epi == EPI_NONE ? EPI_STATIC_F32 : -1;
+  return (g.epi >= EPI_NONE && g.epi <= EPI_DGELU) ? g.epi : -1;
 }
 
 // Fills the kernel parameters that do not depend on the tile shape.

@@ -249,6 +249,7 @@ fax_status fax_gemm_tc2(fax_ctx* ctx, const FaxGemm& g) {
   if (!attr_set) {
 #define FAX_SET_SMEM(E) FAX_CUDA_TRY(ctx, cudaFuncSetAttribute(gemm_tcgen05_2cta_kernel<E>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))
     FAX_SET_SMEM(-1); FAX_SET_SMEM(0); FAX_SET_SMEM(1); FAX_SET_SMEM(2); FAX_SET_SMEM(3); FAX_SET_SMEM(4);
+    FAX_SET_SMEM(EPI_STATIC_F32);
 #undef FAX_SET_SMEM
     attr_set = true;
   }
@@ -261,7 +262,7 @@ fax_status fax_gemm_tc2(fax_ctx* ctx, const FaxGemm& g) {
   const int pairs = items < max_pairs ? items : max_pairs;
   switch (gemm_static_epi(g)) {
 #define FAX_LAUNCH(E) case E: gemm_tcgen05_2cta_kernel<E><<<2 * pairs, NUM_THREADS, SMEM_BYTES, ctx->stream>>>(ma, mb, p); break
-    FAX_LAUNCH(0); FAX_LAUNCH(1); FAX_LAUNCH(2); FAX_LAUNCH(3); FAX_LAUNCH(4);
+    FAX_LAUNCH(0); FAX_LAUNCH(1); FAX_LAUNCH(2); FAX_LAUNCH(3); FAX_LAUNCH(4); FAX_LAUNCH(EPI_STATIC_F32);
     default: gemm_tcgen05_2cta_kernel<-1><<<2 * pairs, NUM_THREADS, SMEM_BYTES, ctx->stream>>>(ma, mb, p); break;
 #undef FAX_LAUNCH
   }
