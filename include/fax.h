@@ -247,6 +247,10 @@ fax_status fax_block_step_host(fax_ctx* ctx, const fax_block_cfg* cfg, const fax
 typedef struct {
   int32_t n_layers, vocab, max_seq;
   fax_block_cfg block;
+  int32_t head_rows;   /* rows of logits held at a time by the output projection + loss; 0 = as many as
+                          fit a 4 GiB logits buffer (at least 8192).  Positive values must be multiples of
+                          128; the head then walks the batch*seq rows in chunks of that many (the last
+                          one shorter), adding each chunk's share into the gradient of wte. */
 } fax_lm_cfg;
 
 typedef struct {

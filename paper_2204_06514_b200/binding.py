@@ -75,7 +75,8 @@ class BlockState(C.Structure):
 
 
 class LmCfg(C.Structure):
-    _fields_ = [("n_layers", C.c_int32), ("vocab", C.c_int32), ("max_seq", C.c_int32), ("block", BlockCfg)]
+    _fields_ = [("n_layers", C.c_int32), ("vocab", C.c_int32), ("max_seq", C.c_int32), ("block", BlockCfg),
+                ("head_rows", C.c_int32)]
 
 
 class LmState(C.Structure):

@@ -15,9 +15,10 @@ namespace {
 // waves instead of four.
 constexpr int HEAD_ROWS_MIN = 8192;
 constexpr size_t HEAD_LOGITS_BYTES = (size_t)4 << 30;
-int head_rows_for(size_t N, size_t V, size_t es) {
+int head_rows_for(const fax_lm_cfg* c, size_t N, size_t V, size_t es) {
   size_t rows = HEAD_LOGITS_BYTES / (V * es) / 256 * 256;
   if (rows < (size_t)HEAD_ROWS_MIN) rows = HEAD_ROWS_MIN;
+  if (c->head_rows > 0) rows = (size_t)c->head_rows;
   return (int)(N < rows ? N : rows);
 }
 
@@ -38,6 +39,7 @@ fax_status lm_validate(const fax_lm_cfg* c) {
   if (!c) return FAX_ERR_INVALID_ARG;
   FAX_TRY(fax_block_validate(&c->block));
   if (c->n_layers <= 0 || c->vocab <= 0 || c->max_seq < c->block.seq) return FAX_ERR_INVALID_ARG;
+  if (c->head_rows < 0 || c->head_rows % 128) return FAX_ERR_INVALID_ARG;
   if (c->block.prec == FAX_PREC_BF16 && c->vocab % 128) return FAX_ERR_UNSUPPORTED_SHAPE;
   return FAX_OK;
 }
@@ -62,7 +64,7 @@ void carve_scratch(const fax_lm_cfg* c, FaxArena& ar, LmScratch* s) {
   fax_block_carve_scratch(&c->block, ar, &s->blk);
   s->dxa = ar.take(N * d * es);
   s->dxb = ar.take(N * d * es);
-  s->head_rows = head_rows_for(N, (size_t)c->vocab, es);
+  s->head_rows = head_rows_for(c, N, (size_t)c->vocab, es);
   s->logits = ar.take((size_t)s->head_rows * c->vocab * es);
   s->row_loss = (float*)ar.take(N * 4);
 }

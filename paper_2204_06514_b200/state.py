@@ -123,9 +123,10 @@ class LmRunner:
     """N-layer LM with its training state resident on the device."""
 
     def __init__(self, sess: Session, cfg: Config, lm: dict, prec: int = fx.FAX_PREC_BF16,
-                 weight_decay: float = 0.1, recompute: bool = False):
+                 weight_decay: float = 0.1, recompute: bool = False, head_rows: int = 0):
         self.sess, self.cfg, self.prec = sess, cfg, prec
-        self.lcfg = fx.LmCfg(cfg.n_layers, cfg.vocab, lm["wpe"].shape[0], block_cfg(cfg, prec, int(recompute)))
+        self.lcfg = fx.LmCfg(cfg.n_layers, cfg.vocab, lm["wpe"].shape[0], block_cfg(cfg, prec, int(recompute)),
+                             head_rows)
         mk = lambda a: ParamSet(a, prec, sess.device, weight_decay)
         self.wte, self.wpe = mk(lm["wte"]), mk(lm["wpe"])
         self.lnf_g, self.lnf_b = mk(lm["lnf_g"]), mk(lm["lnf_b"])

@@ -261,7 +261,7 @@ def test_block_error_paths(sess):
     assert e.value.status == fx.FAX_ERR_INVALID_ARG
 
 
-def lm_case(sess, cfg, prec, lm):
+def lm_case(sess, cfg, prec, lm, head_rows=0):
     ids, tg = synth.lm_tokens(cfg)
     B, T, H, hd = cfg.batch, cfg.seq, cfg.n_heads, cfg.head_dim
     rnd = (lambda a: synth.round_to_bf16(a).astype(np.float64)) if prec == 0 else (lambda a: a.astype(np.float64))
@@ -272,7 +272,7 @@ def lm_case(sess, cfg, prec, lm):
     zeros = {n: np.zeros_like(a, dtype=np.float64) for n, a in O.lm_tensors(lm)}
     rloss, rg, rw, rm, rv = O.lm_step(ids, tg, lmc, zeros, zeros, B, T, H, hd,
                                       dict(weight_decay=wd, step=1, **hp), cfg.ln_eps, lm_master=lm)
-    r = LmRunner(sess, cfg, lm, prec, weight_decay=wd)
+    r = LmRunner(sess, cfg, lm, prec, weight_decay=wd, head_rows=head_rows)
     tids = torch.as_tensor(ids).to(sess.device)
     ttg = torch.as_tensor(tg).to(sess.device)
     tol_f = TOL_FWD_BF16 if prec == 0 else TOL_FP32
@@ -283,7 +283,7 @@ def lm_case(sess, cfg, prec, lm):
     for name, ps in r.named_params():
         assert relerr(host(ps.g).reshape(rg[name].shape), rg[name]) <= tol_g, name
     # full step on fresh state, host loss readback
-    r2 = LmRunner(sess, cfg, lm, prec, weight_decay=wd)
+    r2 = LmRunner(sess, cfg, lm, prec, weight_decay=wd, head_rows=head_rows)
     l2 = r2.step(tids, ttg, hparams(step=1, **hp), want_host_loss=True)
     assert abs(l2 - rloss) <= tol_f * abs(rloss)
     for name, ps in r2.named_params():
@@ -293,7 +293,7 @@ def lm_case(sess, cfg, prec, lm):
         assert relerr(host(ps.w).reshape(w0.shape), cw) <= TOL_ADAMW, name
         check_adamw_update(name, host(ps.w).reshape(w0.shape), w0, rg[name], rw[name], hp["lr"], wd, tol_g, tol_g)
     # host-buffer entry point gives the same loss
-    r3 = LmRunner(sess, cfg, lm, prec, weight_decay=wd)
+    r3 = LmRunner(sess, cfg, lm, prec, weight_decay=wd, head_rows=head_rows)
     l3 = r3.step_host(torch.as_tensor(ids).pin_memory(), torch.as_tensor(tg).pin_memory(), hparams(step=1, **hp))
     assert l3 == l2
     st, _ = fx.fax_check_device_status(sess.ctx)
@@ -314,6 +314,15 @@ def test_lm_bf16_c4_shape_reduced(sess):
     # C4's widths and full vocabulary (d 768, 12 x 64, FFN 3072, V 50304), 2 layers, 2 x 128 tokens
     cfg = synth.scaled(synth.CONFIGS["C4"], batch=2, seq=128, n_layers=2)
     lm_case(sess, cfg, fx.FAX_PREC_BF16, synth.lm_params(cfg))
+
+
+@pytest.mark.parametrize("prec", [fx.FAX_PREC_FP32_VALIDATE, fx.FAX_PREC_BF16])
+def test_lm_head_in_row_chunks(sess, prec):
+    # 3 x 128 tokens with 256 logits rows at a time: a full chunk and a shorter last one, the
+    # gradient of the tied embedding accumulated over both (the path batches above ~42k tokens take)
+    cfg = synth.Config("lm_chunks", 11, batch=3, seq=128, d_model=256, n_heads=4, head_dim=64, d_ff=1024, n_layers=1,
+                       vocab=1024)
+    lm_case(sess, cfg, prec, synth.lm_params(cfg), head_rows=256)
 
 
 def test_lm_three_steps_and_resume_fp32(sess):
