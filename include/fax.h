@@ -206,6 +206,13 @@ fax_status fax_set_graph_replay(fax_ctx* ctx, int32_t enable);
  * one-CTA 128 x N kernel.  Same arithmetic either way.  Default: enabled. */
 fax_status fax_set_gemm_two_cta(fax_ctx* ctx, int32_t enable);
 
+/* Kernels are launched with programmatic dependent launch allowed: a kernel's
+ * blocks may become resident, and run their set-up, while the kernel before it
+ * on the stream is finishing; each kernel waits for that predecessor to
+ * complete before it touches global memory, so results are the same.
+ * enable = 0 launches every kernel fully serialised.  Default: enabled. */
+fax_status fax_set_dependent_launch(fax_ctx* ctx, int32_t enable);
+
 /* One trainable tensor of a training state: float32 master, compute-precision
  * copy (bf16; in FP32_VALIDATE may equal w or be NULL), Adam moments, float32
  * gradient, element count and its weight decay. */

@@ -95,6 +95,7 @@ _SIGNATURES = {
     "fax_launch_count": (C.c_uint64, [_P]),
     "fax_set_adamw_overlap": (C.c_int32, [_P, C.c_int32]),
     "fax_set_gemm_two_cta": (C.c_int32, [_P, C.c_int32]),
+    "fax_set_dependent_launch": (C.c_int32, [_P, C.c_int32]),
     "fax_set_graph_replay": (C.c_int32, [_P, C.c_int32]),
     "fax_set_fused_update": (C.c_int32, [_P, C.c_int32, C.c_int32]),
     "fax_profile_begin": (C.c_int32, [_P]),
@@ -202,6 +203,10 @@ def fax_set_graph_replay(ctx, enable: bool):
 
 def fax_set_gemm_two_cta(ctx, enable: bool):
     _check(load_library().fax_set_gemm_two_cta(ctx, int(bool(enable))), "fax_set_gemm_two_cta")
+
+
+def fax_set_dependent_launch(ctx, enable: bool):
+    _check(load_library().fax_set_dependent_launch(ctx, int(bool(enable))), "fax_set_dependent_launch")
 
 
 def fax_profile_begin(ctx):

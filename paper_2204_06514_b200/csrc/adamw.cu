@@ -39,6 +39,7 @@ __device__ __forceinline__ void adam_elem(float& w, float& m, float& v, float g,
 template <bool G_BF16>
 __global__ void __launch_bounds__(THREADS)
 adamw_kernel(const __grid_constant__ AdamBatch batch, AdamScalars sc) {
+  fax_grid_dependency_wait();
   for (unsigned int chunk = blockIdx.x; chunk < batch.total_chunks; chunk += gridDim.x) {
     // find the tensor this chunk belongs to (few tensors: linear scan from a binary start)
     int lo = 0, hi = batch.n_tensors - 1;
@@ -162,9 +163,9 @@ fax_status fax_adamw_launch(fax_ctx* ctx, const fax_adamw_tensor* tensors, int n
     const unsigned long long cap = (unsigned long long)ctx->sm_count * (ctx->stream == ctx->side ? 2 : 16);
     unsigned int grid = (unsigned int)(want < cap ? want : cap);
     if (hp->grad_is_bf16)
-      adamw_kernel<true><<<grid, THREADS, 0, ctx->stream>>>(batch, sc);
+      fax_launch(ctx, adamw_kernel<true>, dim3(grid), dim3(THREADS), 0, batch, sc);
     else
-      adamw_kernel<false><<<grid, THREADS, 0, ctx->stream>>>(batch, sc);
+      fax_launch(ctx, adamw_kernel<false>, dim3(grid), dim3(THREADS), 0, batch, sc);
     FAX_TRY(fax_after_launch(ctx));
   }
   return FAX_OK;

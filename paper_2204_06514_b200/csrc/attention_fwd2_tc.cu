@@ -81,6 +81,7 @@ attn_fwd2_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnFwd2Para
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  fax_grid_dependency_wait();    // set-up above may run under the previous kernel's tail; global memory only from here
   auto q_s = [&](int x) { return base + C_::Q_OFF + x * C_::TILE_BYTES; };
   auto k_s = [&](int i) { return base + C_::K_OFF + i * C_::TILE_BYTES; };
   auto v_s = [&](int i) { return base + C_::V_OFF + i * C_::TILE_BYTES; };
@@ -309,7 +310,7 @@ fax_status launch_fwd2(fax_ctx* ctx, int B, int T, int H, const void* qkv, void*
   }
   const long long items = (long long)B * H * (T / 256);
   const int grid = (int)(items < ctx->sm_count ? items : ctx->sm_count);
-  attn_fwd2_tc_kernel<HD><<<grid, F2_THREADS, Fwd2Cfg<HD>::SMEM_BYTES, ctx->stream>>>(map, p);
+  fax_launch(ctx, attn_fwd2_tc_kernel<HD>, dim3(grid), dim3(F2_THREADS), Fwd2Cfg<HD>::SMEM_BYTES, map, p);
   return fax_after_launch(ctx);
 }
 

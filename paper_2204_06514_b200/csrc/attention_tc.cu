@@ -91,6 +91,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnFwdParams
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  fax_grid_dependency_wait();    // set-up above may run under the previous kernel's tail; global memory only from here
   const uint32_t tmem_o = tmem + 256;
   const uint32_t q_s = base + C_::Q_OFF, p_s = base + C_::P_OFF;
   auto k_s = [&](int i) { return base + C_::K_OFF + i * C_::TILE_BYTES; };
@@ -278,7 +279,7 @@ fax_status launch_fwd(fax_ctx* ctx, int B, int T, int H, const void* qkv, void* 
     attr_set = true;
   }
   const int grid = B * H * (T / TQ);
-  attn_fwd_tc_kernel<HD><<<grid, FWD_THREADS, FwdCfg<HD>::SMEM_BYTES, ctx->stream>>>(map, p);
+  fax_launch(ctx, attn_fwd_tc_kernel<HD>, dim3(grid), dim3(FWD_THREADS), FwdCfg<HD>::SMEM_BYTES, map, p);
   return fax_after_launch(ctx);
 }
 
@@ -372,6 +373,7 @@ attn_bwd2_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_c
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  fax_grid_dependency_wait();    // set-up above may run under the previous kernel's tail; global memory only from here
   const uint32_t tm_st = tmem, tm_dp = tmem + 128, tm_dv = tmem + 256, tm_dk = tmem + 384;
   const uint32_t k_s = base + C_::K_OFF, v_s = base + C_::V_OFF, ds_s = base + C_::DS_OFF;
   auto q_s = [&](int i) { return base + C_::Q_OFF + i * C_::TILE_BYTES; };
@@ -671,6 +673,7 @@ attn_bwd2_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_c
 // D[b,h,t] = sum_c dO[t,c] * O[t,c] over the head's columns; one warp per (token, head)
 __global__ void attn_rowdot_bf16_kernel(int n_tok, int T, int H, int hd, const bf16* __restrict__ d_o,
                                         const bf16* __restrict__ o, float* __restrict__ Dv) {
+  fax_grid_dependency_wait();
   const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (gw >= n_tok * H) return;
   const int tok = gw / H, h = gw % H;
@@ -688,6 +691,7 @@ __global__ void attn_rowdot_bf16_kernel(int n_tok, int T, int H, int hd, const b
 // dqkv[n, 0:d] = bf16(dq_acc[n, :] * scale)
 __global__ void attn_dq_convert_kernel(long long n_tok, int d, const float* __restrict__ dq_acc, float scale,
                                        bf16* __restrict__ dqkv) {
+  fax_grid_dependency_wait();
   const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;     // one per 4 elements
   const long long total = n_tok * d / 4;
   if (idx >= total) return;
@@ -714,8 +718,8 @@ fax_status launch_bwd(fax_ctx* ctx, int B, int T, int H, const void* qkv, const 
     const long long warps = n_tok * H;
     const int threads = 256;
     const long long blocks = (warps * 32 + threads - 1) / threads;
-    attn_rowdot_bf16_kernel<<<(unsigned)blocks, threads, 0, ctx->stream>>>((int)n_tok, T, H, HD, (const bf16*)d_o,
-                                                                          (const bf16*)o, Dv);
+    fax_launch(ctx, attn_rowdot_bf16_kernel, dim3((unsigned)blocks), dim3(threads), 0, (int)n_tok, T, H, HD,
+               (const bf16*)d_o, (const bf16*)o, Dv);
     FAX_TRY(fax_after_launch(ctx));
   }
   AttnBwdParams p;
@@ -731,11 +735,11 @@ fax_status launch_bwd(fax_ctx* ctx, int B, int T, int H, const void* qkv, const 
   }
   const long long items = (long long)B * H * (T / 128);
   const int grid = (int)(items < ctx->sm_count ? items : ctx->sm_count);
-  attn_bwd2_tc_kernel<HD><<<grid, BWD_THREADS, Bwd2Cfg<HD>::SMEM_BYTES, ctx->stream>>>(mq, md, mdq, p);
+  fax_launch(ctx, attn_bwd2_tc_kernel<HD>, dim3(grid), dim3(BWD_THREADS), Bwd2Cfg<HD>::SMEM_BYTES, mq, md, mdq, p);
   FAX_TRY(fax_after_launch(ctx));
   const long long quads = n_tok * (long long)d / 4;
-  attn_dq_convert_kernel<<<(unsigned)((quads + 255) / 256), 256, 0, ctx->stream>>>(n_tok, (int)d, dq_acc, p.scale,
-                                                                                  (bf16*)dqkv);
+  fax_launch(ctx, attn_dq_convert_kernel, dim3((unsigned)((quads + 255) / 256)), dim3(256), 0, n_tok, (int)d, dq_acc,
+             p.scale, (bf16*)dqkv);
   return fax_after_launch(ctx);
 }
 

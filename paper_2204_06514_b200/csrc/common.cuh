@@ -58,6 +58,7 @@ struct fax_ctx {
   bool fused_update;         // whole-step calls fuse AdamW of the weight matrices into the dW GEMM epilogue
   bool keep_fused_grads;     // ... and still store those gradients
   bool use_2cta;             // GEMMs whose M and N are multiples of 256 use the two-CTA kernel
+  bool use_pdl;              // kernels are launched with programmatic stream serialization allowed
 };
 
 // Brackets the launches of one operator with CUDA events while profiling is on.
@@ -101,6 +102,25 @@ static inline fax_status fax_after_launch(fax_ctx* ctx) {
   return FAX_OK;
 }
 
+// Launch on the context's stream with programmatic dependent launch allowed: the grid may be
+// scheduled while its predecessor on the stream is still running, so its blocks become resident
+// as SMs free up and run their set-up (barrier initialisation, tensor-memory allocation,
+// descriptor prefetch) under the predecessor's tail.  ONLY for kernels whose every thread calls
+// fax_grid_dependency_wait() before its first access to global memory: that call returns once
+// the predecessor has completed and its writes are visible, which keeps the stream's ordering.
+template <typename... KArgs, typename... Args>
+static inline void fax_launch(fax_ctx* ctx, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                              Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = ctx->stream;
+  cudaLaunchAttribute attr = {};
+  attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr.val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = &attr;
+  cfg.numAttrs = ctx->use_pdl ? 1 : 0;
+  (void)cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);     // errors surface in fax_after_launch
+}
+
 static inline bool fax_aligned(const void* p, size_t a) { return ((uintptr_t)p & (a - 1)) == 0; }
 static inline size_t fax_round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 static inline size_t fax_elem_size(int prec) { return prec == FAX_PREC_BF16 ? 2 : 4; }
@@ -116,6 +136,14 @@ struct FaxArena {
   }
   size_t used() const { return fax_round_up(off, 256); }
 };
+
+// Counterpart of fax_launch in the kernel: blocks until the preceding grid on the stream has
+// completed (a no-op when the kernel was launched without the attribute), then lets the grid
+// that follows be scheduled behind this one.
+__device__ __forceinline__ void fax_grid_dependency_wait() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
 
 // ---- device numeric helpers -------------------------------------------------
 __device__ __forceinline__ float to_f32(float v) { return v; }

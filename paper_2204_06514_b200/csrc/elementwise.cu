@@ -6,6 +6,7 @@
 namespace {
 
 __global__ void __launch_bounds__(256) gelu_bf16_kernel(size_t n8, const uint4* __restrict__ h, uint4* __restrict__ g) {
+  fax_grid_dependency_wait();
   const size_t stride = (size_t)gridDim.x * blockDim.x;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += stride) {
     uint4 u = h[i], o;
@@ -21,6 +22,7 @@ __global__ void __launch_bounds__(256) gelu_bf16_kernel(size_t n8, const uint4* 
 }
 
 __global__ void __launch_bounds__(256) gelu_f32_kernel(size_t n, const float* __restrict__ h, float* __restrict__ g) {
+  fax_grid_dependency_wait();
   const size_t stride = (size_t)gridDim.x * blockDim.x;
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride) g[i] = gelu_tanh_f(h[i]);
 }
@@ -33,9 +35,9 @@ fax_status fax_gelu_fwd(fax_ctx* ctx, int prec, size_t n, const void* h, void* g
   const int blocks = 8 * ctx->sm_count;
   if (prec == FAX_PREC_BF16) {
     if (n % 8 || !fax_aligned(h, 16) || !fax_aligned(g, 16)) return FAX_ERR_UNSUPPORTED_SHAPE;
-    gelu_bf16_kernel<<<blocks, 256, 0, ctx->stream>>>(n / 8, (const uint4*)h, (uint4*)g);
+    fax_launch(ctx, gelu_bf16_kernel, dim3(blocks), dim3(256), 0, n / 8, (const uint4*)h, (uint4*)g);
   } else {
-    gelu_f32_kernel<<<blocks, 256, 0, ctx->stream>>>(n, (const float*)h, (float*)g);
+    fax_launch(ctx, gelu_f32_kernel, dim3(blocks), dim3(256), 0, n, (const float*)h, (float*)g);
   }
   return fax_after_launch(ctx);
 }

@@ -7,6 +7,7 @@ namespace {
 template <typename T>
 __global__ void embed_fwd_kernel(int n_tok, int Tn, int d, int vocab, const int32_t* __restrict__ ids,
                                  const T* __restrict__ wte, const T* __restrict__ wpe, T* __restrict__ x0) {
+  fax_grid_dependency_wait();
   int n = blockIdx.x;
   int id = ids[n];
   id = id < 0 ? 0 : (id >= vocab ? vocab - 1 : id);     // ids are validated upstream; clamp keeps reads in bounds
@@ -20,6 +21,7 @@ __global__ void embed_fwd_kernel(int n_tok, int Tn, int d, int vocab, const int3
 template <typename T>
 __global__ void embed_bwd_wte_kernel(int n_tok, int d, int vocab, const int32_t* __restrict__ ids,
                                      const T* __restrict__ dx0, float* __restrict__ dwte) {
+  fax_grid_dependency_wait();
   int n = blockIdx.x;
   int id = ids[n];
   if (id < 0 || id >= vocab) return;
@@ -31,6 +33,7 @@ __global__ void embed_bwd_wte_kernel(int n_tok, int d, int vocab, const int32_t*
 template <typename T>
 __global__ void embed_bwd_wpe_kernel(int Bn, int Tn, int max_seq, int d, const T* __restrict__ dx0,
                                      float* __restrict__ dwpe, int accumulate) {
+  fax_grid_dependency_wait();
   int t = blockIdx.x;
   for (int c = threadIdx.x; c < d; c += blockDim.x) {
     float s = 0.f;
@@ -65,6 +68,7 @@ template <typename T>
 __global__ void __launch_bounds__(512)
 xent_kernel(int rows, int vocab, T* __restrict__ logits, int64_t ld, const int32_t* __restrict__ targets,
             float inv_n, float* __restrict__ row_loss) {
+  fax_grid_dependency_wait();
   __shared__ float red[32];
   int r = blockIdx.x;
   T* row = logits + (size_t)r * ld;
@@ -95,6 +99,7 @@ xent_kernel(int rows, int vocab, T* __restrict__ logits, int64_t ld, const int32
 __global__ void __launch_bounds__(512)
 xent_smem_kernel(int rows, int vocab, bf16* __restrict__ logits, int64_t ld, const int32_t* __restrict__ targets,
                  float inv_n, float* __restrict__ row_loss) {
+  fax_grid_dependency_wait();
   extern __shared__ uint4 xrow[];               // vocab / 8 vectors of 8 bf16
   __shared__ float red[32];
   const int r = blockIdx.x;
@@ -148,6 +153,7 @@ xent_smem_kernel(int rows, int vocab, bf16* __restrict__ logits, int64_t ld, con
 }
 
 __global__ void loss_mean_kernel(int n, const float* __restrict__ row_loss, float* __restrict__ loss) {
+  fax_grid_dependency_wait();
   __shared__ double red[32];
   double s = 0.0;
   for (int i = threadIdx.x; i < n; i += blockDim.x) s += (double)row_loss[i];
@@ -169,9 +175,9 @@ fax_status fax_embed_fwd(fax_ctx* ctx, int prec, int B, int T, int d, int vocab,
   int n = B * T;
   FaxProfScope prof(ctx, KC_EMBED, 0.0, 3.0 * n * d * fax_elem_size(prec));
   if (prec == FAX_PREC_BF16)
-    embed_fwd_kernel<bf16><<<n, 128, 0, ctx->stream>>>(n, T, d, vocab, ids, (const bf16*)wte, (const bf16*)wpe, (bf16*)x0);
+    fax_launch(ctx, embed_fwd_kernel<bf16>, dim3(n), dim3(128), 0, n, T, d, vocab, ids, (const bf16*)wte, (const bf16*)wpe, (bf16*)x0);
   else
-    embed_fwd_kernel<float><<<n, 128, 0, ctx->stream>>>(n, T, d, vocab, ids, (const float*)wte, (const float*)wpe, (float*)x0);
+    fax_launch(ctx, embed_fwd_kernel<float>, dim3(n), dim3(128), 0, n, T, d, vocab, ids, (const float*)wte, (const float*)wpe, (float*)x0);
   return fax_after_launch(ctx);
 }
 
@@ -180,13 +186,13 @@ fax_status fax_embed_bwd(fax_ctx* ctx, int prec, int B, int T, int max_seq, int 
   int n = B * T;
   FaxProfScope prof(ctx, KC_EMBED, 0.0, (double)n * d * (2.0 * fax_elem_size(prec) + 8.0));
   if (prec == FAX_PREC_BF16) {
-    embed_bwd_wte_kernel<bf16><<<n, 128, 0, ctx->stream>>>(n, d, vocab, ids, (const bf16*)dx0, dwte);
+    fax_launch(ctx, embed_bwd_wte_kernel<bf16>, dim3(n), dim3(128), 0, n, d, vocab, ids, (const bf16*)dx0, dwte);
     FAX_TRY(fax_after_launch(ctx));
-    embed_bwd_wpe_kernel<bf16><<<max_seq, 128, 0, ctx->stream>>>(B, T, max_seq, d, (const bf16*)dx0, dwpe, accumulate_wpe ? 1 : 0);
+    fax_launch(ctx, embed_bwd_wpe_kernel<bf16>, dim3(max_seq), dim3(128), 0, B, T, max_seq, d, (const bf16*)dx0, dwpe, accumulate_wpe ? 1 : 0);
   } else {
-    embed_bwd_wte_kernel<float><<<n, 128, 0, ctx->stream>>>(n, d, vocab, ids, (const float*)dx0, dwte);
+    fax_launch(ctx, embed_bwd_wte_kernel<float>, dim3(n), dim3(128), 0, n, d, vocab, ids, (const float*)dx0, dwte);
     FAX_TRY(fax_after_launch(ctx));
-    embed_bwd_wpe_kernel<float><<<max_seq, 128, 0, ctx->stream>>>(B, T, max_seq, d, (const float*)dx0, dwpe, accumulate_wpe ? 1 : 0);
+    fax_launch(ctx, embed_bwd_wpe_kernel<float>, dim3(max_seq), dim3(128), 0, B, T, max_seq, d, (const float*)dx0, dwpe, accumulate_wpe ? 1 : 0);
   }
   return fax_after_launch(ctx);
 }
@@ -202,15 +208,15 @@ fax_status fax_xent(fax_ctx* ctx, int prec, int rows, int vocab, void* logits, i
       FAX_CUDA_TRY(ctx, cudaFuncSetAttribute(xent_smem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024));
       attr_set = true;
     }
-    xent_smem_kernel<<<rows, 512, row_bytes, ctx->stream>>>(rows, vocab, (bf16*)logits, ld, targets, inv_n, row_loss);
+    fax_launch(ctx, xent_smem_kernel, dim3(rows), dim3(512), row_bytes, rows, vocab, (bf16*)logits, ld, targets, inv_n, row_loss);
   } else if (prec == FAX_PREC_BF16)
-    xent_kernel<bf16><<<rows, 512, 0, ctx->stream>>>(rows, vocab, (bf16*)logits, ld, targets, inv_n, row_loss);
+    fax_launch(ctx, xent_kernel<bf16>, dim3(rows), dim3(512), 0, rows, vocab, (bf16*)logits, ld, targets, inv_n, row_loss);
   else
-    xent_kernel<float><<<rows, 512, 0, ctx->stream>>>(rows, vocab, (float*)logits, ld, targets, inv_n, row_loss);
+    fax_launch(ctx, xent_kernel<float>, dim3(rows), dim3(512), 0, rows, vocab, (float*)logits, ld, targets, inv_n, row_loss);
   return fax_after_launch(ctx);
 }
 
 fax_status fax_loss_mean(fax_ctx* ctx, int n, const float* row_loss, float* loss) {
-  loss_mean_kernel<<<1, 1024, 0, ctx->stream>>>(n, row_loss, loss);
+  fax_launch(ctx, loss_mean_kernel, dim3(1), dim3(1024), 0, n, row_loss, loss);
   return fax_after_launch(ctx);
 }

@@ -79,6 +79,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_base_slot;
+  fax_grid_dependency_wait();    // set-up above may run under the previous kernel's tail; global memory only from here
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
@@ -213,7 +214,7 @@ fax_status launch(fax_ctx* ctx, const FaxGemm& g) {
     FAX_CUDA_TRY(ctx, cudaMemset2DAsync(g.C, (size_t)g.ldc * 4, 0, (size_t)g.N * 4, (size_t)g.M, ctx->stream));
   const int items = tiles * p.splits;
   const int grid = items < ctx->sm_count ? items : ctx->sm_count;
-  gemm_tcgen05_kernel<BN><<<grid, NUM_THREADS, Cfg<BN>::SMEM_BYTES, ctx->stream>>>(ma, mb, p);
+  fax_launch(ctx, gemm_tcgen05_kernel<BN>, dim3(grid), dim3(NUM_THREADS), Cfg<BN>::SMEM_BYTES, ma, mb, p);
   return fax_after_launch(ctx);
 }
 

@@ -117,6 +117,7 @@ gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
   cluster_sync_all();            // both CTAs' barriers exist before either signals the other
   tc_fence_after();
   const uint32_t tmem_base = *tmem_base_slot;
+  fax_grid_dependency_wait();    // set-up above may run under the previous kernel's tail; global memory only from here
 
   if (warp == 0) {
     // ---------------- TMA producer (each CTA loads its own halves) ----------------
@@ -261,9 +262,9 @@ fax_status fax_gemm_tc2(fax_ctx* ctx, const FaxGemm& g) {
   const int items = tiles * p.splits;
   const int pairs = items < max_pairs ? items : max_pairs;
   switch (gemm_static_epi(g)) {
-#define FAX_LAUNCH(E) case E: gemm_tcgen05_2cta_kernel<E><<<2 * pairs, NUM_THREADS, SMEM_BYTES, ctx->stream>>>(ma, mb, p); break
+#define FAX_LAUNCH(E) case E: fax_launch(ctx, gemm_tcgen05_2cta_kernel<E>, dim3(2 * pairs), dim3(NUM_THREADS), SMEM_BYTES, ma, mb, p); break
     FAX_LAUNCH(0); FAX_LAUNCH(1); FAX_LAUNCH(2); FAX_LAUNCH(3); FAX_LAUNCH(4); FAX_LAUNCH(EPI_STATIC_F32);
-    default: gemm_tcgen05_2cta_kernel<-1><<<2 * pairs, NUM_THREADS, SMEM_BYTES, ctx->stream>>>(ma, mb, p); break;
+    default: fax_launch(ctx, gemm_tcgen05_2cta_kernel<-1>, dim3(2 * pairs), dim3(NUM_THREADS), SMEM_BYTES, ma, mb, p); break;
 #undef FAX_LAUNCH
   }
   return fax_after_launch(ctx);

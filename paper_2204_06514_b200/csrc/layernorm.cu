@@ -82,6 +82,7 @@ __global__ void __launch_bounds__(512, (VPT <= 2) ? 2 : 1)
 layernorm_fwd_group_kernel(int rows, int d, const T* __restrict__ x, const T* __restrict__ gamma,
                            const T* __restrict__ beta, float eps, T* __restrict__ out,
                            float* __restrict__ mu_out, float* __restrict__ rstd_out, T* __restrict__ x_copy) {
+  fax_grid_dependency_wait();
   constexpr int VN = Vec<T>::N;
   constexpr int NG = 16 / WG, TG = 32 * WG;
   __shared__ float red[2][16];
@@ -172,6 +173,7 @@ __global__ void __launch_bounds__(512)
 layernorm_fwd_kernel(int rows, int d, const T* __restrict__ x, const T* __restrict__ gamma,
                      const T* __restrict__ beta, float eps, T* __restrict__ out,
                      float* __restrict__ mu_out, float* __restrict__ rstd_out, T* __restrict__ x_copy) {
+  fax_grid_dependency_wait();
   constexpr int VN = Vec<T>::N;
   __shared__ float red[32];
   const int nvec = d / VN;
@@ -227,6 +229,7 @@ layernorm_bwd_fused_kernel(int rows, int d, const T* __restrict__ da, const T* _
                            const float* __restrict__ mu_in, const float* __restrict__ rstd_in,
                            const T* __restrict__ gamma, const T* __restrict__ add, T* __restrict__ dx,
                            float* __restrict__ partial) {
+  fax_grid_dependency_wait();
   constexpr int VN = Vec<T>::N;
   constexpr int NG = 16 / WG, TG = 32 * WG;
   extern __shared__ float fuse_sm[];                 // 2 * d floats
@@ -347,6 +350,7 @@ __global__ void __launch_bounds__(512)
 layernorm_bwd_dx_kernel(int rows, int d, const T* __restrict__ da, const T* __restrict__ x,
                         const float* __restrict__ mu_in, const float* __restrict__ rstd_in,
                         const T* __restrict__ gamma, const T* __restrict__ add, T* __restrict__ dx) {
+  fax_grid_dependency_wait();
   constexpr int VN = Vec<T>::N;
   __shared__ float2 red[32];
   const int nvec = d / VN;
@@ -399,6 +403,7 @@ template <typename T, bool LN>
 __global__ void __launch_bounds__(256)
 colreduce_kernel(int rows, int cols, const T* __restrict__ in, int64_t ld, const T* __restrict__ x,
                  const float* __restrict__ mu, const float* __restrict__ rstd, float* __restrict__ partial) {
+  fax_grid_dependency_wait();
   constexpr int VN = Vec<T>::N;
   __shared__ float sm[LN ? 2 : 1][8][32 * VN + 1];
   const int lane = threadIdx.x & 31, ph = threadIdx.x >> 5;
@@ -452,6 +457,7 @@ colreduce_kernel(int rows, int cols, const T* __restrict__ in, int64_t ld, const
 __global__ void __launch_bounds__(256)
 colreduce_fold_kernel(int slabs, int width, int cols, const float* __restrict__ partial,
                       float* __restrict__ out0, float* __restrict__ out1, int accumulate) {
+  fax_grid_dependency_wait();
   __shared__ float sm[8][33];
   const int lane = threadIdx.x & 31, ph = threadIdx.x >> 5;
   const int c = blockIdx.x * 32 + lane;
@@ -522,8 +528,8 @@ fax_status ln_fwd_t(fax_ctx* ctx, int rows, int d, const void* x, const void* ga
     const int cap = (wide_lane ? 1 : 2) * ctx->sm_count;
     if (grid > cap) grid = cap;
 #define LN_FWDG(V, W)                                                                                   \
-    layernorm_fwd_group_kernel<T, V, W><<<grid, 512, 0, ctx->stream>>>(                                 \
-        rows, d, (const T*)x, (const T*)gamma, (const T*)beta, eps, (T*)out, mu, rstd, (T*)x_copy)
+    fax_launch(ctx, layernorm_fwd_group_kernel<T, V, W>, dim3(grid), dim3(512), 0,                      \
+               rows, d, (const T*)x, (const T*)gamma, (const T*)beta, eps, (T*)out, mu, rstd, (T*)x_copy)
     if (nvec <= 32) LN_FWDG(1, 1);
     else if (nvec <= 64) LN_FWDG(2, 1);
     else if (nvec <= 96) LN_FWDG(3, 1);
@@ -538,8 +544,8 @@ fax_status ln_fwd_t(fax_ctx* ctx, int rows, int d, const void* x, const void* ga
   if (!vpt) return FAX_ERR_UNSUPPORTED_SHAPE;
 #define LN_FWD(V)                                                                                    \
   case V:                                                                                            \
-    layernorm_fwd_kernel<T, V><<<rows, threads, 0, ctx->stream>>>(                                   \
-        rows, d, (const T*)x, (const T*)gamma, (const T*)beta, eps, (T*)out, mu, rstd, (T*)x_copy);   \
+    fax_launch(ctx, layernorm_fwd_kernel<T, V>, dim3(rows), dim3(threads), 0,                        \
+               rows, d, (const T*)x, (const T*)gamma, (const T*)beta, eps, (T*)out, mu, rstd, (T*)x_copy); \
     break;
   switch (vpt) { LN_FWD(1) LN_FWD(2) LN_FWD(3) LN_FWD(4) LN_FWD(6) LN_FWD(8) LN_FWD(12) LN_FWD(16) }
 #undef LN_FWD
@@ -555,8 +561,8 @@ fax_status ln_bwd_dx_t(fax_ctx* ctx, int rows, int d, const void* da, const void
   if (!vpt || vpt > 8) return FAX_ERR_UNSUPPORTED_SHAPE;
 #define LN_BWD(V)                                                                                   \
   case V:                                                                                           \
-    layernorm_bwd_dx_kernel<T, V><<<rows, threads, 0, ctx->stream>>>(                               \
-        rows, d, (const T*)da, (const T*)x, mu, rstd, (const T*)gamma, (const T*)add, (T*)dx);      \
+    fax_launch(ctx, layernorm_bwd_dx_kernel<T, V>, dim3(rows), dim3(threads), 0,                    \
+               rows, d, (const T*)da, (const T*)x, mu, rstd, (const T*)gamma, (const T*)add, (T*)dx); \
     break;
   switch (vpt) { LN_BWD(1) LN_BWD(2) LN_BWD(3) LN_BWD(4) LN_BWD(6) LN_BWD(8) }
 #undef LN_BWD
@@ -571,8 +577,8 @@ fax_status ln_bwd_fused_t(fax_ctx* ctx, int rows, int d, const void* da, const v
   const int grid = ln_bwd_fused_grid(ctx, rows, nvec);
   const size_t smem = (size_t)2 * d * sizeof(float);
 #define LN_FUSED(V, W)                                                                                 \
-  layernorm_bwd_fused_kernel<T, V, W><<<grid, 512, smem, ctx->stream>>>(                               \
-      rows, d, (const T*)da, (const T*)x, mu, rstd, (const T*)gamma, (const T*)add, (T*)dx, partial)
+  fax_launch(ctx, layernorm_bwd_fused_kernel<T, V, W>, dim3(grid), dim3(512), smem,                    \
+             rows, d, (const T*)da, (const T*)x, mu, rstd, (const T*)gamma, (const T*)add, (T*)dx, partial)
   if (nvec <= 32) LN_FUSED(1, 1);
   else if (nvec <= 64) LN_FUSED(2, 1);
   else if (nvec <= 128) LN_FUSED(2, 2);
@@ -580,8 +586,8 @@ fax_status ln_bwd_fused_t(fax_ctx* ctx, int rows, int d, const void* da, const v
   else LN_FUSED(2, 8);
 #undef LN_FUSED
   FAX_TRY(fax_after_launch(ctx));
-  colreduce_fold_kernel<<<(2 * d + 31) / 32, 256, 0, ctx->stream>>>(grid, 2 * d, d, partial, dgamma, dbeta,
-                                                                   accumulate ? 1 : 0);
+  fax_launch(ctx, colreduce_fold_kernel, dim3((2 * d + 31) / 32), dim3(256), 0, grid, 2 * d, d, (const float*)partial,
+             dgamma, dbeta, accumulate ? 1 : 0);
   return fax_after_launch(ctx);
 }
 
@@ -592,11 +598,11 @@ fax_status colreduce_t(fax_ctx* ctx, int rows, int cols, const void* in, int64_t
   const int nvec = cols / Vec<T>::N;
   const int slabs = colreduce_slabs(ctx, rows, nvec, LN ? kLnColBlocksPerSm : kColsumBlocksPerSm);
   dim3 grid((nvec + 31) / 32, slabs);
-  colreduce_kernel<T, LN><<<grid, 256, 0, ctx->stream>>>(rows, cols, (const T*)in, ld, (const T*)x, mu, rstd, partial);
+  fax_launch(ctx, colreduce_kernel<T, LN>, grid, dim3(256), 0, rows, cols, (const T*)in, ld, (const T*)x, mu, rstd, partial);
   FAX_TRY(fax_after_launch(ctx));
   const int width = LN ? 2 * cols : cols;
-  colreduce_fold_kernel<<<(width + 31) / 32, 256, 0, ctx->stream>>>(slabs, width, cols, partial, out0, out1,
-                                                                    accumulate ? 1 : 0);
+  fax_launch(ctx, colreduce_fold_kernel, dim3((width + 31) / 32), dim3(256), 0, slabs, width, cols, (const float*)partial,
+             out0, out1, accumulate ? 1 : 0);
   return fax_after_launch(ctx);
 }
 
