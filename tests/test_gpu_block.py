@@ -156,6 +156,40 @@ def test_block_step_host_matches_device_step(sess):
                 assert relerr(host(yh), host(a.y)) <= TOL_FWD_BF16
 
 
+def test_dependent_launch_switch_leaves_results_unchanged(sess):
+    """Kernels launched with programmatic dependent launch wait for their predecessor before they
+    touch global memory, so a step gives the same forward bits and the same gradients (to the
+    rounding of the arrival-order adds) as with every launch fully serialised; repeated steps go
+    through the captured graph as well."""
+    cfg = synth.CONFIGS["C2"]
+    params = synth.block_params(cfg)
+    x, dy = synth.block_inputs(cfg)
+    hp = dict(synth.ADAMW)
+    wd = hp.pop("weight_decay")
+    runs = {}
+    try:
+        for on in (True, False):
+            fx.fax_set_dependent_launch(sess.ctx, on)
+            r = BlockRunner(sess, cfg, params, fx.FAX_PREC_BF16, weight_decay=wd)
+            tx, tdy = r.to_device(x), r.to_device(dy)
+            ys = []
+            for step in (1, 2, 3, 4):
+                r.step(tx, tdy, hparams(step=step, **hp))
+                torch.cuda.synchronize()
+                ys.append(r.y.clone())
+            runs[on] = (ys, r.dx.clone(), {k: r.p[k].g.clone() for k in O.PARAM_NAMES})
+    finally:
+        fx.fax_set_dependent_launch(sess.ctx, True)
+    assert torch.equal(runs[True][0][0], runs[False][0][0])          # first forward: identical weights
+    for a, b in zip(runs[True][0][1:], runs[False][0][1:]):
+        assert relerr(host(a), host(b)) <= TOL_FWD_BF16
+    assert relerr(host(runs[True][1]), host(runs[False][1])) <= TOL_GRAD_BF16
+    for k in O.PARAM_NAMES:
+        assert relerr(host(runs[True][2][k]), host(runs[False][2][k])) <= TOL_GRAD_BF16, k
+    st, _ = fx.fax_check_device_status(sess.ctx)
+    assert st == fx.FAX_OK
+
+
 def test_graph_replay_patches_the_adamw_scalars(sess):
     """From the third call on a whole step is a replayed CUDA graph; the only arguments that change
     are AdamW's scalars.  A step with lr = 0 must leave every weight exactly as it was."""
