@@ -317,7 +317,12 @@ template <int HD> struct Bwd2Cfg {
   static constexpr int DS_OFF = DO_OFF + NDO * TILE_BYTES;  // dS tile (32 KB); the dQ staging boxes start here too
   static constexpr int STG_BYTES = 128 * HD * 4;            // dQ tile in float32
   static constexpr int DS_BYTES = (STG_BYTES > 32768) ? STG_BYTES : 32768;
-  static constexpr int STAT_OFF = DS_OFF + DS_BYTES;        // [2][2][128] floats: log2e*LSE and D of the query tile
+  // head_dim 64 leaves room for dQ staging buffers of their own, two of them: the write of dS and the
+  // staging of a dQ tile then never wait for the bulk reduction of the step before (only for the one
+  // two steps back).  At head_dim 128 the staging boxes share the dS tile's bytes.
+  static constexpr int NSTG = (HD == 64) ? 2 : 1;
+  static constexpr int STG_OFF = (HD == 64) ? DS_OFF + DS_BYTES : DS_OFF;
+  static constexpr int STAT_OFF = (HD == 64) ? STG_OFF + NSTG * STG_BYTES : DS_OFF + DS_BYTES;   // [2][2][128] floats: log2e*LSE and D of the query tile
   static constexpr int BAR_OFF = STAT_OFF + 2048;
   static constexpr int LAYOUT_BYTES = BAR_OFF + 256;
   // 768 bytes of slack for aligning the tiles to 1024 bytes (at hd 128 this is exactly the 227 KB a CTA
@@ -575,12 +580,11 @@ attn_bwd2_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_c
             }
         }
         tc_st32(tm_st + lane_base + 64 * hc + 32, dd);
-        if (gs > 0) {
+        if (HD == 128 && gs > 0) {
           // the dS buffer staged the first 32 KB of the previous dQ tile: the bulk reductions of those
-          // boxes (the older of the two groups at hd 128, the only group at hd 64) must have read it
+          // boxes (the older of the step's two groups) must have read it
           if (tid == 0) {
-            if (HD == 128) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-            else bulk_wait_read_all();
+            asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
             mbar_arrive(bar(C_::STGFREE));
           }
           if (!mbar_wait_warp(bar(C_::STGFREE), (gs - 1) & 1u, abort_flag, p.status, 333)) { ok = false; break; }
@@ -602,6 +606,16 @@ attn_bwd2_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_c
           if (tid == 0) { bulk_wait_read_all(); mbar_arrive(bar(C_::STGFREE2)); }
           if (hc == 1 && !mbar_wait_warp(bar(C_::STGFREE2), (gs - 1) & 1u, abort_flag, p.status, 337)) { ok = false; break; }
         }
+        if (HD == 64 && gs > 1) {
+          // staging buffer gs & 1 was last the source of the reduction issued two steps ago (one bulk
+          // group per step): all but the newest group must have read their boxes
+          if (tid == 0) {
+            asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+            mbar_arrive(bar(C_::STGFREE));
+          }
+          if (!mbar_wait_warp(bar(C_::STGFREE), gs & 1u, abort_flag, p.status, 333)) { ok = false; break; }
+        }
+        const uint32_t stg_off = (uint32_t)C_::STG_OFF + (HD == 64 ? (gs & 1u) * (uint32_t)C_::STG_BYTES : 0u);
         {
           constexpr int NB = HD / 64;          // this warp's half of the head's columns: two boxes or one
           const int c0 = hc * (HD / 2);
@@ -611,7 +625,7 @@ attn_bwd2_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_c
           tc_wait_ld();
 #pragma unroll
           for (int cc = 0; cc < NB; ++cc) {
-            uint8_t* box = gbase + C_::DS_OFF + ((c0 >> 5) + cc) * 16384 + kr * 128;
+            uint8_t* box = gbase + stg_off + ((c0 >> 5) + cc) * 16384 + kr * 128;
 #pragma unroll
             for (int k = 0; k < 8; ++k)
               *reinterpret_cast<uint4*>(box + ((k ^ (kr & 7)) << 4)) =
@@ -625,7 +639,7 @@ attn_bwd2_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_c
         if (tid == 0 && mbar_wait(bar(C_::STGFULL), ph, abort_flag, p.status, 336)) {
 #pragma unroll
           for (int i = 0; i < HD / 32; ++i) {
-            tma_reduce_add_2d(&tmap_dq, base + C_::DS_OFF + i * 16384, h * HD + 32 * i, (int)(row0 + qi * 128));
+            tma_reduce_add_2d(&tmap_dq, base + stg_off + i * 16384, h * HD + 32 * i, (int)(row0 + qi * 128));
             if (HD == 128 && i == 1) bulk_commit_group();     // boxes 0, 1 (the dS tile's bytes) as a group of their own
           }
           bulk_commit_group();
