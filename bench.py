@@ -27,6 +27,7 @@ if ROOT not in sys.path:
 METRIC = "training tokens/sec, fwd+bwd+AdamW, 1 GPU (MFU reported beside it)"
 UNIT = "tokens/s"
 NOMINAL_BF16_TFLOPS = 2250.0        # B200 dense bf16, datasheet
+GEMM_DRAM_BYTES_PER_LAUNCH = {"C3": 960.9e6}     # mean over the step's 12 GEMM launches (algorithmic: 459e6)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -363,9 +364,13 @@ def run_ours(args):
         kernels[name] = ent
     top = max(kernels, key=lambda k: kernels[k]["ms_per_step"])
     tk = kernels[top]
+    # DRAM bytes (read + written) per launch of the dominant kernel, from one ncu capture of this very
+    # command line (profiles/gemm_dram_traffic_block_step_C3.md); None where no capture of the current
+    # kernels exists for the workload
+    traffic = GEMM_DRAM_BYTES_PER_LAUNCH.get(cfg.name) if top == "gemm_tcgen05" and not args.recompute else None
     roofline = {"kernel": top, "bound": tk["bound"], "achieved": tk["achieved"],
                 "peak": peaks["bf16_tflops_sustained"] if tk["bound"] == "tensor" else peaks["hbm_gbs"],
-                "unit": tk["unit"], "frac": tk["frac"], "traffic": None,
+                "unit": tk["unit"], "frac": tk["frac"], "traffic": traffic,
                 "peak_source": f"{peaks_kind} ({'sustained bf16 GEMM' if tk['bound'] == 'tensor' else 'copy'})",
                 "per_launch": {"avg_ms": tk["avg_launch_ms"],
                                "algorithmic": (prof[top]["flops"] or prof[top]["bytes"]) / prof[top]["launches"]}}
