@@ -217,63 +217,97 @@ layernorm_fwd_kernel(int rows, int d, const T* __restrict__ x, const T* __restri
   }
 }
 
+// ---- asynchronous copies into shared memory (each thread later reads only what it copied) ----
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;"
+               ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
+constexpr int LN_RING = 3;        // rows in flight per row group: the current one and two ahead
+
 // Backward, fused: dx and the per-block column sums for dgamma / dbeta in one pass over da and x.
 // A block of 512 threads holds 16 / WG row groups of WG warps; a group walks rows
 // (group index + k * groups in the grid), every thread owning the same VPT vector columns in all
-// of them, so the column sums accumulate in registers.  The next row's vectors are requested
-// before the current row is reduced.  At the end the groups of a block add their sums in shared
-// memory and the block writes one slab: partial[block][0][c] = sum da*xhat, partial[block][1][c] = sum da.
+// of them, so the column sums accumulate in registers.  Rows are staged through shared memory: a
+// group keeps LN_RING rows of da, x (and the residual gradient) in flight as asynchronous 16-byte
+// copies, each thread copying exactly the vectors it will read, so no barrier guards the ring and
+// the memory latency of two rows hides under the current one.  At the end the groups of a block add
+// their sums in shared memory and the block writes one slab: partial[block][0][c] = sum da*xhat,
+// partial[block][1][c] = sum da.
+// Dynamic shared memory: 2 * d floats for the final reduction, then the ring
+// [row group][slot][da | x | add][32 * WG * VPT vectors].
 template <typename T, int VPT, int WG>
 __global__ void __launch_bounds__(512, 1)
-layernorm_bwd_fused_kernel(int rows, int d, const T* __restrict__ da, const T* __restrict__ x,
-                           const float* __restrict__ mu_in, const float* __restrict__ rstd_in,
-                           const T* __restrict__ gamma, const T* __restrict__ add, T* __restrict__ dx,
-                           float* __restrict__ partial) {
+layernorm_bwd_ring_kernel(int rows, int d, const T* __restrict__ da, const T* __restrict__ x,
+                          const float* __restrict__ mu_in, const float* __restrict__ rstd_in,
+                          const T* __restrict__ gamma, const T* __restrict__ add, T* __restrict__ dx,
+                          float* __restrict__ partial) {
   fax_grid_dependency_wait();
   constexpr int VN = Vec<T>::N;
-  constexpr int NG = 16 / WG, TG = 32 * WG;
-  extern __shared__ float fuse_sm[];                 // 2 * d floats
+  constexpr int NG = 16 / WG, TG = 32 * WG, PER = TG * VPT;
+  extern __shared__ uint4 ring_sm_raw[];
+  float* fuse_sm = reinterpret_cast<float*>(ring_sm_raw);              // 2 * d floats
   __shared__ float2 red[2][16];
   const int grp = threadIdx.x / TG, t = threadIdx.x % TG;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nvec = d / VN;
   const int stride = NG * gridDim.x;
   const float inv_d = 1.f / (float)d;
+  uint4* ring = ring_sm_raw + (2 * d * 4 + 15) / 16 + (size_t)grp * LN_RING * 3 * PER;
   float ag[VPT][VN], ab[VPT][VN];
-  uint4 gm[VPT], nda[VPT], nx[VPT], nad[VPT];
+  uint4 gm[VPT];
 #pragma unroll
   for (int i = 0; i < VPT; ++i) {
 #pragma unroll
     for (int j = 0; j < VN; ++j) { ag[i][j] = 0.f; ab[i][j] = 0.f; }
     const int vi = t + TG * i;
     gm[i] = (vi < nvec) ? reinterpret_cast<const uint4*>(gamma)[vi] : make_uint4(0, 0, 0, 0);
-    nda[i] = nx[i] = nad[i] = make_uint4(0, 0, 0, 0);
   }
-  int row = NG * blockIdx.x + grp;
-  float nmu = 0.f, nrs = 0.f;
-#define LN_FETCH(r)                                                                      \
-  {                                                                                      \
-    const uint4* dar = reinterpret_cast<const uint4*>(da + (size_t)(r) * d);             \
-    const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)(r) * d);               \
-    const uint4* adr = reinterpret_cast<const uint4*>(add + (size_t)(r) * d);            \
-    _Pragma("unroll") for (int i = 0; i < VPT; ++i) {                                    \
-      const int vi = t + TG * i;                                                         \
-      if (vi < nvec) { nda[i] = dar[vi]; nx[i] = xr[vi]; if (add) nad[i] = adr[vi]; }    \
-    }                                                                                    \
-    nmu = mu_in[r]; nrs = rstd_in[r];                                                    \
-  }
-  if (row < rows) LN_FETCH(row)
-  for (int it = 0; row < rows; row += stride, ++it) {
-    uint4 cda[VPT], cx[VPT], cad[VPT];
+  auto issue = [&](int r, int slot) {
+    if (r < rows) {
+      uint4* s0 = ring + (size_t)slot * 3 * PER;
+      const uint4* dar = reinterpret_cast<const uint4*>(da + (size_t)r * d);
+      const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)r * d);
+      const uint4* adr = reinterpret_cast<const uint4*>(add + (size_t)r * d);
 #pragma unroll
-    for (int i = 0; i < VPT; ++i) { cda[i] = nda[i]; cx[i] = nx[i]; cad[i] = nad[i]; }
-    const float mu = nmu, rstd = nrs;
-    const int nr = row + stride;
-    if (nr < rows) LN_FETCH(nr)
+      for (int i = 0; i < VPT; ++i) {
+        const int vi = t + TG * i;
+        if (vi < nvec) {
+          cp_async16(s0 + vi, dar + vi);
+          cp_async16(s0 + PER + vi, xr + vi);
+          if (add) cp_async16(s0 + 2 * PER + vi, adr + vi);
+        }
+      }
+    }
+    cp_async_commit();          // one group per call, empty past the last row, so the counting stays uniform
+  };
+  int row = NG * blockIdx.x + grp;
+  issue(row, 0);
+  issue(row + stride, 1);
+  float mu0 = 0.f, rs0 = 0.f, mu1 = 0.f, rs1 = 0.f;
+  if (row < rows) { mu0 = mu_in[row]; rs0 = rstd_in[row]; }
+  if (row + stride < rows) { mu1 = mu_in[row + stride]; rs1 = rstd_in[row + stride]; }
+  int slot = 0;
+  for (int it = 0; row < rows; row += stride, ++it) {
+    const int ahead = row + 2 * stride;
+    issue(ahead, slot >= 1 ? slot - 1 : LN_RING - 1);        // the slot read in the iteration before this one
+    float mu2 = 0.f, rs2 = 0.f;
+    if (ahead < rows) { mu2 = mu_in[ahead]; rs2 = rstd_in[ahead]; }
+    cp_async_wait<2>();                                       // all but the two newest groups: this row has landed
+    const float mu = mu0, rstd = rs0;
+    mu0 = mu1; rs0 = rs1; mu1 = mu2; rs1 = rs2;
+    const uint4* s0 = ring + (size_t)slot * 3 * PER;
+    uint4 cda[VPT], cx[VPT];
     float s1 = 0.f, s2 = 0.f;
 #pragma unroll
     for (int i = 0; i < VPT; ++i) {
-      if (t + TG * i < nvec) {
+      const int vi = t + TG * i;
+      if (vi < nvec) {
+        cda[i] = s0[vi]; cx[i] = s0[PER + vi];
         float fd[VN], fx[VN], g[VN];
         unpack<T>(cda[i], fd); unpack<T>(cx[i], fx); unpack<T>(gm[i], g);
 #pragma unroll
@@ -282,8 +316,6 @@ layernorm_bwd_fused_kernel(int rows, int d, const T* __restrict__ da, const T* _
     }
     s1 = warp_sum(s1); s2 = warp_sum(s2);
     if (WG > 1) {
-      // the WG warps of this row meet at a barrier of their own; red is double-buffered by
-      // iteration parity, so one barrier per row is enough
       if (lane == 0) red[it & 1][warp] = make_float2(s1, s2);
       asm volatile("bar.sync %0, %1;" ::"r"(1 + grp), "r"(TG) : "memory");
       s1 = 0.f; s2 = 0.f;
@@ -306,15 +338,17 @@ layernorm_bwd_fused_kernel(int rows, int d, const T* __restrict__ da, const T* _
         }
         if (add) {
           float av[VN];
-          unpack<T>(cad[i], av);
+          unpack<T>(s0[2 * PER + vi], av);
 #pragma unroll
           for (int j = 0; j < VN; ++j) o[j] += av[j];
         }
         store_vec<T>(dx + (size_t)row * d + vi * VN, o);
       }
     }
+    slot = (slot + 1 == LN_RING) ? 0 : slot + 1;
   }
-#undef LN_FETCH
+  cp_async_wait<0>();
+  __syncthreads();
   // the groups add their column sums one after the other (fixed order: deterministic)
   for (int g = 0; g < NG; ++g) {
     if (grp == g) {
@@ -575,15 +609,28 @@ fax_status ln_bwd_fused_t(fax_ctx* ctx, int rows, int d, const void* da, const v
                           float* dbeta, bool accumulate, float* partial) {
   const int nvec = d / Vec<T>::N;
   const int grid = ln_bwd_fused_grid(ctx, rows, nvec);
-  const size_t smem = (size_t)2 * d * sizeof(float);
+  // dynamic shared memory: 2 * d floats for the final reduction (rounded up to whole 16-byte vectors),
+  // then the ring: 16 / W groups x LN_RING slots x 3 arrays x 32 * W * V vectors of 16 bytes; the
+  // opt-in limit covers the widest row an instantiation serves (512 vectors)
+  auto ring_bytes = [](int V, int W) { return (size_t)(16 / W) * LN_RING * 3 * (32 * W * V) * 16; };
 #define LN_FUSED(V, W)                                                                                 \
-  fax_launch(ctx, layernorm_bwd_fused_kernel<T, V, W>, dim3(grid), dim3(512), smem,                    \
-             rows, d, (const T*)da, (const T*)x, mu, rstd, (const T*)gamma, (const T*)add, (T*)dx, partial)
-  if (nvec <= 32) LN_FUSED(1, 1);
-  else if (nvec <= 64) LN_FUSED(2, 1);
-  else if (nvec <= 128) LN_FUSED(2, 2);
-  else if (nvec <= 256) LN_FUSED(2, 4);
-  else LN_FUSED(2, 8);
+  {                                                                                                    \
+    const size_t smem = ((size_t)2 * d * sizeof(float) + 15) / 16 * 16 + ring_bytes(V, W);             \
+    static bool attr_set = false;                                                                      \
+    if (!attr_set) {                                                                                   \
+      FAX_CUDA_TRY(ctx, cudaFuncSetAttribute(layernorm_bwd_ring_kernel<T, V, W>,                       \
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize,              \
+                                             (int)((size_t)2 * 512 * Vec<T>::N * sizeof(float) + ring_bytes(V, W)))); \
+      attr_set = true;                                                                                 \
+    }                                                                                                  \
+    fax_launch(ctx, layernorm_bwd_ring_kernel<T, V, W>, dim3(grid), dim3(512), smem,                   \
+               rows, d, (const T*)da, (const T*)x, mu, rstd, (const T*)gamma, (const T*)add, (T*)dx, partial); \
+  }
+  if (nvec <= 32) LN_FUSED(1, 1)
+  else if (nvec <= 64) LN_FUSED(2, 1)
+  else if (nvec <= 128) LN_FUSED(2, 2)
+  else if (nvec <= 256) LN_FUSED(2, 4)
+  else LN_FUSED(2, 8)
 #undef LN_FUSED
   FAX_TRY(fax_after_launch(ctx));
   fax_launch(ctx, colreduce_fold_kernel, dim3((2 * d + 31) / 32), dim3(256), 0, grid, 2 * d, d, (const float*)partial,
