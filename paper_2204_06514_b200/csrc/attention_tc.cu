@@ -684,22 +684,38 @@ attn_bwd2_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_c
   if (warp == 8) { tc_fence_after(); tmem_dealloc(tmem, C_::TMEM_COLS); }
 }
 
-// D[b,h,t] = sum_c dO[t,c] * O[t,c] over the head's columns; one warp per (token, head)
-__global__ void attn_rowdot_bf16_kernel(int n_tok, int T, int H, int hd, const bf16* __restrict__ d_o,
-                                        const bf16* __restrict__ o, float* __restrict__ Dv) {
+// D[b,h,t] = sum_c dO[t,c] * O[t,c] over the head's columns.  A thread takes 8 columns (one 16-byte
+// vector of each operand), hd / 8 neighbouring lanes share a (token, head) and add up with shuffles.
+// The same thread also clears its 8 elements of the float32 dQ accumulator [n_tok, H * hd], which
+// the backward kernel's bulk reductions add into (no separate memset).
+__global__ void __launch_bounds__(256)
+attn_rowdot_bf16_kernel(int n_tok, int T, int H, int hd, const bf16* __restrict__ d_o,
+                        const bf16* __restrict__ o, float* __restrict__ Dv, float* __restrict__ dq_acc) {
   fax_grid_dependency_wait();
-  const int gw = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-  if (gw >= n_tok * H) return;
-  const int tok = gw / H, h = gw % H;
-  const long long off = (long long)tok * H * hd + h * hd;
+  const int lanes = hd >> 3;                                   // 8 (hd 64) or 16 (hd 128): divides the warp
+  const long long vec = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const long long total = (long long)n_tok * H * lanes;
+  const bool in = vec < total;
   float s = 0.f;
-  for (int c = lane * 2; c < hd; c += 64) {
-    float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(d_o + off + c));
-    float2 bq = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(o + off + c));
-    s += a.x * bq.x + a.y * bq.y;
+  if (in) {
+    const uint4 a = reinterpret_cast<const uint4*>(d_o)[vec];  // rows are dense: vector index = element / 8
+    const uint4 b = reinterpret_cast<const uint4*>(o)[vec];
+    reinterpret_cast<float4*>(dq_acc)[2 * vec] = make_float4(0.f, 0.f, 0.f, 0.f);
+    reinterpret_cast<float4*>(dq_acc)[2 * vec + 1] = make_float4(0.f, 0.f, 0.f, 0.f);
+    const __nv_bfloat162* ha = reinterpret_cast<const __nv_bfloat162*>(&a);
+    const __nv_bfloat162* hb = reinterpret_cast<const __nv_bfloat162*>(&b);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const float2 fa = __bfloat1622float2(ha[e]), fb = __bfloat1622float2(hb[e]);
+      s += fa.x * fb.x + fa.y * fb.y;
+    }
   }
-  s = warp_sum(s);
-  if (lane == 0) Dv[((long long)(tok / T) * H + h) * T + (tok % T)] = s;
+  for (int off = lanes >> 1; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+  if (in && (vec % lanes) == 0) {
+    const long long th = vec / lanes;                          // token * H + head
+    const int tok = (int)(th / H), h = (int)(th % H);
+    Dv[((long long)(tok / T) * H + h) * T + (tok % T)] = s;
+  }
 }
 
 // dqkv[n, 0:d] = bf16(dq_acc[n, :] * scale)
@@ -727,13 +743,12 @@ fax_status launch_bwd(fax_ctx* ctx, int B, int T, int H, const void* qkv, const 
   if (!make_map(ctx, &mq, qkv, 3 * d, (uint64_t)n_tok, 3 * d, 64, 128)) return FAX_ERR_INVALID_ARG;
   if (!make_map(ctx, &md, d_o, d, (uint64_t)n_tok, d, 64, 128)) return FAX_ERR_INVALID_ARG;
   if (!make_map_f32(ctx, &mdq, dq_acc, d, (uint64_t)n_tok, d, 32, 128)) return FAX_ERR_INVALID_ARG;
-  FAX_CUDA_TRY(ctx, cudaMemsetAsync(dq_acc, 0, (size_t)n_tok * d * sizeof(float), ctx->stream));
   {
-    const long long warps = n_tok * H;
+    const long long vecs = n_tok * H * (HD / 8);
     const int threads = 256;
-    const long long blocks = (warps * 32 + threads - 1) / threads;
+    const long long blocks = (vecs + threads - 1) / threads;
     fax_launch(ctx, attn_rowdot_bf16_kernel, dim3((unsigned)blocks), dim3(threads), 0, (int)n_tok, T, H, HD,
-               (const bf16*)d_o, (const bf16*)o, Dv);
+               (const bf16*)d_o, (const bf16*)o, Dv, dq_acc);
     FAX_TRY(fax_after_launch(ctx));
   }
   AttnBwdParams p;
