@@ -1,6 +1,6 @@
 // Embedding lookup / scatter and softmax cross-entropy of the LM step
 // (steps LM-E, LM-H loss part, LM-B).  All HBM-bound.
-#include "common.cuh"
+#include "tc_common.cuh"
 
 namespace {
 
@@ -93,62 +93,139 @@ xent_kernel(int rows, int vocab, T* __restrict__ logits, int64_t ld, const int32
   }
 }
 
-// bf16 rows that fit in shared memory: the row is read from HBM once.  Pass 1 copies it to
-// shared memory and takes the maximum; pass 2 replaces each logit by exp(logit - max)
-// (bf16) while summing the unrounded exponentials; pass 3 writes (e / sum - onehot) * inv_n.
-__global__ void __launch_bounds__(512)
-xent_smem_kernel(int rows, int vocab, bf16* __restrict__ logits, int64_t ld, const int32_t* __restrict__ targets,
-                 float inv_n, float* __restrict__ row_loss) {
-  fax_grid_dependency_wait();
-  extern __shared__ uint4 xrow[];               // vocab / 8 vectors of 8 bf16
+// bf16 rows of which two fit in shared memory: a row is read from HBM once.  Pass 1 takes the
+// maximum; pass 2 replaces each logit by exp(logit - max) (bf16) while summing the unrounded
+// exponentials; pass 3 writes (e / sum - onehot) * inv_n.  A persistent kernel (one block per SM)
+// that keeps HBM busy while it computes: an extra warp moves rows with bulk
+// asynchronous copies, global -> shared into one of two row buffers ahead of the compute warps and
+// shared -> global behind them, so the load of row i+1 and the store of row i-1 run under the
+// passes over row i.  Hand-offs are mbarriers (full[b]: the row has landed; done[b]: all 16
+// compute warps have finished it); every wait is bounded.
+constexpr int XS_COMPUTE_THREADS = 512;
+constexpr int XS_THREADS = XS_COMPUTE_THREADS + 32;
+
+__device__ __forceinline__ void bulk_load_row(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void bulk_store_row(void* dst, uint32_t src, uint32_t bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes) : "memory");
+}
+
+__global__ void __launch_bounds__(XS_THREADS, 1)
+xent_stream_kernel(int rows, int vocab, bf16* __restrict__ logits, int64_t ld, const int32_t* __restrict__ targets,
+                   float inv_n, float* __restrict__ row_loss, int32_t* status) {
+  using namespace tc;
+  extern __shared__ uint4 xs_raw[];                  // [2][vocab / 8] vectors, then barriers
   __shared__ float red[32];
-  const int r = blockIdx.x;
-  uint4* grow = reinterpret_cast<uint4*>(logits + (size_t)r * ld);
+  __shared__ uint64_t bars_mem[4];
+  __shared__ int abort_mem;
+  const uint32_t row_bytes = (uint32_t)vocab * 2u;
   const int nvec = vocab >> 3;
-  float mx = -INFINITY;
-  for (int i = threadIdx.x; i < nvec; i += blockDim.x) {
-    const uint4 u = grow[i];
-    xrow[i] = u;
-    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
-#pragma unroll
-    for (int e = 0; e < 4; ++e) { float2 f = __bfloat1622float2(h[e]); mx = fmaxf(mx, fmaxf(f.x, f.y)); }
-  }
-  mx = block_reduce_max(mx, red);
-  const int tg = targets[r];
-  float s = 0.f;
-  for (int i = threadIdx.x; i < nvec; i += blockDim.x) {
-    uint4 u = xrow[i];
-    __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&u);
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      float2 f = __bfloat1622float2(h[e]);
-      const float e0 = __expf(f.x - mx), e1 = __expf(f.y - mx);
-      s += e0 + e1;
-      h[e] = __floats2bfloat162_rn(e0, e1);
-    }
-    xrow[i] = u;
-  }
-  float lt = 0.f;
-  if (threadIdx.x == 0 && tg >= 0 && tg < vocab) lt = __bfloat162float(logits[(size_t)r * ld + tg]);   // still the logit: global row not yet rewritten
-  s = block_reduce_sum(s, red);
+  const uint32_t bars = smem_u32(bars_mem);
+  auto full_bar = [&](int b) { return bars + 8u * b; };
+  auto done_bar = [&](int b) { return bars + 8u * (2 + b); };
+  volatile int* abort_flag = &abort_mem;
   if (threadIdx.x == 0) {
-    const float lse = mx + logf(s);
-    row_loss[r] = (tg >= 0 && tg < vocab) ? lse - lt : 0.f;
+    mbar_init(full_bar(0), 1); mbar_init(full_bar(1), 1);
+    mbar_init(done_bar(0), XS_COMPUTE_THREADS / 32); mbar_init(done_bar(1), XS_COMPUTE_THREADS / 32);
+    abort_mem = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  const float k = inv_n / s;
-  for (int i = threadIdx.x; i < nvec; i += blockDim.x) {
-    uint4 u = xrow[i];
-    __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&u);
-    const int c0 = i << 3;
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      float2 f = __bfloat1622float2(h[e]);
-      float p0 = f.x * k, p1 = f.y * k;
-      if (c0 + 2 * e == tg) p0 -= inv_n;
-      if (c0 + 2 * e + 1 == tg) p1 -= inv_n;
-      h[e] = __floats2bfloat162_rn(p0, p1);
+  __syncthreads();
+  fax_grid_dependency_wait();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_mine = (rows - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;      // rows blockIdx.x + k * gridDim.x
+
+  if (warp == XS_COMPUTE_THREADS / 32) {
+    // ---------------- copy warp ----------------
+    if (lane == 0) {
+      bool ok = true;
+      for (int k = 0; k < n_mine && k < 2; ++k) {
+        mbar_expect_tx(full_bar(k), row_bytes);
+        bulk_load_row(smem_u32(xs_raw) + (uint32_t)k * row_bytes, logits + (size_t)(blockIdx.x + k * gridDim.x) * ld,
+                      row_bytes, full_bar(k));
+      }
+      for (int k = 0; k < n_mine && ok; ++k) {
+        const int b = k & 1;
+        if (!mbar_wait(done_bar(b), (uint32_t)(k >> 1) & 1u, abort_flag, status, 401)) { ok = false; break; }
+        const size_t r = (size_t)blockIdx.x + (size_t)k * gridDim.x;
+        bulk_store_row(logits + r * ld, smem_u32(xs_raw) + (uint32_t)b * row_bytes, row_bytes);
+        bulk_commit_group();
+        if (k + 2 < n_mine) {
+          bulk_wait_read_all();                     // the store has read the buffer: it may be refilled
+          mbar_expect_tx(full_bar(b), row_bytes);
+          bulk_load_row(smem_u32(xs_raw) + (uint32_t)b * row_bytes, logits + (r + 2 * (size_t)gridDim.x) * ld, row_bytes,
+                        full_bar(b));
+        }
+      }
+      bulk_wait_all();                              // all stores have landed before the block exits
     }
-    grow[i] = u;
+  } else {
+    // ---------------- compute warps ----------------
+    bool ok = true;
+    for (int k = 0; k < n_mine && ok; ++k) {
+      const int b = k & 1;
+      const int r = (int)blockIdx.x + k * (int)gridDim.x;
+      uint4* xrow = xs_raw + (size_t)b * nvec;
+      if (!mbar_wait_warp(full_bar(b), (uint32_t)(k >> 1) & 1u, abort_flag, status, 402)) { ok = false; break; }
+      const int tg = targets[r];
+      float mx = -INFINITY;
+      for (int i = threadIdx.x; i < nvec; i += XS_COMPUTE_THREADS) {
+        const uint4 u = xrow[i];
+        const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) { float2 f = __bfloat1622float2(h[e]); mx = fmaxf(mx, fmaxf(f.x, f.y)); }
+      }
+      float lt = 0.f;
+      if (threadIdx.x == 0 && tg >= 0 && tg < vocab) lt = __bfloat162float(reinterpret_cast<const bf16*>(xrow)[tg]);
+      // block-wide reductions among the compute warps only (named barrier 1)
+      auto reduce = [&](float v, bool is_max) {
+        v = is_max ? warp_max(v) : warp_sum(v);
+        named_barrier_sync(1, XS_COMPUTE_THREADS);
+        if (lane == 0) red[warp] = v;
+        named_barrier_sync(1, XS_COMPUTE_THREADS);
+        float t = lane < XS_COMPUTE_THREADS / 32 ? red[lane] : (is_max ? -INFINITY : 0.f);
+        return is_max ? warp_max(t) : warp_sum(t);
+      };
+      mx = reduce(mx, true);
+      float s = 0.f;
+      for (int i = threadIdx.x; i < nvec; i += XS_COMPUTE_THREADS) {
+        uint4 u = xrow[i];
+        __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&u);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          float2 f = __bfloat1622float2(h[e]);
+          const float e0 = __expf(f.x - mx), e1 = __expf(f.y - mx);
+          s += e0 + e1;
+          h[e] = __floats2bfloat162_rn(e0, e1);
+        }
+        xrow[i] = u;
+      }
+      s = reduce(s, false);
+      if (threadIdx.x == 0) {
+        const float lse = mx + logf(s);
+        row_loss[r] = (tg >= 0 && tg < vocab) ? lse - lt : 0.f;
+      }
+      const float kk = inv_n / s;
+      for (int i = threadIdx.x; i < nvec; i += XS_COMPUTE_THREADS) {
+        uint4 u = xrow[i];
+        __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&u);
+        const int c0 = i << 3;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          float2 f = __bfloat1622float2(h[e]);
+          float p0 = f.x * kk, p1 = f.y * kk;
+          if (c0 + 2 * e == tg) p0 -= inv_n;
+          if (c0 + 2 * e + 1 == tg) p1 -= inv_n;
+          h[e] = __floats2bfloat162_rn(p0, p1);
+        }
+        xrow[i] = u;
+      }
+      fence_proxy_async();                          // this thread's shared-memory writes, for the bulk store
+      __syncwarp();
+      if (lane == 0) mbar_arrive(done_bar(b));
+    }
   }
 }
 
@@ -202,13 +279,17 @@ fax_status fax_xent(fax_ctx* ctx, int prec, int rows, int vocab, void* logits, i
   // read the logits once, write dlogits once
   FaxProfScope prof(ctx, KC_XENT, 0.0, 2.0 * rows * (double)vocab * fax_elem_size(prec));
   const size_t row_bytes = (size_t)vocab * 2;
-  if (prec == FAX_PREC_BF16 && vocab % 8 == 0 && ld % 8 == 0 && row_bytes <= 110 * 1024 && fax_aligned(logits, 16)) {
+  const bool vec_ok = prec == FAX_PREC_BF16 && vocab % 8 == 0 && ld % 8 == 0 && fax_aligned(logits, 16);
+  if (vec_ok && 2 * row_bytes <= 220 * 1024) {
+    // two rows fit: persistent kernel, rows streamed through shared memory by bulk copies
     static bool attr_set = false;
     if (!attr_set) {
-      FAX_CUDA_TRY(ctx, cudaFuncSetAttribute(xent_smem_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024));
+      FAX_CUDA_TRY(ctx, cudaFuncSetAttribute(xent_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
       attr_set = true;
     }
-    fax_launch(ctx, xent_smem_kernel, dim3(rows), dim3(512), row_bytes, rows, vocab, (bf16*)logits, ld, targets, inv_n, row_loss);
+    const int grid = rows < ctx->sm_count ? rows : ctx->sm_count;
+    fax_launch(ctx, xent_stream_kernel, dim3(grid), dim3(XS_THREADS), 2 * row_bytes, rows, vocab, (bf16*)logits,
+               ld, targets, inv_n, row_loss, ctx->dev_status);
   } else if (prec == FAX_PREC_BF16)
     fax_launch(ctx, xent_kernel<bf16>, dim3(rows), dim3(512), 0, rows, vocab, (bf16*)logits, ld, targets, inv_n, row_loss);
   else
