@@ -185,6 +185,9 @@ fax_status fax_block_backward_impl(fax_ctx* ctx, const fax_block_cfg* c, const f
     return matrix_done ? fax_adamw_async(ctx, hook->t + first + 1, 1, hook->hp)      // only the bias is left
                        : fax_adamw_async(ctx, hook->t + first, 2, hook->hp);
   };
+  // The gradients of the two biases beside LayerNorm 2 - db_fc2 = column sums of dY (the residual
+  // gradient that B3 adds) and db_o = column sums of dx1 (what B3 writes) - are taken inside the
+  // LayerNorm backward kernel of B3, so b_fc2 is updated there, together with the LayerNorm's own tensors.
   bool fz = false;
   // B1: through FC2 and GELU
   if (rc) {
@@ -197,8 +200,7 @@ fax_status fax_block_backward_impl(fax_ctx* ctx, const fax_block_cfg* c, const f
     FAX_TRY(linear_bwd_weight(ctx, prec, N, f, d, s.g, dy, gr->w_fc2, acc, try_fuse ? hook->t + 10 : nullptr,
                               try_fuse ? hook->hp : nullptr, &fz));
   }
-  FAX_TRY(fax_colsum(ctx, prec, N, d, dy, d, gr->b_fc2, acc, w.partial, w.partial_floats));
-  FAX_TRY(update(10, fz));
+  if (hook && !fz) FAX_TRY(fax_adamw_async(ctx, hook->t + 10, 1, hook->hp));                    // w_fc2; b_fc2 after B3
   // B2: through FC1
   FAX_TRY(linear_bwd_data(ctx, prec, N, d, f, w.bufF, p->w_fc1, EPI_NONE, nullptr, w.bufA));    // dm
   const void* m_in = s.m;
@@ -212,13 +214,15 @@ fax_status fax_block_backward_impl(fax_ctx* ctx, const fax_block_cfg* c, const f
   FAX_TRY(update(8, fz));
   // B3: LN2 backward plus the residual branch
   FAX_TRY(fax_layernorm_bwd(ctx, prec, N, d, w.bufA, s.x1, s.mu2, s.rstd2, p->ln2_g, dy, w.bufB,
-                            gr->ln2_g, gr->ln2_b, acc, w.partial, w.partial_floats));           // dx1
-  FAX_TRY(update(6));
+                            gr->ln2_g, gr->ln2_b, acc, w.partial, w.partial_floats, gr->b_fc2, gr->b_o));   // dx1
+  if (hook) {
+    const fax_adamw_tensor t3[3] = {hook->t[6], hook->t[7], hook->t[11]};                       // ln2_g, ln2_b, b_fc2
+    FAX_TRY(fax_adamw_async(ctx, t3, 3, hook->hp));
+  }
   // B4: through the attention output projection
   FAX_TRY(linear_bwd_data(ctx, prec, N, d, d, w.bufB, p->w_o, EPI_NONE, nullptr, w.bufA));      // do
   FAX_TRY(linear_bwd_weight(ctx, prec, N, d, d, s.o, w.bufB, gr->w_o, acc, try_fuse ? hook->t + 4 : nullptr,
                             try_fuse ? hook->hp : nullptr, &fz));
-  FAX_TRY(fax_colsum(ctx, prec, N, d, w.bufB, d, gr->b_o, acc, w.partial, w.partial_floats));
   FAX_TRY(update(4, fz));
   // B5: attention backward
   FAX_TRY(fax_attention_bwd(ctx, prec, c->batch, c->seq, c->n_heads, c->head_dim, s.qkv, s.o, s.lse,

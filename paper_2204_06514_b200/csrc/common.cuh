@@ -225,11 +225,13 @@ bool fax_gemm_patch_info_2cta(const void* func, const void* param, size_t* size,
 
 fax_status fax_layernorm_fwd(fax_ctx* ctx, int prec, int rows, int d, const void* x, const void* gamma,
                              const void* beta, float eps, void* out, float* mu, float* rstd, void* x_copy);
-// dx = (add ? add : 0) + LNbwd(da); partial: float scratch [2 * slabs * d]
+// dx = (add ? add : 0) + LNbwd(da); partial: float scratch [2 * slabs * d] ([4 * slabs * d] with the sums).
+// sum_add, sum_out (both or neither; need add): also sum_add[c] (+)= sum_r add[r, c] and
+// sum_out[c] (+)= sum_r dx[r, c], taken inside the LayerNorm kernel where the row width allows.
 fax_status fax_layernorm_bwd(fax_ctx* ctx, int prec, int rows, int d, const void* da, const void* x,
                              const float* mu, const float* rstd, const void* gamma, const void* add,
                              void* dx, float* dgamma, float* dbeta, bool accumulate, float* partial,
-                             size_t partial_floats);
+                             size_t partial_floats, float* sum_add = nullptr, float* sum_out = nullptr);
 size_t fax_layernorm_bwd_partial_floats(int rows, int d);
 
 // out[c] (+)= sum_r in[r, c]

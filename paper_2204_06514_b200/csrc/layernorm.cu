@@ -238,9 +238,12 @@ constexpr int LN_RING = 3;        // rows in flight per row group: the current o
 // the memory latency of two rows hides under the current one.  At the end the groups of a block add
 // their sums in shared memory and the block writes one slab: partial[block][0][c] = sum da*xhat,
 // partial[block][1][c] = sum da.
-// Dynamic shared memory: 2 * d floats for the final reduction, then the ring
+// Dynamic shared memory: 2 (with SUMS: 4) * d floats for the final reduction, then the ring
 // [row group][slot][da | x | add][32 * WG * VPT vectors].
-template <typename T, int VPT, int WG>
+// SUMS: also the column sums of `add` and of the output dx (the bias gradients of the linear layers on
+// either side of the LayerNorm: partial[block][2][c] = sum add, partial[block][3][c] = sum dx), which
+// costs two more accumulators per column and no memory traffic.
+template <typename T, int VPT, int WG, bool SUMS>
 __global__ void __launch_bounds__(512, 1)
 layernorm_bwd_ring_kernel(int rows, int d, const T* __restrict__ da, const T* __restrict__ x,
                           const float* __restrict__ mu_in, const float* __restrict__ rstd_in,
@@ -250,20 +253,21 @@ layernorm_bwd_ring_kernel(int rows, int d, const T* __restrict__ da, const T* __
   constexpr int VN = Vec<T>::N;
   constexpr int NG = 16 / WG, TG = 32 * WG, PER = TG * VPT;
   extern __shared__ uint4 ring_sm_raw[];
-  float* fuse_sm = reinterpret_cast<float*>(ring_sm_raw);              // 2 * d floats
+  constexpr int NS = SUMS ? 4 : 2;                                     // column sums per column
+  float* fuse_sm = reinterpret_cast<float*>(ring_sm_raw);              // NS * d floats
   __shared__ float2 red[2][16];
   const int grp = threadIdx.x / TG, t = threadIdx.x % TG;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nvec = d / VN;
   const int stride = NG * gridDim.x;
   const float inv_d = 1.f / (float)d;
-  uint4* ring = ring_sm_raw + (2 * d * 4 + 15) / 16 + (size_t)grp * LN_RING * 3 * PER;
-  float ag[VPT][VN], ab[VPT][VN];
+  uint4* ring = ring_sm_raw + (NS * d * 4 + 15) / 16 + (size_t)grp * LN_RING * 3 * PER;
+  float ag[VPT][VN], ab[VPT][VN], aa[SUMS ? VPT : 1][VN], ao[SUMS ? VPT : 1][VN];
   uint4 gm[VPT];
 #pragma unroll
   for (int i = 0; i < VPT; ++i) {
 #pragma unroll
-    for (int j = 0; j < VN; ++j) { ag[i][j] = 0.f; ab[i][j] = 0.f; }
+    for (int j = 0; j < VN; ++j) { ag[i][j] = 0.f; ab[i][j] = 0.f; if (SUMS) { aa[i][j] = 0.f; ao[i][j] = 0.f; } }
     const int vi = t + TG * i;
     gm[i] = (vi < nvec) ? reinterpret_cast<const uint4*>(gamma)[vi] : make_uint4(0, 0, 0, 0);
   }
@@ -340,7 +344,11 @@ layernorm_bwd_ring_kernel(int rows, int d, const T* __restrict__ da, const T* __
           float av[VN];
           unpack<T>(s0[2 * PER + vi], av);
 #pragma unroll
-          for (int j = 0; j < VN; ++j) o[j] += av[j];
+          for (int j = 0; j < VN; ++j) { o[j] += av[j]; if (SUMS) aa[i][j] += av[j]; }
+        }
+        if (SUMS) {
+#pragma unroll
+          for (int j = 0; j < VN; ++j) ao[i][j] += o[j];
         }
         store_vec<T>(dx + (size_t)row * d + vi * VN, o);
       }
@@ -350,32 +358,34 @@ layernorm_bwd_ring_kernel(int rows, int d, const T* __restrict__ da, const T* __
   cp_async_wait<0>();
   __syncthreads();
   // the groups add their column sums one after the other (fixed order: deterministic)
+  auto fold4 = [&](float* base, const float (&v)[VN], int vi, bool first) {
+#pragma unroll
+    for (int j = 0; j < VN; j += 4) {
+      float4* pp = reinterpret_cast<float4*>(base + vi * VN + j);
+      float4 w = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+      if (!first) { const float4 o4 = *pp; w.x += o4.x; w.y += o4.y; w.z += o4.z; w.w += o4.w; }
+      *pp = w;
+    }
+  };
   for (int g = 0; g < NG; ++g) {
     if (grp == g) {
 #pragma unroll
       for (int i = 0; i < VPT; ++i) {
         const int vi = t + TG * i;
         if (vi < nvec) {
-#pragma unroll
-          for (int j = 0; j < VN; j += 4) {
-            float4* pg = reinterpret_cast<float4*>(fuse_sm + vi * VN + j);
-            float4* pb = reinterpret_cast<float4*>(fuse_sm + d + vi * VN + j);
-            float4 vg = make_float4(ag[i][j], ag[i][j + 1], ag[i][j + 2], ag[i][j + 3]);
-            float4 vb = make_float4(ab[i][j], ab[i][j + 1], ab[i][j + 2], ab[i][j + 3]);
-            if (g > 0) {
-              const float4 og = *pg, ob = *pb;
-              vg.x += og.x; vg.y += og.y; vg.z += og.z; vg.w += og.w;
-              vb.x += ob.x; vb.y += ob.y; vb.z += ob.z; vb.w += ob.w;
-            }
-            *pg = vg; *pb = vb;
+          fold4(fuse_sm, ag[i], vi, g == 0);
+          fold4(fuse_sm + d, ab[i], vi, g == 0);
+          if (SUMS) {
+            fold4(fuse_sm + 2 * d, aa[i], vi, g == 0);
+            fold4(fuse_sm + 3 * d, ao[i], vi, g == 0);
           }
         }
       }
     }
     __syncthreads();
   }
-  float4* dst = reinterpret_cast<float4*>(partial + (size_t)blockIdx.x * 2 * d);
-  for (int c = threadIdx.x; c < 2 * d / 4; c += blockDim.x) dst[c] = reinterpret_cast<const float4*>(fuse_sm)[c];
+  float4* dst = reinterpret_cast<float4*>(partial + (size_t)blockIdx.x * NS * d);
+  for (int c = threadIdx.x; c < NS * d / 4; c += blockDim.x) dst[c] = reinterpret_cast<const float4*>(fuse_sm)[c];
 }
 
 // Backward dx, one block per row (wide rows).
@@ -486,11 +496,12 @@ colreduce_kernel(int rows, int cols, const T* __restrict__ in, int64_t ld, const
   }
 }
 
-// out[c] (+)= sum_s partial[s][c] for c < width (width = cols, or 2*cols with out split in two).
+// out[c] (+)= sum_s partial[s][c] for c < width (width = cols, 2*cols or 4*cols with out split accordingly).
 // Block = 32 columns x 8 slab phases, summed in a fixed order.
 __global__ void __launch_bounds__(256)
 colreduce_fold_kernel(int slabs, int width, int cols, const float* __restrict__ partial,
-                      float* __restrict__ out0, float* __restrict__ out1, int accumulate) {
+                      float* __restrict__ out0, float* __restrict__ out1, float* __restrict__ out2,
+                      float* __restrict__ out3, int accumulate) {
   fax_grid_dependency_wait();
   __shared__ float sm[8][33];
   const int lane = threadIdx.x & 31, ph = threadIdx.x >> 5;
@@ -506,7 +517,8 @@ colreduce_fold_kernel(int slabs, int width, int cols, const float* __restrict__ 
     s = 0.f;
 #pragma unroll
     for (int k = 0; k < 8; ++k) s += sm[k][lane];
-    float* dst = (c < cols) ? (out0 + c) : (out1 + (c - cols));
+    const int q = c / cols;                      // which of the (up to four) sums of width `cols`
+    float* dst = (q == 0 ? out0 : q == 1 ? out1 : q == 2 ? out2 : out3) + (c - q * cols);
     *dst = accumulate ? (*dst + s) : s;
   }
 }
@@ -606,35 +618,39 @@ fax_status ln_bwd_dx_t(fax_ctx* ctx, int rows, int d, const void* da, const void
 template <typename T>
 fax_status ln_bwd_fused_t(fax_ctx* ctx, int rows, int d, const void* da, const void* x, const float* mu,
                           const float* rstd, const void* gamma, const void* add, void* dx, float* dgamma,
-                          float* dbeta, bool accumulate, float* partial) {
+                          float* dbeta, bool accumulate, float* partial, float* sum_add, float* sum_out) {
   const int nvec = d / Vec<T>::N;
   const int grid = ln_bwd_fused_grid(ctx, rows, nvec);
+  const bool sums = sum_add && sum_out && add;
+  const int ns = sums ? 4 : 2;
   // dynamic shared memory: 2 * d floats for the final reduction (rounded up to whole 16-byte vectors),
   // then the ring: 16 / W groups x LN_RING slots x 3 arrays x 32 * W * V vectors of 16 bytes; the
   // opt-in limit covers the widest row an instantiation serves (512 vectors)
   auto ring_bytes = [](int V, int W) { return (size_t)(16 / W) * LN_RING * 3 * (32 * W * V) * 16; };
-#define LN_FUSED(V, W)                                                                                 \
+#define LN_FUSED_S(V, W, S)                                                                            \
   {                                                                                                    \
-    const size_t smem = ((size_t)2 * d * sizeof(float) + 15) / 16 * 16 + ring_bytes(V, W);             \
+    const size_t smem = ((size_t)ns * d * sizeof(float) + 15) / 16 * 16 + ring_bytes(V, W);            \
     static bool attr_set = false;                                                                      \
     if (!attr_set) {                                                                                   \
-      FAX_CUDA_TRY(ctx, cudaFuncSetAttribute(layernorm_bwd_ring_kernel<T, V, W>,                       \
+      FAX_CUDA_TRY(ctx, cudaFuncSetAttribute(layernorm_bwd_ring_kernel<T, V, W, S>,                    \
                                              cudaFuncAttributeMaxDynamicSharedMemorySize,              \
-                                             (int)((size_t)2 * 512 * Vec<T>::N * sizeof(float) + ring_bytes(V, W)))); \
+                                             (int)((size_t)(S ? 4 : 2) * 512 * Vec<T>::N * sizeof(float) + ring_bytes(V, W)))); \
       attr_set = true;                                                                                 \
     }                                                                                                  \
-    fax_launch(ctx, layernorm_bwd_ring_kernel<T, V, W>, dim3(grid), dim3(512), smem,                   \
+    fax_launch(ctx, layernorm_bwd_ring_kernel<T, V, W, S>, dim3(grid), dim3(512), smem,                \
                rows, d, (const T*)da, (const T*)x, mu, rstd, (const T*)gamma, (const T*)add, (T*)dx, partial); \
   }
+#define LN_FUSED(V, W) { if (sums) LN_FUSED_S(V, W, true) else LN_FUSED_S(V, W, false) }
   if (nvec <= 32) LN_FUSED(1, 1)
   else if (nvec <= 64) LN_FUSED(2, 1)
   else if (nvec <= 128) LN_FUSED(2, 2)
   else if (nvec <= 256) LN_FUSED(2, 4)
   else LN_FUSED(2, 8)
 #undef LN_FUSED
+#undef LN_FUSED_S
   FAX_TRY(fax_after_launch(ctx));
-  fax_launch(ctx, colreduce_fold_kernel, dim3((2 * d + 31) / 32), dim3(256), 0, grid, 2 * d, d, (const float*)partial,
-             dgamma, dbeta, accumulate ? 1 : 0);
+  fax_launch(ctx, colreduce_fold_kernel, dim3((ns * d + 31) / 32), dim3(256), 0, grid, ns * d, d, (const float*)partial,
+             dgamma, dbeta, sum_add, sum_out, accumulate ? 1 : 0);
   return fax_after_launch(ctx);
 }
 
@@ -649,7 +665,7 @@ fax_status colreduce_t(fax_ctx* ctx, int rows, int cols, const void* in, int64_t
   FAX_TRY(fax_after_launch(ctx));
   const int width = LN ? 2 * cols : cols;
   fax_launch(ctx, colreduce_fold_kernel, dim3((width + 31) / 32), dim3(256), 0, slabs, width, cols, (const float*)partial,
-             out0, out1, accumulate ? 1 : 0);
+             out0, out1, (float*)nullptr, (float*)nullptr, accumulate ? 1 : 0);
   return fax_after_launch(ctx);
 }
 
@@ -657,7 +673,7 @@ fax_status colreduce_t(fax_ctx* ctx, int rows, int cols, const void* in, int64_t
 
 size_t fax_layernorm_bwd_partial_floats(int rows, int d) {
   (void)rows;
-  return (size_t)2 * 256 * d;     // 256 = upper bound of the slab count
+  return (size_t)4 * 256 * d;     // 256 = upper bound of the slab count; four sums per column with the bias gradients
 }
 
 fax_status fax_layernorm_fwd(fax_ctx* ctx, int prec, int rows, int d, const void* x, const void* gamma,
@@ -675,15 +691,26 @@ fax_status fax_layernorm_fwd(fax_ctx* ctx, int prec, int rows, int d, const void
 fax_status fax_layernorm_bwd(fax_ctx* ctx, int prec, int rows, int d, const void* da, const void* x,
                              const float* mu, const float* rstd, const void* gamma, const void* add,
                              void* dx, float* dgamma, float* dbeta, bool accumulate, float* partial,
-                             size_t partial_floats) {
+                             size_t partial_floats, float* sum_add, float* sum_out) {
   if (d % (prec == FAX_PREC_BF16 ? 8 : 4)) return FAX_ERR_UNSUPPORTED_SHAPE;
-  if (partial_floats < (size_t)2 * ln_bwd_slabs(ctx, rows, d, prec) * d) return FAX_ERR_WORKSPACE_TOO_SMALL;
+  const bool sums = sum_add && sum_out && add;
+  const bool fused = ln_bwd_is_fused(d / (prec == FAX_PREC_BF16 ? 8 : 4));
+  if (partial_floats < (size_t)(sums && fused ? 4 : 2) * ln_bwd_slabs(ctx, rows, d, prec) * d) return FAX_ERR_WORKSPACE_TOO_SMALL;
+  if (sums && !fused) {
+    // wide rows: the column sums of add and dx as reductions of their own, after the LayerNorm kernels
+    FAX_TRY(fax_layernorm_bwd(ctx, prec, rows, d, da, x, mu, rstd, gamma, add, dx, dgamma, dbeta, accumulate, partial,
+                              partial_floats, nullptr, nullptr));
+    FAX_TRY(fax_colsum(ctx, prec, rows, d, add, d, sum_add, accumulate, partial, partial_floats));
+    return fax_colsum(ctx, prec, rows, d, dx, d, sum_out, accumulate, partial, partial_floats);
+  }
   // dx pass reads da, x (and add) and writes dx; the dgamma/dbeta pass reads da and x again
   FaxProfScope prof(ctx, KC_LN_BWD, 0.0, (double)rows * d * fax_elem_size(prec) * (add ? 4 : 3));
   if (ln_bwd_is_fused(d / (prec == FAX_PREC_BF16 ? 8 : 4))) {
     if (prec == FAX_PREC_BF16)
-      return ln_bwd_fused_t<bf16>(ctx, rows, d, da, x, mu, rstd, gamma, add, dx, dgamma, dbeta, accumulate, partial);
-    return ln_bwd_fused_t<float>(ctx, rows, d, da, x, mu, rstd, gamma, add, dx, dgamma, dbeta, accumulate, partial);
+      return ln_bwd_fused_t<bf16>(ctx, rows, d, da, x, mu, rstd, gamma, add, dx, dgamma, dbeta, accumulate, partial,
+                                  sum_add, sum_out);
+    return ln_bwd_fused_t<float>(ctx, rows, d, da, x, mu, rstd, gamma, add, dx, dgamma, dbeta, accumulate, partial,
+                                 sum_add, sum_out);
   }
   if (prec == FAX_PREC_BF16) {
     FAX_TRY(ln_bwd_dx_t<bf16>(ctx, rows, d, da, x, mu, rstd, gamma, add, dx));
