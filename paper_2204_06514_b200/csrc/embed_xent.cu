@@ -170,13 +170,14 @@ xent_stream_kernel(int rows, int vocab, bf16* __restrict__ logits, int64_t ld, c
       uint4* xrow = xs_raw + (size_t)b * nvec;
       if (!mbar_wait_warp(full_bar(b), (uint32_t)(k >> 1) & 1u, abort_flag, status, 402)) { ok = false; break; }
       const int tg = targets[r];
-      float mx = -INFINITY;
+      // maximum in packed bf16 pairs (exact: the values are bf16)
+      __nv_bfloat162 m2 = __float2bfloat162_rn(-INFINITY);
       for (int i = threadIdx.x; i < nvec; i += XS_COMPUTE_THREADS) {
         const uint4 u = xrow[i];
         const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&u);
-#pragma unroll
-        for (int e = 0; e < 4; ++e) { float2 f = __bfloat1622float2(h[e]); mx = fmaxf(mx, fmaxf(f.x, f.y)); }
+        m2 = __hmax2(__hmax2(m2, h[0]), __hmax2(h[1], __hmax2(h[2], h[3])));
       }
+      float mx = fmaxf(__low2float(m2), __high2float(m2));
       float lt = 0.f;
       if (threadIdx.x == 0 && tg >= 0 && tg < vocab) lt = __bfloat162float(reinterpret_cast<const bf16*>(xrow)[tg]);
       // block-wide reductions among the compute warps only (named barrier 1)
@@ -208,17 +209,26 @@ xent_stream_kernel(int rows, int vocab, bf16* __restrict__ logits, int64_t ld, c
         row_loss[r] = (tg >= 0 && tg < vocab) ? lse - lt : 0.f;
       }
       const float kk = inv_n / s;
+      const int tgv = (tg >= 0 && tg < vocab) ? (tg >> 3) : -1;       // the one vector that holds the target column
       for (int i = threadIdx.x; i < nvec; i += XS_COMPUTE_THREADS) {
         uint4 u = xrow[i];
         __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&u);
-        const int c0 = i << 3;
+        if (i != tgv) {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          float2 f = __bfloat1622float2(h[e]);
-          float p0 = f.x * kk, p1 = f.y * kk;
-          if (c0 + 2 * e == tg) p0 -= inv_n;
-          if (c0 + 2 * e + 1 == tg) p1 -= inv_n;
-          h[e] = __floats2bfloat162_rn(p0, p1);
+          for (int e = 0; e < 4; ++e) {
+            const float2 f = __bfloat1622float2(h[e]);
+            h[e] = __floats2bfloat162_rn(f.x * kk, f.y * kk);
+          }
+        } else {
+          const int c0 = i << 3;
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float2 f = __bfloat1622float2(h[e]);
+            float p0 = f.x * kk, p1 = f.y * kk;
+            if (c0 + 2 * e == tg) p0 -= inv_n;
+            if (c0 + 2 * e + 1 == tg) p1 -= inv_n;
+            h[e] = __floats2bfloat162_rn(p0, p1);
+          }
         }
         xrow[i] = u;
       }
