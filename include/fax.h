@@ -17,6 +17,10 @@
  *    synchronising, except the *_host entry points and an explicit host loss
  *    readback, which synchronise the stream before returning.
  *  - Calls on one context are not thread-safe; contexts are independent.
+ *  - Current device: fax_create and fax_destroy make the context's device
+ *    current themselves (and leave it current); every other call must be made
+ *    with the context's device current on the calling thread.  A process may
+ *    hold contexts on several devices.
  *  - Inputs are never modified unless stated (AdamW updates state in place).
  *  - Shapes: tokens N = batch*seq; d_model = n_heads*head_dim; head_dim is 64
  *    or 128; in FAX_PREC_BF16 d_model, d_ff and vocab must be multiples of 128
@@ -212,6 +216,13 @@ fax_status fax_set_gemm_two_cta(fax_ctx* ctx, int32_t enable);
  * complete before it touches global memory, so results are the same.
  * enable = 0 launches every kernel fully serialised.  Default: enabled. */
 fax_status fax_set_dependent_launch(fax_ctx* ctx, int32_t enable);
+
+/* Attention backward at head_dim 128 walks the queries of a key tile in
+ * sub-tiles of 64 with two of them in flight (the row warps work on one while
+ * the tensor cores run the other's products); enable = 0 keeps the kernel with
+ * one 128-query tile in flight, which also serves head_dim 64.  Same arithmetic
+ * (the float32 dQ additions arrive in another order).  Default: enabled. */
+fax_status fax_set_attention_backward_two_chains(fax_ctx* ctx, int32_t enable);
 
 /* One trainable tensor of a training state: float32 master, compute-precision
  * copy (bf16; in FP32_VALIDATE may equal w or be NULL), Adam moments, float32

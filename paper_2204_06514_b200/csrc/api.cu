@@ -40,6 +40,7 @@ extern "C" fax_status fax_create(fax_ctx** out, int32_t device_ordinal, void* cu
   c->overlap_adamw = true;
   c->use_2cta = true;
   c->use_pdl = true;
+  c->attn_bwd_two_chains = true;
   c->use_graphs = true;
   c->fused_update = false;
   c->keep_fused_grads = false;
@@ -141,6 +142,14 @@ extern "C" fax_status fax_set_gemm_two_cta(fax_ctx* ctx, int32_t enable) {
 extern "C" fax_status fax_set_dependent_launch(fax_ctx* ctx, int32_t enable) {
   if (!ctx) return FAX_ERR_INVALID_ARG;
   ctx->use_pdl = enable != 0;
+  cudaStreamSynchronize(ctx->stream);
+  fax_graph_clear(ctx);
+  return FAX_OK;
+}
+
+extern "C" fax_status fax_set_attention_backward_two_chains(fax_ctx* ctx, int32_t enable) {
+  if (!ctx) return FAX_ERR_INVALID_ARG;
+  ctx->attn_bwd_two_chains = enable != 0;
   cudaStreamSynchronize(ctx->stream);
   fax_graph_clear(ctx);
   return FAX_OK;

@@ -302,12 +302,8 @@ fax_status launch_fwd2(fax_ctx* ctx, int B, int T, int H, const void* qkv, void*
   p.B = B; p.T = T; p.H = H; p.o = (bf16*)o; p.lse = lse;
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
   p.status = ctx->dev_status;
-  static bool attr_set = false;
-  if (!attr_set) {
-    FAX_CUDA_TRY(ctx, cudaFuncSetAttribute(attn_fwd2_tc_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           Fwd2Cfg<HD>::SMEM_BYTES));
-    attr_set = true;
-  }
+  static bool attr_set[FAX_MAX_DEVICES] = {};
+  FAX_TRY(fax_opt_in_shared_memory(ctx, attn_fwd2_tc_kernel<HD>, Fwd2Cfg<HD>::SMEM_BYTES, attr_set));
   const long long items = (long long)B * H * (T / 256);
   const int grid = (int)(items < ctx->sm_count ? items : ctx->sm_count);
   fax_launch(ctx, attn_fwd2_tc_kernel<HD>, dim3(grid), dim3(F2_THREADS), Fwd2Cfg<HD>::SMEM_BYTES, map, p);

@@ -272,12 +272,8 @@ fax_status launch_fwd(fax_ctx* ctx, int B, int T, int H, const void* qkv, void* 
   p.B = B; p.T = T; p.H = H; p.o = (bf16*)o; p.lse = lse;
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)HD);
   p.status = ctx->dev_status;
-  static bool attr_set = false;
-  if (!attr_set) {
-    FAX_CUDA_TRY(ctx, cudaFuncSetAttribute(attn_fwd_tc_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           FwdCfg<HD>::SMEM_BYTES));
-    attr_set = true;
-  }
+  static bool attr_set[FAX_MAX_DEVICES] = {};
+  FAX_TRY(fax_opt_in_shared_memory(ctx, attn_fwd_tc_kernel<HD>, FwdCfg<HD>::SMEM_BYTES, attr_set));
   const int grid = B * H * (T / TQ);
   fax_launch(ctx, attn_fwd_tc_kernel<HD>, dim3(grid), dim3(FWD_THREADS), FwdCfg<HD>::SMEM_BYTES, map, p);
   return fax_after_launch(ctx);
@@ -756,16 +752,16 @@ fax_status launch_bwd(fax_ctx* ctx, int B, int T, int H, const void* qkv, const 
   p.scale = 1.0f / sqrtf((float)HD);
   p.scale_log2 = 1.4426950408889634f * p.scale;
   p.status = ctx->dev_status;
-  static bool attr_set = false;
-  if (!attr_set) {
-    FAX_CUDA_TRY(ctx, cudaFuncSetAttribute(attn_bwd2_tc_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           Bwd2Cfg<HD>::SMEM_BYTES));
-    attr_set = true;
+  if (HD == 128 && ctx->attn_bwd_two_chains && fax_attention_bwd3_supported(B, T, H, HD)) {
+    FAX_TRY(fax_attention_bwd3_tc(ctx, B, T, H, qkv, lse, d_o, dqkv, Dv, dq_acc));
+  } else {
+    static bool attr_set[FAX_MAX_DEVICES] = {};
+    FAX_TRY(fax_opt_in_shared_memory(ctx, attn_bwd2_tc_kernel<HD>, Bwd2Cfg<HD>::SMEM_BYTES, attr_set));
+    const long long items = (long long)B * H * (T / 128);
+    const int grid = (int)(items < ctx->sm_count ? items : ctx->sm_count);
+    fax_launch(ctx, attn_bwd2_tc_kernel<HD>, dim3(grid), dim3(BWD_THREADS), Bwd2Cfg<HD>::SMEM_BYTES, mq, md, mdq, p);
+    FAX_TRY(fax_after_launch(ctx));
   }
-  const long long items = (long long)B * H * (T / 128);
-  const int grid = (int)(items < ctx->sm_count ? items : ctx->sm_count);
-  fax_launch(ctx, attn_bwd2_tc_kernel<HD>, dim3(grid), dim3(BWD_THREADS), Bwd2Cfg<HD>::SMEM_BYTES, mq, md, mdq, p);
-  FAX_TRY(fax_after_launch(ctx));
   const long long quads = n_tok * (long long)d / 4;
   fax_launch(ctx, attn_dq_convert_kernel, dim3((unsigned)((quads + 255) / 256)), dim3(256), 0, n_tok, (int)d, dq_acc,
              p.scale, (bf16*)dqkv);

@@ -59,6 +59,7 @@ struct fax_ctx {
   bool keep_fused_grads;     // ... and still store those gradients
   bool use_2cta;             // GEMMs whose M and N are multiples of 256 use the two-CTA kernel
   bool use_pdl;              // kernels are launched with programmatic stream serialization allowed
+  bool attn_bwd_two_chains;  // head_dim-128 attention backward runs the kernel with two query sub-tiles in flight
 };
 
 // Brackets the launches of one operator with CUDA events while profiling is on.
@@ -119,6 +120,22 @@ static inline void fax_launch(fax_ctx* ctx, void (*kernel)(KArgs...), dim3 grid,
   cfg.attrs = &attr;
   cfg.numAttrs = ctx->use_pdl ? 1 : 0;
   (void)cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);     // errors surface in fax_after_launch
+}
+
+// Kernels that need more than 48 KB of dynamic shared memory opt in once per device (the attribute is
+// per device, a process may hold contexts on several): `done` is the call site's own flag array.
+constexpr int FAX_MAX_DEVICES = 64;
+template <typename K>
+static inline fax_status fax_opt_in_shared_memory(fax_ctx* ctx, K* kernel, int bytes, bool* done) {
+  const bool tracked = ctx->device >= 0 && ctx->device < FAX_MAX_DEVICES;
+  if (tracked && done[ctx->device]) return FAX_OK;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e != cudaSuccess) {
+    ctx->last_cuda_error = (int32_t)e;
+    return FAX_ERR_CUDA;
+  }
+  if (tracked) done[ctx->device] = true;
+  return FAX_OK;
 }
 
 static inline bool fax_aligned(const void* p, size_t a) { return ((uintptr_t)p & (a - 1)) == 0; }
@@ -276,5 +293,9 @@ fax_status fax_gelu_fwd(fax_ctx* ctx, int prec, size_t n, const void* h, void* g
 bool fax_attention_fwd2_supported(int B, int T, int H, int hd);
 fax_status fax_attention_fwd2_tc(fax_ctx* ctx, int B, int T, int H, int hd, const void* qkv, void* o, float* lse);
 size_t fax_attention_bwd_tc_scratch_bytes(int B, int T, int H, int hd);
+// head_dim-128 backward with two query sub-tiles in flight (the main kernel only; see its definition)
+bool fax_attention_bwd3_supported(int B, int T, int H, int hd);
+fax_status fax_attention_bwd3_tc(fax_ctx* ctx, int B, int T, int H, const void* qkv, const float* lse,
+                                 const void* d_o, void* dqkv, const float* Dv, float* dq_acc);
 fax_status fax_attention_bwd_tc(fax_ctx* ctx, int B, int T, int H, int hd, const void* qkv, const void* o,
                                 const float* lse, const void* d_o, void* dqkv, void* scratch, size_t scratch_bytes);

@@ -292,11 +292,8 @@ fax_status fax_xent(fax_ctx* ctx, int prec, int rows, int vocab, void* logits, i
   const bool vec_ok = prec == FAX_PREC_BF16 && vocab % 8 == 0 && ld % 8 == 0 && fax_aligned(logits, 16);
   if (vec_ok && 2 * row_bytes <= 220 * 1024) {
     // two rows fit: persistent kernel, rows streamed through shared memory by bulk copies
-    static bool attr_set = false;
-    if (!attr_set) {
-      FAX_CUDA_TRY(ctx, cudaFuncSetAttribute(xent_stream_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
-      attr_set = true;
-    }
+    static bool attr_set[FAX_MAX_DEVICES] = {};
+    FAX_TRY(fax_opt_in_shared_memory(ctx, xent_stream_kernel, 220 * 1024, attr_set));
     const int grid = rows < ctx->sm_count ? rows : ctx->sm_count;
     fax_launch(ctx, xent_stream_kernel, dim3(grid), dim3(XS_THREADS), 2 * row_bytes, rows, vocab, (bf16*)logits,
                ld, targets, inv_n, row_loss, ctx->dev_status);

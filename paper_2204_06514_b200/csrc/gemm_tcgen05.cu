@@ -200,12 +200,8 @@ fax_status launch(fax_ctx* ctx, const FaxGemm& g) {
   if (!ok) return FAX_ERR_INVALID_ARG;
   GemmParams p;
   fill_gemm_params(p, g, ctx->dev_status);
-  static bool attr_set = false;
-  if (!attr_set) {
-    FAX_CUDA_TRY(ctx, cudaFuncSetAttribute(gemm_tcgen05_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           Cfg<BN>::SMEM_BYTES));
-    attr_set = true;
-  }
+  static bool attr_set[FAX_MAX_DEVICES] = {};
+  FAX_TRY(fax_opt_in_shared_memory(ctx, gemm_tcgen05_kernel<BN>, Cfg<BN>::SMEM_BYTES, attr_set));
   const int tiles = (g.M / BM) * (g.N / BN);
   // Few output tiles and a long K (the weight-gradient shapes of narrow models): slice K so that
   // the machine is filled; partial tiles are added into the float output with vector atomics.

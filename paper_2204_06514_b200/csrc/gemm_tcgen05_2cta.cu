@@ -246,13 +246,12 @@ fax_status fax_gemm_tc2(fax_ctx* ctx, const FaxGemm& g) {
   if (!ok) return FAX_ERR_INVALID_ARG;
   GemmParams p;
   fill_gemm_params(p, g, ctx->dev_status);
-  static bool attr_set = false;
-  if (!attr_set) {
-#define FAX_SET_SMEM(E) FAX_CUDA_TRY(ctx, cudaFuncSetAttribute(gemm_tcgen05_2cta_kernel<E>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES))
-    FAX_SET_SMEM(-1); FAX_SET_SMEM(0); FAX_SET_SMEM(1); FAX_SET_SMEM(2); FAX_SET_SMEM(3); FAX_SET_SMEM(4);
-    FAX_SET_SMEM(EPI_STATIC_F32);
+  {
+    static bool attr_set[7][FAX_MAX_DEVICES] = {};
+#define FAX_SET_SMEM(I, E) FAX_TRY(fax_opt_in_shared_memory(ctx, gemm_tcgen05_2cta_kernel<E>, SMEM_BYTES, attr_set[I]))
+    FAX_SET_SMEM(0, -1); FAX_SET_SMEM(1, 0); FAX_SET_SMEM(2, 1); FAX_SET_SMEM(3, 2); FAX_SET_SMEM(4, 3); FAX_SET_SMEM(5, 4);
+    FAX_SET_SMEM(6, EPI_STATIC_F32);
 #undef FAX_SET_SMEM
-    attr_set = true;
   }
   const int tiles = (g.M / 256) * (g.N / 256);
   const int max_pairs = ctx->sm_count / 2;

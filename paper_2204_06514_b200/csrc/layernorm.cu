@@ -630,13 +630,10 @@ fax_status ln_bwd_fused_t(fax_ctx* ctx, int rows, int d, const void* da, const v
 #define LN_FUSED_S(V, W, S)                                                                            \
   {                                                                                                    \
     const size_t smem = ((size_t)ns * d * sizeof(float) + 15) / 16 * 16 + ring_bytes(V, W);            \
-    static bool attr_set = false;                                                                      \
-    if (!attr_set) {                                                                                   \
-      FAX_CUDA_TRY(ctx, cudaFuncSetAttribute(layernorm_bwd_ring_kernel<T, V, W, S>,                    \
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize,              \
-                                             (int)((size_t)(S ? 4 : 2) * 512 * Vec<T>::N * sizeof(float) + ring_bytes(V, W)))); \
-      attr_set = true;                                                                                 \
-    }                                                                                                  \
+    static bool attr_set[FAX_MAX_DEVICES] = {};                                                        \
+    FAX_TRY(fax_opt_in_shared_memory(ctx, layernorm_bwd_ring_kernel<T, V, W, S>,                       \
+                                     (int)((size_t)(S ? 4 : 2) * 512 * Vec<T>::N * sizeof(float) + ring_bytes(V, W)), \
+                                     attr_set));                                                       \
     fax_launch(ctx, layernorm_bwd_ring_kernel<T, V, W, S>, dim3(grid), dim3(512), smem,                \
                rows, d, (const T*)da, (const T*)x, mu, rstd, (const T*)gamma, (const T*)add, (T*)dx, partial); \
   }
@@ -764,9 +761,15 @@ extern "C" fax_status fax_op_layernorm_backward_static(fax_ctx* ctx, int32_t pre
     return FAX_ERR_WORKSPACE_TOO_SMALL;
   if (!g_ln_static_ptr[ctx->device]) {
     // one-time set-up on this device (no allocation: the array already exists in the loaded module)
+    // (the symbol is looked up on the current device, so the context's device is made current
+    // for the query and the caller's choice put back afterwards)
+    int caller_device = -1;
+    FAX_CUDA_TRY(ctx, cudaGetDevice(&caller_device));
     FAX_CUDA_TRY(ctx, cudaSetDevice(ctx->device));
     float* ptr = nullptr;
-    FAX_CUDA_TRY(ctx, cudaGetSymbolAddress((void**)&ptr, g_ln_static_partial));
+    const cudaError_t e = cudaGetSymbolAddress((void**)&ptr, g_ln_static_partial);
+    if (caller_device != ctx->device) (void)cudaSetDevice(caller_device);
+    FAX_CUDA_TRY(ctx, e);
     if (!ptr) return FAX_ERR_CUDA;
     g_ln_static_ptr[ctx->device] = ptr;
   }

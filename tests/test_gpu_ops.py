@@ -189,7 +189,7 @@ def test_gemm_weight_gradient_shapes_split_k(sess, M, N, K, accumulate):
 
 # T a multiple of 256 takes the two-tile persistent forward kernel; the last two bf16 shapes give it more
 # work items than the GPU has SMs, so CTAs loop over several query-tile pairs
-ATTN_SHAPES = [(0, 2, 128, 4, 64), (0, 1, 384, 2, 128), (0, 2, 1024, 2, 64), (0, 1, 2048, 1, 128),
+ATTN_SHAPES = [(0, 2, 128, 4, 64), (0, 1, 128, 1, 128), (0, 1, 384, 2, 128), (0, 2, 1024, 2, 64), (0, 1, 2048, 1, 128),
                (0, 8, 512, 24, 64), (0, 4, 768, 13, 128),
                (1, 2, 5, 2, 4), (1, 2, 130, 3, 64), (1, 1, 77, 2, 128)]
 
