@@ -8,11 +8,12 @@ inputs resident in HBM; `e2e` = the same through the host-buffer entry point
 (host->device copies of the step's inputs and device->host read of its results
 inside the timed region).  N > 1 runs N independent replicas (one process per
 GPU, no data-path collective): the step has no exchange step on one device.
-`--impl reference` times the fp64 CPU oracle on a bounded sample instead.
+`--impl reference` times the fp64 CPU oracle instead.
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import subprocess
@@ -27,8 +28,12 @@ if ROOT not in sys.path:
 METRIC = "training tokens/sec, fwd+bwd+AdamW, 1 GPU (MFU reported beside it)"
 UNIT = "tokens/s"
 NOMINAL_BF16_TFLOPS = 2250.0        # B200 dense bf16, datasheet
-GEMM_DRAM_BYTES_PER_LAUNCH = {"C3": 960.9e6}     # mean over the step's 12 GEMM launches (algorithmic: 459e6)
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "gemm_dram_traffic.json")
+# A tensor kernel is compared with the burst GEMM peak when the GPU never settled into the power-capped
+# state the sustained figure was measured in: timed region under a second, or SM clock sampled above this
+BURST_MHZ = 1600.0
+BURST_REGION_MS = 1000.0
 
 
 def load_peaks():
@@ -42,8 +47,31 @@ def load_peaks():
     return dict(FALLBACK_PEAKS), "fallback"
 
 
+def gemm_source_digest() -> str:
+    """sha256 over the GEMM kernel sources: a stored traffic figure holds only for the kernels it was taken on."""
+    h = hashlib.sha256()
+    for name in ("gemm_tcgen05_2cta.cu", "gemm_tcgen05.cu", "gemm_common.cuh", "tc_common.cuh"):
+        with open(os.path.join(ROOT, "paper_2204_06514_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def stored_gemm_traffic(workload: str):
+    """DRAM bytes (read + written) per GEMM launch of a workload's step, the mean over its launches, taken
+    from one-launch ncu captures of each shape; None when no capture exists for the workload or the GEMM
+    sources have changed since."""
+    try:
+        d = json.load(open(TRAFFIC_FILE))
+    except (OSError, ValueError):
+        return None
+    if d.get("gemm_source_digest") != gemm_source_digest():
+        return None
+    w = d.get("workloads", {}).get(workload)
+    return float(w["dram_bytes_per_launch_mean"]) if w else None
+
+
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    """Samples nvidia-smi clocks and throttle reasons for the life of the run; windows are cut out afterwards."""
 
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
@@ -56,7 +84,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "50"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
             return
@@ -67,16 +95,23 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.rows.append((time.time(), [c.strip() for c in line.split(",")]))
 
-    def stop(self, t0: float, t1: float) -> dict:
+    def stop(self):
         if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+            return
         time.sleep(0.15)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
-        rows = [r for t, r in self.rows if t0 <= t <= t1 + 0.2] or [r for _, r in self.rows]
+
+    def window(self, t0: float, t1: float) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        allrows = list(self.rows)
+        rows = [r for t, r in allrows if t0 <= t <= t1 + 0.05]
+        if not rows:      # a region shorter than the sampling period: the nearest sample
+            rows = [r for _, r in sorted(allrows, key=lambda tr: abs(tr[0] - 0.5 * (t0 + t1)))[:1]]
         sm, mx, reasons, pw = [], [], set(), []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in rows:
@@ -92,94 +127,114 @@ class ClockSampler:
                 "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
+# ---------------------------------------------------------------------------------------------
+# The oracle on host cores.  Where host memory and a few minutes allow, ONE whole full-size step
+# is timed (forward, loss, backward, AdamW on every tensor).  Otherwise a bounded sample at the
+# full sequence length: fewer sequences of the batch (time scales with tokens, attention included),
+# or AdamW on a leading slice of every tensor (time scales with elements); the line then says
+# "extrapolated": true and gives the factors.
+# name -> (sequences timed, AdamW divisor)
+ORACLE_PLAN = {"C1": (None, 1), "C2": (None, 1), "C3": (None, 1), "C4": (None, 1),
+               "C5": (None, 16), "P1": (None, 16), "P2": (None, 16), "P3": (None, 16),
+               "F2": (4, 1), "F3": (4, 1)}
 _ORACLE_INPUTS = {}
 
 
-def oracle_sample(cfg, n_tokens: int):
-    """Time the fp64 oracle (as it stands) on a bounded sample of the workload and
-    extrapolate to tokens/s of the full step.  Block configs: forward + backward at
-    full widths on one sequence of n_tokens tokens (time scaled by tokens), plus the
-    oracle's AdamW on the leading 1/16 of every tensor (time scaled by 16).  The LM
-    config: lm_step on one n_tokens sequence with 2 layers, scaled by FLOPs per token."""
+def oracle_step_seconds(cfg):
+    """Seconds the oracle needs for one step of `cfg` on this host, with what was timed.
+    Returns (seconds for the full step, cores, description, extrapolated, factors)."""
     import numpy as np
     import threadpoolctl
     from oracle import fax_oracle as O
     from paper_2204_06514_b200 import synth
-    seq = min(cfg.seq, n_tokens)
-    small = synth.scaled(cfg, batch=1, seq=seq, n_layers=min(cfg.n_layers, 2) if cfg.is_lm else 1)
+    seqs, adam_div = ORACLE_PLAN[cfg.name]
+    batch = cfg.batch if seqs is None else min(seqs, cfg.batch)
+    small = synth.scaled(cfg, batch=batch)
     hp = dict(synth.ADAMW, step=1)
     info = threadpoolctl.threadpool_info()
     cores = max((i.get("num_threads", 1) for i in info), default=1)
-    key = (cfg.name, seq)
+    key = (cfg.name, batch)
     if key not in _ORACLE_INPUTS:
         rng = np.random.default_rng(0)
-        blocks = [{k: rng.standard_normal(s) * 0.02 for k, s in small.block_param_shapes().items()}
-                  for _ in range(small.n_layers)]
+        blocks = [{k: (rng.standard_normal(s) * 0.02 if k.startswith("w_") else
+                       (np.ones(s) if k.endswith("_g") else np.zeros(s)))
+                   for k, s in small.block_param_shapes().items()} for _ in range(small.n_layers)]
         if small.is_lm:
             _ORACLE_INPUTS[key] = dict(
                 lm=dict(wte=rng.standard_normal((small.vocab, small.d_model)) * 0.02,
-                        wpe=rng.standard_normal((seq, small.d_model)) * 0.02, blocks=blocks,
+                        wpe=rng.standard_normal((small.seq, small.d_model)) * 0.02, blocks=blocks,
                         lnf_g=np.ones(small.d_model), lnf_b=np.zeros(small.d_model)),
-                ids=rng.integers(0, small.vocab, (1, seq)))
+                ids=rng.integers(0, small.vocab, (batch, small.seq + 1)))
         else:
-            _ORACLE_INPUTS[key] = dict(p=blocks[0], x=rng.standard_normal((seq, small.d_model)),
-                                       dy=rng.standard_normal((seq, small.d_model)))
+            _ORACLE_INPUTS[key] = dict(p=blocks[0], x=rng.standard_normal((small.tokens, small.d_model)),
+                                       dy=rng.standard_normal((small.tokens, small.d_model)))
     inp = _ORACLE_INPUTS[key]
+    tok_factor = cfg.tokens / small.tokens
     if small.is_lm:
         lm, ids = inp["lm"], inp["ids"]
         zeros = {n: np.zeros(a.shape) for n, a in O.lm_tensors(lm)}
         t0 = time.perf_counter()
-        O.lm_step(ids, ids, lm, zeros, zeros, 1, seq, small.n_heads, small.head_dim, hp, small.ln_eps)
+        O.lm_step(ids[:, :-1], ids[:, 1:], lm, zeros, zeros, batch, small.seq, small.n_heads, small.head_dim, hp,
+                  small.ln_eps)
         dt = time.perf_counter() - t0
-        frac = (small.step_flops() / small.tokens) / (cfg.step_flops() / cfg.tokens)
-        full = dt / frac * (cfg.tokens / seq)
-        what = (f"oracle lm_step on 1 x {seq} tokens with {small.n_layers} of {cfg.n_layers} layers, "
-                f"time scaled by FLOPs per token and by tokens to the full step")
-    else:
-        p, x, dy = inp["p"], inp["x"], inp["dy"]
+        if tok_factor == 1:
+            return dt, cores, f"one whole oracle lm_step (forward, loss, backward, AdamW) at full size", False, {}
+        # AdamW does not scale with tokens: time it apart on the same tensors
         t0 = time.perf_counter()
-        y, sv = O.block_forward(x, p, 1, seq, small.n_heads, small.head_dim, small.ln_eps)
-        dx, gr, _ = O.block_backward(dy, sv, p, 1, seq, small.n_heads, small.head_dim)
-        t_fb = time.perf_counter() - t0
-        div = 16 if cfg.n_params > 10_000_000 else 1
-        t0 = time.perf_counter()
-        for k in O.PARAM_NAMES:
-            n = max(1, p[k].shape[0] // div)
-            w, g = p[k][:n], gr[k][:n]
-            O.adamw(w, np.zeros_like(w), np.zeros_like(w), g, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"],
-                    hp["weight_decay"], 1)
-        t_ad = (time.perf_counter() - t0) * div
-        full = t_fb * (cfg.tokens / seq) + t_ad
-        what = (f"oracle block forward+backward at full widths on 1 x {seq} tokens (time scaled by tokens) "
-                f"+ oracle AdamW on the leading 1/{div} of every tensor (time scaled by {div})")
-    return cfg.tokens / full, cores, what
-
-
-SAMPLE_TOKENS = {"C1": 128, "C2": 512, "C3": 128, "C4": 128, "C5": 32, "P1": 128, "P2": 32, "P3": 16,
-                 "F3": 128, "F2": 128}
+        for n, a in O.lm_tensors(lm):
+            O.adamw(a, zeros[n], zeros[n], zeros[n], hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["weight_decay"], 1)
+        t_ad = time.perf_counter() - t0
+        full = (dt - t_ad) * tok_factor + t_ad
+        return (full, cores, f"oracle lm_step on {batch} of {cfg.batch} sequences at the full sequence length and depth; "
+                f"forward+loss+backward time scaled by tokens, AdamW (all tensors) counted once", True,
+                {"tokens": tok_factor})
+    p, x, dy = inp["p"], inp["x"], inp["dy"]
+    t0 = time.perf_counter()
+    y, sv = O.block_forward(x, p, small.batch, small.seq, small.n_heads, small.head_dim, small.ln_eps)
+    dx, gr, _ = O.block_backward(dy, sv, p, small.batch, small.seq, small.n_heads, small.head_dim)
+    t_fb = time.perf_counter() - t0
+    del sv
+    t0 = time.perf_counter()
+    for k in O.PARAM_NAMES:
+        n = max(1, p[k].shape[0] // adam_div)
+        w, g = p[k][:n], gr[k][:n]
+        O.adamw(w, np.zeros_like(w), np.zeros_like(w), g, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"],
+                hp["weight_decay"], 1)
+    t_ad = (time.perf_counter() - t0) * adam_div
+    full = t_fb * tok_factor + t_ad
+    if adam_div == 1 and tok_factor == 1:
+        return full, cores, "one whole oracle block step (forward, backward, AdamW on all twelve tensors) at full size", False, {}
+    return (full, cores, f"oracle block forward+backward at full size (all {cfg.tokens} tokens) + oracle AdamW on the leading "
+            f"1/{adam_div} of every tensor, that time scaled by {adam_div} (float64 copies of the optimizer state of "
+            f"{cfg.n_params / 1e9:.1f}e9 parameters do not fit beside the gradients)", True, {"adamw": adam_div})
 
 
 def run_reference(args):
-    """Reference arm: the fp64 oracle on host cores, bounded sample per step."""
+    """Reference arm: the fp64 oracle on host cores.  Small workloads: warm-up and K real steps; from C3 on,
+    one real step (or the bounded sample), timed once."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     from paper_2204_06514_b200 import synth
     cfg = synth.CONFIGS[args.config]
-    budget = SAMPLE_TOKENS[args.config]
-    vals, cores, what = [], 1, ""
-    for i in range(args.warmup + args.steps):
-        v, cores, what = oracle_sample(cfg, budget)
-        if i >= args.warmup:
-            vals.append(v)
-    tps = sum(vals) / len(vals)
+    t_proc = time.perf_counter()
+    repeat = cfg.name in ("C1", "C2")
+    secs, cores, what, extrap, factors = [], 1, "", False, {}
+    for i in range((args.warmup + args.steps) if repeat else 1):
+        s, cores, what, extrap, factors = oracle_step_seconds(cfg)
+        if not repeat or i >= args.warmup:
+            secs.append(s)
+    sec = sum(secs) / len(secs)
+    tps = cfg.tokens / sec
     line = {"impl": "reference", "metric": METRIC, "value": tps, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * cfg.tokens / tps,
+            "steps": args.steps, "warmup": args.warmup, "steps_timed": len(secs), "ms_per_step": 1e3 * sec,
+            "extrapolated": extrap, "extrapolation_factors": factors,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
             "data": "synthetic", "config": {"workload": workload_name(cfg)},
-            "cpu_baseline": {"value": tps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what},
+            "cpu_baseline": {"value": tps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what,
+                             "extrapolated": extrap},
             "e2e": {"value": tps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
-            "gpu_launches": 0}
+            "gpu_launches": 0, "process_seconds": time.perf_counter() - t_proc}
     print(json.dumps(line), flush=True)
 
 
@@ -192,7 +247,6 @@ def workload_name(cfg):
 
 
 def run_ours(args):
-    import numpy as np
     import torch
     import torch.distributed as dist
 
@@ -273,13 +327,15 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     step_marks = []
+    windows = {}
 
-    def timed(fn, steps, marks=None):
+    def timed(fn, steps, marks=None, tag=None):
         """K steps between two CUDA events on the launching stream; max over ranks.  With `marks`, an event
         after every step as well (per-step median / minimum; the total is what the metric uses)."""
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         evs = [torch.cuda.Event(enable_timing=True) for _ in range(steps)] if marks is not None else None
         barrier()
+        h0 = time.time()
         e0.record(sess.stream)
         for i in range(steps):
             fn()
@@ -287,6 +343,9 @@ def run_ours(args):
                 evs[i].record(sess.stream)
         e1.record(sess.stream)
         barrier()
+        if tag:
+            a, b = windows.get(tag, (h0, h0))
+            windows[tag] = (min(a, h0) if tag in windows else h0, time.time())
         if evs:
             prev = e0
             for e in evs:
@@ -294,17 +353,15 @@ def run_ours(args):
                 prev = e
         return dist_util.max_over_ranks(e0.elapsed_time(e1), dev)
 
-    for _ in range(max(args.warmup, 3)):
-        step()
     sampler = ClockSampler(local)
     sampler.start()
-    time.sleep(0.25)
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    time.sleep(0.1)
     l0 = sess.launches()
-    t0 = time.time()
-    ms = timed(step, args.steps, step_marks)
-    t1 = time.time()
+    ms = timed(step, args.steps, step_marks, tag="timed")
     launches = sess.launches() - l0
-    clocks = sampler.stop(t0, t1)
     st, detail = fx.fax_check_device_status(sess.ctx)
     if st != fx.FAX_OK:
         raise RuntimeError(f"device status {st} detail {detail}")
@@ -312,32 +369,38 @@ def run_ours(args):
     # end to end through the host-buffer entry point
     step_host()
     e2e_steps = max(1, min(args.steps, 10))
-    ms_e2e = timed(step_host, e2e_steps)
+    ms_e2e = timed(step_host, e2e_steps, tag="e2e")
 
     # per-kernel profile over whole steps (events around every operator launch)
     # (AdamW is kept on the main stream here so that no kernel's events include another's work)
     fx.fax_set_adamw_overlap(sess.ctx, False)
     fx.fax_profile_begin(sess.ctx)
     prof_steps = max(1, min(args.steps, 5))
+    hp_t0 = time.time()
     for _ in range(prof_steps):
         step()
     prof = fx.fax_profile_end(sess.ctx)
+    windows["profile"] = (hp_t0, time.time())
     fx.fax_set_adamw_overlap(sess.ctx, True)
 
     # per-phase split (the paper's Fig. 3 reports forward, loss and backward separately): the phase
     # entry points timed on their own, outside the step's timed region
     ph_steps = max(1, min(args.steps, 5))
     if cfg.is_lm:
-        fb = timed(lambda: runner.forward_backward(ids, tg), ph_steps) / ph_steps
+        fb = timed(lambda: runner.forward_backward(ids, tg), ph_steps, tag="phases") / ph_steps
         phases = {"forward_loss_backward_ms": fb, "adamw_ms": max(ms / args.steps - fb, 0.0),
                   "note": "forward + loss + backward through fax_lm_forward_backward; AdamW = step - that"}
+        sum_phases = None
     else:
         hp_ph = hparams(step=1, **hp0)
-        fwd = timed(lambda: runner.forward(x), ph_steps) / ph_steps
-        bwd = timed(lambda: runner.backward(dy), ph_steps) / ph_steps
-        adw = timed(lambda: runner.adamw(hp_ph), ph_steps) / ph_steps
+        fwd = timed(lambda: runner.forward(x), ph_steps, tag="phases") / ph_steps
+        bwd = timed(lambda: runner.backward(dy), ph_steps, tag="phases") / ph_steps
+        adw = timed(lambda: runner.adamw(hp_ph), ph_steps, tag="phases") / ph_steps
         phases = {"forward_ms": fwd, "backward_ms": bwd, "adamw_ms": adw,
                   "note": "fax_block_forward, fax_block_backward, fax_adamw_step timed separately"}
+        sum_phases = fwd + bwd + adw
+    sampler.stop()
+    clocks = {k: sampler.window(*w) for k, w in windows.items()}
 
     if rank != 0:
         if world > 1:
@@ -349,6 +412,12 @@ def run_ours(args):
     tps = dist_util.whole_job_rate(tokens, world, ms_step)
     flops = cfg.step_flops()
     achieved_tf = flops / (ms_step * 1e-3) / 1e12
+    # which measured GEMM peak fits this run: the burst figure unless the run sat in the power-capped state
+    # the sustained figure was taken in (a timed region of a second or more AND the SM clock sampled low)
+    timed_mhz = clocks["timed"].get("sm_mhz")
+    burst = ms < BURST_REGION_MS or (timed_mhz is not None and timed_mhz >= BURST_MHZ)
+    regime = "burst" if burst else "sustained"
+    tensor_peak = peaks["bf16_tflops"] if burst else peaks["bf16_tflops_sustained"]
     kernels = {}
     total_ms = sum(v["ms"] for v in prof.values()) or 1.0
     for name, v in prof.items():
@@ -356,26 +425,39 @@ def run_ours(args):
         ent = {"launches_per_step": v["launches"] / prof_steps, "ms_per_step": v["ms"] / prof_steps,
                "share": v["ms"] / total_ms, "avg_launch_ms": per}
         if v["flops"] > 0:
-            ent.update(bound="tensor", achieved=v["flops"] / (v["ms"] * 1e-3) / 1e12, unit="TFLOP/s")
-            ent["frac"] = ent["achieved"] / peaks["bf16_tflops_sustained"]
+            ach = v["flops"] / (v["ms"] * 1e-3) / 1e12
+            ent.update(bound="tensor", achieved=ach, unit="TFLOP/s", frac=ach / tensor_peak,
+                       frac_burst=ach / peaks["bf16_tflops"], frac_sustained=ach / peaks["bf16_tflops_sustained"])
         else:
             ent.update(bound="hbm", achieved=v["bytes"] / (v["ms"] * 1e-3) / 1e9, unit="GB/s")
             ent["frac"] = ent["achieved"] / peaks["hbm_gbs"]
         kernels[name] = ent
     top = max(kernels, key=lambda k: kernels[k]["ms_per_step"])
     tk = kernels[top]
-    # DRAM bytes (read + written) per launch of the dominant kernel, from one ncu capture of this very
-    # command line (profiles/gemm_dram_traffic_block_step_C3.md); None where no capture of the current
-    # kernels exists for the workload
-    traffic = GEMM_DRAM_BYTES_PER_LAUNCH.get(cfg.name) if top == "gemm_tcgen05" and not args.recompute else None
+    traffic = stored_gemm_traffic(cfg.name) if top == "gemm_tcgen05" and not args.recompute else None
     roofline = {"kernel": top, "bound": tk["bound"], "achieved": tk["achieved"],
-                "peak": peaks["bf16_tflops_sustained"] if tk["bound"] == "tensor" else peaks["hbm_gbs"],
+                "peak": tensor_peak if tk["bound"] == "tensor" else peaks["hbm_gbs"],
                 "unit": tk["unit"], "frac": tk["frac"], "traffic": traffic,
-                "peak_source": f"{peaks_kind} ({'sustained bf16 GEMM' if tk['bound'] == 'tensor' else 'copy'})",
+                "peak_source": (f"{peaks_kind} ({regime} bf16 GEMM: burst when the timed region is under "
+                                f"{BURST_REGION_MS:.0f} ms or the SM clock sampled in it is at least {BURST_MHZ:.0f} MHz, "
+                                f"sustained otherwise)" if tk["bound"] == "tensor" else f"{peaks_kind} (copy)"),
                 "per_launch": {"avg_ms": tk["avg_launch_ms"],
                                "algorithmic": (prof[top]["flops"] or prof[top]["bytes"]) / prof[top]["launches"]}}
+    if tk["bound"] == "tensor":
+        roofline.update(frac_burst=tk["frac_burst"], frac_sustained=tk["frac_sustained"], regime=regime)
+    # where the step's time is: the step as timed, the per-kernel events of the profile pass (AdamW not
+    # overlapped there) and the phase calls, each with the SM clock sampled while it ran
+    sum_kernels = total_ms / prof_steps
+    mhz = {k: c.get("sm_mhz") for k, c in clocks.items()}
+    accounting = {"step_ms": ms_step, "sum_kernels_ms": sum_kernels, "sum_phases_ms": sum_phases, "sm_mhz": mhz,
+                  "step_minus_kernels_ms": ms_step - sum_kernels,
+                  "sum_kernels_ms_at_timed_clock": (sum_kernels * mhz["profile"] / mhz["timed"]
+                                                    if mhz.get("profile") and mhz.get("timed") else None),
+                  "note": "the profile pass runs a few steps from idle at a higher clock than the timed region; "
+                          "sum_kernels_ms_at_timed_clock rescales it by the sampled clocks (tensor kernels follow "
+                          "the SM clock, HBM-bound ones do not)"}
 
-    cpu_val, cores, what = oracle_sample(cfg, SAMPLE_TOKENS[cfg.name])
+    cpu_sec, cores, what, extrap, factors = oracle_step_seconds(cfg)
 
     line = {
         "metric": METRIC, "value": tps, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -388,13 +470,15 @@ def run_ours(args):
                    if cfg.n_params * 2 > 200e6 else "working set is L2-resident (small parity config)"},
         "mfu": {"step_flops": flops, "achieved_tflops": achieved_tf,
                 "vs_nominal_2250": achieved_tf / NOMINAL_BF16_TFLOPS,
-                "vs_measured_sustained": achieved_tf / peaks["bf16_tflops_sustained"],
+                "vs_measured_burst": achieved_tf / peaks["bf16_tflops"],
+                "vs_measured_sustained": achieved_tf / peaks["bf16_tflops_sustained"], "regime": regime,
                 "flops_convention": "6*matmul_params*tokens + causal-halved attention (6*B*T^2*d per layer)"},
-        "roofline": roofline, "kernels": kernels, "phases": phases,
-        "cpu_baseline": {"value": cpu_val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what},
+        "roofline": roofline, "kernels": kernels, "phases": phases, "accounting": accounting,
+        "cpu_baseline": {"value": cfg.tokens / cpu_sec, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what,
+                         "extrapolated": extrap, "extrapolation_factors": factors, "seconds_per_step": cpu_sec},
         "e2e": {"value": dist_util.whole_job_rate(tokens, world, ms_e2e / e2e_steps), "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
-        "gpu_launches": launches, "clocks": clocks,
+        "gpu_launches": launches, "clocks": clocks["timed"], "clocks_by_pass": clocks,
     }
     print(json.dumps(line), flush=True)
     sess.close()

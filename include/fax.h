@@ -244,7 +244,12 @@ typedef struct {
 } fax_block_state;
 
 /* One whole training step of a single block: forward, backward (gradients
- * overwritten), AdamW on the twelve tensors.  x, dy in; y, dx out (device). */
+ * overwritten), AdamW on the twelve tensors.  x, dy in; y, dx out (device).
+ * Backward reads x in place, so afterwards the saved arena holds this step's
+ * activations but no copy of x (it does when dx == x); a later
+ * fax_block_backward on that arena needs a fax_block_forward first.
+ * hp is checked before anything is enqueued (step >= 1, betas in [0, 1), lr
+ * and eps finite, eps >= 0): FAX_ERR_INVALID_ARG otherwise, on every call. */
 fax_status fax_block_step(fax_ctx* ctx, const fax_block_cfg* cfg, const fax_block_state* st,
                           const void* x, const void* dy, void* y, void* dx,
                           const fax_adamw_hparams* hp);

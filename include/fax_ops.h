@@ -31,8 +31,12 @@ enum {
  * B is [N,K] row-major (b_mn_major = 0) or [K,N] row-major (b_mn_major = 1);
  * lda / ldb / ldc / ldr / ldaux are row strides in elements.  C is T, or
  * float when c_f32 != 0; accumulate != 0 adds into a float C.  bias [N],
- * resid [M,N] and aux [M,N] are T.  force_simt != 0 selects the plain
- * float-FMA kernel even where the tensor-core kernel applies. */
+ * resid [M,N] and aux [M,N] are T.  In FAX_PREC_BF16 the problem runs on the
+ * tensor-core kernels (M a multiple of 128, N and K of 64, 16-byte aligned rows)
+ * and any other shape is refused with FAX_ERR_UNSUPPORTED_SHAPE: it never lands
+ * on the far slower float-FMA kernel unasked.  force_simt != 0 selects that
+ * kernel, for any shape and in either precision (FAX_PREC_FP32_VALIDATE always
+ * uses it). */
 typedef struct {
   int32_t M, N, K;
   const void* A; int64_t lda; int32_t a_mn_major;

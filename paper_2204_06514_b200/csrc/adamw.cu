@@ -125,8 +125,7 @@ void fax_adamw_scalars(const fax_adamw_hparams* hp, void* out32) {
 
 fax_status fax_adamw_launch(fax_ctx* ctx, const fax_adamw_tensor* tensors, int n, const fax_adamw_hparams* hp) {
   if (!tensors || !hp || n < 0) return FAX_ERR_INVALID_ARG;
-  if (hp->step < 1 || !(hp->beta1 >= 0.f && hp->beta1 < 1.f) || !(hp->beta2 >= 0.f && hp->beta2 < 1.f))
-    return FAX_ERR_INVALID_ARG;
+  FAX_TRY(fax_adamw_check_hparams(hp));
   AdamScalars sc = make_scalars(hp);
   for (int i = 0; i < n; ++i) {
     const fax_adamw_tensor& t = tensors[i];

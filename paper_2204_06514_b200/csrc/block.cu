@@ -351,14 +351,17 @@ static fax_status block_step_impl(fax_ctx* ctx, const fax_block_cfg* cfg, const 
     FAX_CUDA_TRY(ctx, cudaMemcpyAsync(io->dy_dev, io->dy_host, io->bytes, cudaMemcpyHostToDevice, ctx->copy));
     FAX_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_copy_b, ctx->copy));
   }
-  FAX_TRY(fax_block_forward_impl(ctx, cfg, &p, x, y, s, true, &w));
+  // the caller's x stays valid through the step, so backward reads it in place and the saved arena gets
+  // no copy of it (unless dx is to overwrite x)
+  const bool copy_x = (x == dx);
+  FAX_TRY(fax_block_forward_impl(ctx, cfg, &p, x, y, s, copy_x, &w));
   if (io) {
     FAX_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_copy_a, ctx->stream));              // y is complete
     FAX_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->copy, ctx->ev_copy_a, 0));
     FAX_CUDA_TRY(ctx, cudaMemcpyAsync(io->y_host, y, io->bytes, cudaMemcpyDeviceToHost, ctx->copy));
     FAX_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->stream, ctx->ev_copy_b, 0));       // dY has arrived
   }
-  FAX_TRY(fax_block_backward_impl(ctx, cfg, &p, dy, s, s.x, dx, &g, false, w, &hook));
+  FAX_TRY(fax_block_backward_impl(ctx, cfg, &p, dy, s, copy_x ? s.x : x, dx, &g, false, w, &hook));
   return fax_adamw_join(ctx);
 }
 
@@ -368,13 +371,14 @@ extern "C" fax_status fax_block_step(fax_ctx* ctx, const fax_block_cfg* cfg, con
   if (!ctx || !st || !x || !dy || !y || !dx || !hp || !st->saved || !st->scratch || x == y) return FAX_ERR_INVALID_ARG;
   FAX_TRY(fax_block_validate(cfg));
   FAX_TRY(fax_layer_check(&st->layer, cfg));
-  if (hp->step < 1) return FAX_ERR_INVALID_ARG;
-  uint64_t key = fax_hash(FAX_HASH_SEED, 'B');
-  key = fax_hash(key, *cfg);
-  key = fax_hash_layer(key, &st->layer);
-  key = fax_hash(key, st->saved); key = fax_hash(key, st->saved_bytes);
-  key = fax_hash(key, st->scratch); key = fax_hash(key, st->scratch_bytes);
-  key = fax_hash(key, x); key = fax_hash(key, dy); key = fax_hash(key, y); key = fax_hash(key, dx);
+  FAX_TRY(fax_adamw_check_hparams(hp));
+  FaxStepKey key;
+  key.add('B');
+  key.add(*cfg);
+  key.add_layer(&st->layer);
+  key.add(st->saved); key.add(st->saved_bytes);
+  key.add(st->scratch); key.add(st->scratch_bytes);
+  key.add(x); key.add(dy); key.add(y); key.add(dx);
   return fax_run_step(ctx, key, hp, [&]() { return block_step_impl(ctx, cfg, st, x, dy, y, dx, hp, 0); });
 }
 
@@ -391,6 +395,7 @@ extern "C" fax_status fax_block_step_host(fax_ctx* ctx, const fax_block_cfg* cfg
                                           void* dx_host, const fax_adamw_hparams* hp) {
   if (!ctx || !st || !x_host || !dy_host || !y_host || !dx_host || !hp || !st->saved || !st->scratch)
     return FAX_ERR_INVALID_ARG;
+  FAX_TRY(fax_adamw_check_hparams(hp));
   FAX_TRY(fax_block_validate(cfg));
   FAX_TRY(fax_layer_check(&st->layer, cfg));
   const size_t bytes = (size_t)cfg->batch * cfg->seq * cfg->d_model * fax_elem_size(cfg->prec);

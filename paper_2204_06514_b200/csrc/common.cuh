@@ -28,6 +28,7 @@ struct FaxGemmPatch {
 struct FaxGraphEntry {
   std::vector<FaxGemmPatch> gemm_nodes;
   uint64_t key;
+  std::vector<unsigned char> material;   // the bytes the key was hashed from (compared on a hash hit)
   cudaGraph_t graph; cudaGraphExec_t exec;
   std::vector<cudaGraphNode_t> adam_nodes;
   std::vector<cudaKernelNodeParams> adam_params;
@@ -231,7 +232,9 @@ fax_status fax_gemm_tc(fax_ctx* ctx, const FaxGemm& g);       // bf16 tcgen05 pa
 bool fax_gemm_tc_supported(const FaxGemm& g);
 bool fax_gemm_tc2_supported(const FaxGemm& g);                 // two-CTA 256 x 256 tiles
 fax_status fax_gemm_tc2(fax_ctx* ctx, const FaxGemm& g);
-fax_status fax_gemm(fax_ctx* ctx, int prec, const FaxGemm& g); // dispatch
+// dispatch; allow_simt: a bf16 problem that the tensor-core kernels do not take may run on the SIMT kernel
+// (otherwise FAX_ERR_UNSUPPORTED_SHAPE); kernel_class (optional) receives KC_GEMM_TC or KC_GEMM_SIMT
+fax_status fax_gemm(fax_ctx* ctx, int prec, const FaxGemm& g, bool allow_simt = false, int* kernel_class = nullptr);
 // Would fax_gemm run this (bf16) problem on a tensor-core kernel without slicing K?  Only then
 // can AdamW be fused into its epilogue.
 bool fax_gemm_can_fuse_adam(fax_ctx* ctx, const FaxGemm& g);
@@ -263,6 +266,14 @@ fax_status fax_attention_bwd(fax_ctx* ctx, int prec, int B, int T, int H, int hd
                              void* scratch, size_t scratch_bytes);
 size_t fax_attention_bwd_scratch_bytes(int prec, int B, int T, int H, int hd);
 
+// step >= 1, both betas in [0, 1), lr and eps finite and eps >= 0.  Checked before anything of a step is
+// enqueued, on the direct path and on graph replay alike.
+static inline fax_status fax_adamw_check_hparams(const fax_adamw_hparams* hp) {
+  if (!hp || hp->step < 1) return FAX_ERR_INVALID_ARG;
+  if (!(hp->beta1 >= 0.f && hp->beta1 < 1.f) || !(hp->beta2 >= 0.f && hp->beta2 < 1.f)) return FAX_ERR_INVALID_ARG;
+  if (!(hp->lr == hp->lr) || !(hp->eps >= 0.f) || hp->lr - hp->lr != 0.f || hp->eps - hp->eps != 0.f) return FAX_ERR_INVALID_ARG;
+  return FAX_OK;
+}
 fax_status fax_adamw_launch(fax_ctx* ctx, const fax_adamw_tensor* tensors, int n, const fax_adamw_hparams* hp);
 // Enqueue AdamW on the context's optimizer stream, ordered after everything enqueued on the main
 // stream so far; fax_adamw_join makes the main stream wait for all of it.

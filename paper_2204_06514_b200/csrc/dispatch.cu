@@ -1,9 +1,17 @@
 // Operator dispatch between the tensor-core kernels and the SIMT kernels.
 #include "common.cuh"
 
-fax_status fax_gemm(fax_ctx* ctx, int prec, const FaxGemm& g) {
-  if (prec == FAX_PREC_BF16 && fax_gemm_tc_supported(g)) return fax_gemm_tc(ctx, g);
+// bf16 problems run on the tensor cores or not at all, unless the caller has allowed the SIMT
+// kernel for them: a shape the tensor-core kernels reject would otherwise run one to two orders of
+// magnitude slower with nothing telling the caller.
+fax_status fax_gemm(fax_ctx* ctx, int prec, const FaxGemm& g, bool allow_simt, int* kernel_class) {
+  if (prec == FAX_PREC_BF16 && fax_gemm_tc_supported(g)) {
+    if (kernel_class) *kernel_class = KC_GEMM_TC;
+    return fax_gemm_tc(ctx, g);
+  }
   if (g.adam) return FAX_ERR_INVALID_ARG;               // callers ask fax_gemm_can_fuse_adam first
+  if (prec == FAX_PREC_BF16 && !allow_simt) return FAX_ERR_UNSUPPORTED_SHAPE;
+  if (kernel_class) *kernel_class = KC_GEMM_SIMT;
   return fax_gemm_simt(ctx, prec, g);
 }
 

@@ -44,11 +44,11 @@ static fax_status patch_and_launch(fax_ctx* ctx, FaxGraphEntry& e, const fax_ada
   return FAX_OK;
 }
 
-fax_status fax_run_step(fax_ctx* ctx, uint64_t key, const fax_adamw_hparams* hp,
+fax_status fax_run_step(fax_ctx* ctx, const FaxStepKey& key, const fax_adamw_hparams* hp,
                         const std::function<fax_status()>& enqueue) {
   if (!ctx->use_graphs || ctx->prof_on || !hp) return enqueue();
   for (FaxGraphEntry& e : ctx->graphs)
-    if (e.key == key) {
+    if (e.key == key.hash && e.material == key.material) {
       if (e.exec) return patch_and_launch(ctx, e, hp);
       if (e.failed) return enqueue();
       // second request with this key: capture
@@ -109,7 +109,7 @@ fax_status fax_run_step(fax_ctx* ctx, uint64_t key, const fax_adamw_hparams* hp,
     ctx->graphs.erase(ctx->graphs.begin() + victim);
   }
   FaxGraphEntry e;
-  e.key = key; e.graph = nullptr; e.exec = nullptr; e.failed = false; e.launches = 0; e.last_use = ++ctx->graph_clock;
+  e.key = key.hash; e.material = key.material; e.graph = nullptr; e.exec = nullptr; e.failed = false; e.launches = 0; e.last_use = ++ctx->graph_clock;
   ctx->graphs.push_back(e);
   return enqueue();
 }

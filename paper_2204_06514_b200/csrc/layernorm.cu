@@ -676,7 +676,9 @@ size_t fax_layernorm_bwd_partial_floats(int rows, int d) {
 fax_status fax_layernorm_fwd(fax_ctx* ctx, int prec, int rows, int d, const void* x, const void* gamma,
                              const void* beta, float eps, void* out, float* mu, float* rstd, void* x_copy) {
   // read x, write out (and the optional copy of x)
-  FaxProfScope prof(ctx, KC_LN_FWD, 0.0, (double)rows * d * fax_elem_size(prec) * (x_copy ? 3 : 2));
+  // algorithmic bytes: read x, write the normalised rows (a copy of x kept for backward, where a caller
+  // asks for one, is extra traffic and not counted)
+  FaxProfScope prof(ctx, KC_LN_FWD, 0.0, (double)rows * d * fax_elem_size(prec) * 2);
   if (prec == FAX_PREC_BF16) {
     if (d % 8) return FAX_ERR_UNSUPPORTED_SHAPE;
     return ln_fwd_t<bf16>(ctx, rows, d, x, gamma, beta, eps, out, mu, rstd, x_copy);

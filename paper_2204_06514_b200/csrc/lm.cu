@@ -259,7 +259,8 @@ extern "C" fax_status fax_lm_accumulate(fax_ctx* ctx, const fax_lm_cfg* cfg, con
 
 extern "C" fax_status fax_lm_apply_adamw(fax_ctx* ctx, const fax_lm_cfg* cfg, const fax_lm_state* st,
                                          const fax_adamw_hparams* hp) {
-  if (!ctx || !hp || hp->step < 1) return FAX_ERR_INVALID_ARG;
+  if (!ctx || !hp) return FAX_ERR_INVALID_ARG;
+  FAX_TRY(fax_adamw_check_hparams(hp));
   FAX_TRY(lm_validate(cfg));
   FAX_TRY(lm_check_state(cfg, st));
   fax_adamw_hparams h = *hp;
@@ -278,14 +279,16 @@ extern "C" fax_status fax_lm_step(fax_ctx* ctx, const fax_lm_cfg* cfg, const fax
                                   float* loss_device, float* loss_host) {
   if (!ctx || !ids || !targets || !hp || !cfg || !st) return FAX_ERR_INVALID_ARG;
   if (hp->step < 1 || cfg->n_layers <= 0 || !st->layers) return FAX_ERR_INVALID_ARG;
-  uint64_t key = fax_hash(FAX_HASH_SEED, 'L');
-  key = fax_hash(key, *cfg);
-  key = fax_hash_param(key, st->wte); key = fax_hash_param(key, st->wpe);
-  key = fax_hash_param(key, st->lnf_g); key = fax_hash_param(key, st->lnf_b);
-  for (int l = 0; l < cfg->n_layers; ++l) key = fax_hash_layer(key, &st->layers[l]);
-  key = fax_hash(key, st->saved); key = fax_hash(key, st->saved_bytes);
-  key = fax_hash(key, st->scratch); key = fax_hash(key, st->scratch_bytes);
-  key = fax_hash(key, ids); key = fax_hash(key, targets); key = fax_hash(key, loss_device);
+  FAX_TRY(fax_adamw_check_hparams(hp));
+  FaxStepKey key;
+  key.add('L');
+  key.add(*cfg);
+  key.add_param(st->wte); key.add_param(st->wpe);
+  key.add_param(st->lnf_g); key.add_param(st->lnf_b);
+  for (int l = 0; l < cfg->n_layers; ++l) key.add_layer(&st->layers[l]);
+  key.add(st->saved); key.add(st->saved_bytes);
+  key.add(st->scratch); key.add(st->scratch_bytes);
+  key.add(ids); key.add(targets); key.add(loss_device);
   FAX_TRY(fax_run_step(ctx, key, hp, [&]() { return lm_run(ctx, cfg, st, ids, targets, hp, loss_device, nullptr, nullptr); }));
   if (loss_host) {
     FAX_CUDA_TRY(ctx, cudaMemcpyAsync(loss_host, loss_device, sizeof(float), cudaMemcpyDeviceToHost, ctx->stream));
@@ -298,6 +301,7 @@ extern "C" fax_status fax_lm_step_host(fax_ctx* ctx, const fax_lm_cfg* cfg, cons
                                        const int32_t* ids_host, const int32_t* targets_host,
                                        const fax_adamw_hparams* hp, float* loss_device, float* loss_host) {
   if (!ctx || !ids_host || !targets_host || !hp || !loss_host) return FAX_ERR_INVALID_ARG;
+  FAX_TRY(fax_adamw_check_hparams(hp));
   FAX_TRY(lm_run(ctx, cfg, st, nullptr, nullptr, hp, loss_device, ids_host, targets_host));
   FAX_CUDA_TRY(ctx, cudaMemcpyAsync(loss_host, loss_device, sizeof(float), cudaMemcpyDeviceToHost, ctx->stream));
   FAX_CUDA_TRY(ctx, cudaStreamSynchronize(ctx->stream));

@@ -451,6 +451,21 @@ def test_lm_and_adamw_error_paths(sess):
     r.step(tids, ttg, hparams(step=1, **hp))
     st, _ = fx.fax_check_device_status(sess.ctx)
     assert st == fx.FAX_OK and torch.isfinite(r.loss).all()
+    # once the step is replayed from a graph (third call on) bad hyper-parameters are still refused,
+    # before anything is enqueued: the weights stay as they are and finite
+    for s in (2, 3, 4):
+        r.step(tids, ttg, hparams(step=s, **hp))
+    torch.cuda.synchronize()
+    before = r.wte.w.clone()
+    for bad_hp in (dict(hp, beta1=1.0), dict(hp, beta2=-0.1), dict(hp, lr=float("nan")), dict(hp, eps=float("inf"))):
+        with pytest.raises(fx.FaxError) as e:
+            r.step(tids, ttg, hparams(step=5, **bad_hp))
+        assert e.value.status == fx.FAX_ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    assert torch.equal(before, r.wte.w) and torch.isfinite(r.wte.w).all()
+    r.step(tids, ttg, hparams(step=5, **hp))
+    torch.cuda.synchronize()
+    assert torch.isfinite(r.wte.w).all() and not torch.equal(before, r.wte.w)
 
 
 @pytest.mark.parametrize("prec", [fx.FAX_PREC_FP32_VALIDATE, fx.FAX_PREC_BF16])

@@ -119,6 +119,12 @@ def test_gemm_layouts(sess, prec, a_mn, b_mn, shape, force_simt):
     tC = torch.empty((M, N), dtype=dt, device=sess.device)
     desc = ops.GemmDesc(M, N, K, ptr(tA), M if a_mn else K, a_mn, ptr(tB), N if b_mn else K, b_mn,
                         ptr(tC), N, 0, 0, ops.FAX_EPI_NONE, None, None, 0, None, 0, 1.0, force_simt)
+    if prec == 0 and not force_simt and (M % 128 or N % 64 or K % 64):
+        # a bf16 shape the tensor-core kernels do not take is refused, never run on the SIMT kernel unasked
+        with pytest.raises(fx.FaxError) as e:
+            ops.fax_op_gemm(sess.ctx, prec, desc)
+        assert e.value.status == fx.FAX_ERR_UNSUPPORTED_SHAPE
+        return
     ops.fax_op_gemm(sess.ctx, prec, desc)
     st, detail = fx.fax_check_device_status(sess.ctx)
     assert st == fx.FAX_OK, detail
@@ -187,6 +193,99 @@ def test_gemm_weight_gradient_shapes_split_k(sess, M, N, K, accumulate):
     assert st == fx.FAX_OK, detail
 
 
+def _step_gemm_shapes(cfg):
+    """The twelve contractions of one block step at a config's full size:
+    (name, M, N, K, a_mn, b_mn, epilogue, float output)."""
+    n, d, f = cfg.tokens, cfg.d_model, cfg.d_ff
+    E = ops
+    return [
+        ("qkv", n, 3 * d, d, 0, 1, E.FAX_EPI_BIAS, 0), ("out_proj", n, d, d, 0, 1, E.FAX_EPI_BIAS_RESID, 0),
+        ("fc1", n, f, d, 0, 1, E.FAX_EPI_BIAS_GELU, 0), ("fc2", n, d, f, 0, 1, E.FAX_EPI_BIAS_RESID, 0),
+        ("fc2_dx", n, f, d, 0, 0, E.FAX_EPI_DGELU, 0), ("fc1_dx", n, d, f, 0, 0, E.FAX_EPI_NONE, 0),
+        ("out_proj_dx", n, d, d, 0, 0, E.FAX_EPI_NONE, 0), ("qkv_dx", n, d, 3 * d, 0, 0, E.FAX_EPI_NONE, 0),
+        ("fc2_dw", f, d, n, 1, 1, E.FAX_EPI_NONE, 1), ("fc1_dw", d, f, n, 1, 1, E.FAX_EPI_NONE, 1),
+        ("out_proj_dw", d, d, n, 1, 1, E.FAX_EPI_NONE, 1), ("qkv_dw", d, 3 * d, n, 1, 1, E.FAX_EPI_NONE, 1),
+    ]
+
+
+@pytest.mark.parametrize("name", ["C3", "C5"])
+def test_gemm_full_size_sampled(sess, name):
+    """Dense seeded data through every GEMM shape of a full-size block step (forward, dX with the
+    transposed weight, dW with the long token contraction, all fused epilogues): sampled output rows,
+    all their columns, against float64.  A K block skipped or read twice, or a tile written to the
+    wrong place, shows up here; the full-size block tests feed the dW products mostly zeros."""
+    cfg = synth.CONFIGS[name]
+    rng = np.random.default_rng(cfg.seed + 4242)
+    bf = torch.bfloat16
+    cache = {}
+
+    def operand(rows, cols, scale):
+        # one bf16 matrix per (rows, cols): weights are reused by the forward and the dX product
+        key = (rows, cols)
+        if key not in cache:
+            a = synth.round_to_bf16(rng.standard_normal((rows, cols), dtype=np.float32) * np.float32(scale))
+            cache[key] = (a, dev(a, bf, sess))
+        return cache[key]
+
+    for gname, M, N, K, a_mn, b_mn, epi, c_f32 in _step_gemm_shapes(cfg):
+        A, tA = operand(K, M, 1.0) if a_mn else operand(M, K, 1.0)
+        B, tB = operand(K, N, K ** -0.5) if b_mn else operand(N, K, K ** -0.5)
+        rows = np.sort(rng.choice(M, size=96, replace=False))
+        bias = synth.round_to_bf16(rng.standard_normal(N).astype(np.float32))
+        extra = synth.round_to_bf16(rng.standard_normal((M, N), dtype=np.float32))      # residual or pre-activation
+        tbias, textra = dev(bias, bf, sess), dev(extra, bf, sess)
+        tC = torch.empty((M, N), dtype=torch.float32 if c_f32 else bf, device=sess.device)
+        taux = torch.empty((M, N), dtype=bf, device=sess.device) if epi == ops.FAX_EPI_BIAS_GELU else textra
+        desc = ops.GemmDesc(M, N, K, ptr(tA), M if a_mn else K, a_mn, ptr(tB), N if b_mn else K, b_mn, ptr(tC), N,
+                            c_f32, 0, epi, ptr(tbias), ptr(textra), N, ptr(taux), N, 1.0, 0)
+        ops.fax_op_gemm(sess.ctx, 0, desc)
+        a_rows = (A[:, rows].T if a_mn else A[rows]).astype(np.float64)
+        acc = a_rows @ (B.astype(np.float64) if b_mn else B.astype(np.float64).T)
+        if epi == ops.FAX_EPI_BIAS:
+            ref = acc + bias
+        elif epi == ops.FAX_EPI_BIAS_RESID:
+            ref = acc + bias + extra[rows]
+        elif epi == ops.FAX_EPI_BIAS_GELU:
+            ref = acc + bias
+            g = taux[torch.as_tensor(rows, device=sess.device)]
+            assert relerr(host(g), O.gelu_tanh(ref)) <= TOL_FWD_BF16, (gname, "gelu")
+        elif epi == ops.FAX_EPI_DGELU:
+            ref = acc * O.gelu_tanh_grad(extra[rows])
+        else:
+            ref = acc
+        got = host(tC[torch.as_tensor(rows, device=sess.device)])
+        assert relerr(got, ref) <= (1e-5 if c_f32 else TOL_FWD_BF16), gname
+        del tC, tbias, textra, taux
+    st, detail = fx.fax_check_device_status(sess.ctx)
+    assert st == fx.FAX_OK, detail
+
+
+def test_gemm_two_cta_accumulators_recycled_many_times(sess):
+    """Far more 256 x 256 tiles than SM pairs with a single K block each: the next tile's product is
+    issued the moment an accumulator is handed back, so a hand-back that came before the epilogue had
+    read the accumulator would corrupt tiles.  Tile-dependent data; compared bit for bit with the
+    one-CTA kernel and against float64."""
+    M, N, K = 256 * 40, 256 * 12, 64                       # 480 tiles for 74 SM pairs
+    rng = np.random.default_rng(2026)
+    A = synth.round_to_bf16(rng.standard_normal((M, K), dtype=np.float32) * (1 + np.arange(M, dtype=np.float32)[:, None] % 7))
+    B = synth.round_to_bf16(rng.standard_normal((N, K), dtype=np.float32))
+    tA, tB = dev(A, torch.bfloat16, sess), dev(B, torch.bfloat16, sess)
+    outs = []
+    for two_cta in (1, 0):
+        fx.fax_set_gemm_two_cta(sess.ctx, two_cta)
+        tC = torch.zeros((M, N), dtype=torch.bfloat16, device=sess.device)
+        desc = ops.GemmDesc(M, N, K, ptr(tA), K, 0, ptr(tB), K, 0, ptr(tC), N, 0, 0, ops.FAX_EPI_NONE,
+                            None, None, 0, None, 0, 1.0, 0)
+        for _ in range(3):
+            ops.fax_op_gemm(sess.ctx, 0, desc)
+        outs.append(tC)
+    fx.fax_set_gemm_two_cta(sess.ctx, 1)
+    assert torch.equal(outs[0], outs[1])
+    assert relerr(host(outs[0]), A.astype(np.float64) @ B.astype(np.float64).T) <= TOL_FWD_BF16
+    st, detail = fx.fax_check_device_status(sess.ctx)
+    assert st == fx.FAX_OK, detail
+
+
 # T a multiple of 256 takes the two-tile persistent forward kernel; the last two bf16 shapes give it more
 # work items than the GPU has SMs, so CTAs loop over several query-tile pairs
 ATTN_SHAPES = [(0, 2, 128, 4, 64), (0, 1, 128, 1, 128), (0, 1, 384, 2, 128), (0, 2, 1024, 2, 64), (0, 1, 2048, 1, 128),
@@ -221,5 +320,36 @@ def test_attention_forward_backward(sess, prec, B, T, H, hd):
     got = host(dqkv)
     for i, name in enumerate("qkv"):
         assert relerr(got[:, i * d:(i + 1) * d], rd[:, i * d:(i + 1) * d]) <= tolg, name
+    st, _ = fx.fax_check_device_status(sess.ctx)
+    assert st == fx.FAX_OK
+
+
+def test_attention_backward_kernels_agree(sess):
+    """head_dim 128 has two backward kernels (half-tile hand-offs, and the older single hand-off one
+    that also serves head_dim 64): the same inputs through both, each against the oracle."""
+    B, T, H, hd = 2, 640, 5, 128
+    rng = np.random.default_rng(77)
+    d = H * hd
+    qkv = synth.round_to_bf16(rng.standard_normal((B * T, 3 * d)).astype(np.float32))
+    do = synth.round_to_bf16(rng.standard_normal((B * T, d)).astype(np.float32))
+    tq, tdo = dev(qkv, torch.bfloat16, sess), dev(do, torch.bfloat16, sess)
+    o = torch.empty((B * T, d), dtype=torch.bfloat16, device=sess.device)
+    lse = torch.empty((B, H, T), dtype=torch.float32, device=sess.device)
+    ops.fax_op_attention_forward(sess.ctx, 0, B, T, H, hd, ptr(tq), ptr(o), ptr(lse))
+    ro, rlse, _ = O.attention_fwd(qkv, B, T, H, hd)
+    rd = O.attention_bwd(do, qkv, ro, rlse, B, T, H, hd)
+    nb = ops.fax_op_attention_backward_scratch_bytes(0, B, T, H, hd)
+    scratch = sess.arena(nb)
+    try:
+        for enable in (1, 0):
+            fx.fax_set_attention_backward_two_chains(sess.ctx, enable)
+            dqkv = torch.full_like(tq, float("nan"))
+            ops.fax_op_attention_backward(sess.ctx, 0, B, T, H, hd, ptr(tq), ptr(o), ptr(lse), ptr(tdo), ptr(dqkv),
+                                          ptr(scratch), nb)
+            got = host(dqkv)
+            for i, name in enumerate("qkv"):
+                assert relerr(got[:, i * d:(i + 1) * d], rd[:, i * d:(i + 1) * d]) <= TOL_GRAD_BF16, (enable, name)
+    finally:
+        fx.fax_set_attention_backward_two_chains(sess.ctx, 1)
     st, _ = fx.fax_check_device_status(sess.ctx)
     assert st == fx.FAX_OK

@@ -399,5 +399,7 @@ def test_paper_numbers_golden():
     c4 = synth.CONFIGS["C4"]
     assert c4.n_params == 124_475_904
     assert c4.n_params // 10 ** 6 == vals["fig3_model_params_millions"]
+    f3 = synth.CONFIGS["F3"]                 # Fig. 3's workload: the same 124M model at the caption's sequence length
+    assert f3.seq == vals["fig3_seq_len"] and f3.n_params - c4.n_params == (f3.seq - c4.seq) * f3.d_model
     c5 = synth.CONFIGS["C5"]
     assert c5.seq == vals["table1_seq_len"] and c5.batch == vals["table1_batch"]
