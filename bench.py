@@ -6,8 +6,11 @@
 Prints ONE JSON line.  `value` = training tokens/s of the whole job with the
 inputs resident in HBM; `e2e` = the same through the host-buffer entry point
 (host->device copies of the step's inputs and device->host read of its results
-inside the timed region).  N > 1 runs N independent replicas (one process per
-GPU, no data-path collective): the step has no exchange step on one device.
+inside the timed region).  N > 1: block workloads (C1-C3, C5, P*), whose inputs
+are activations, run as N independent replicas (one process per GPU, no
+data-path collective, "scaling": "weak"); LM workloads (C4, F*) train
+data-parallel over the workload's batch ("strong": reduce-scatter of the
+gradients, AdamW on each rank's shard, all-gather of the bf16 weights).
 `--impl reference` times the fp64 CPU oracle instead.
 """
 from __future__ import annotations
@@ -286,7 +289,37 @@ def run_ours(args):
         return out
 
     step_no = [0]
-    if cfg.is_lm:
+    # LM workloads on several GPUs train data-parallel over the batch (the global batch is the workload's:
+    # strong scaling, one reduce-scatter and one all-gather per step); block workloads, whose inputs are
+    # activations, run as independent replicas
+    data_parallel = cfg.is_lm and world > 1
+    if data_parallel:
+        from paper_2204_06514_b200 import dp
+        gen.manual_seed(cfg.seed)                   # every rank starts from the same model and the same global batch
+        lm = dict(wte=rand((cfg.vocab, cfg.d_model), 0.02), wpe=rand((cfg.seq, cfg.d_model), 0.02),
+                  blocks=[block_params() for _ in range(cfg.n_layers)],
+                  lnf_g=torch.ones(cfg.d_model), lnf_b=torch.zeros(cfg.d_model))
+        lm = {k: ([{n: t.cpu().numpy() for n, t in b.items()} for b in v] if k == "blocks" else v.cpu().numpy())
+              for k, v in lm.items()}
+        runner = dp.DpLmRunner(sess, cfg, lm, weight_decay=wd, rank=rank, world=world)
+        raw = torch.randint(0, cfg.vocab, (cfg.batch, cfg.seq + 1), generator=gen, device=dev, dtype=torch.int32)
+        per = cfg.batch // world
+        ids = raw[rank * per:(rank + 1) * per, :-1].contiguous()
+        tg = raw[rank * per:(rank + 1) * per, 1:].contiguous()
+        ids_h, tg_h = ids.cpu().pin_memory(), tg.cpu().pin_memory()
+        h2d, d2h = 2 * ids_h.numel() * 4 * world, 4 * world
+
+        def step():
+            step_no[0] += 1
+            runner.step(ids, tg, hparams(step=step_no[0], **hp0))
+
+        def step_host():
+            step_no[0] += 1
+            ids.copy_(ids_h, non_blocking=True)
+            tg.copy_(tg_h, non_blocking=True)
+            runner.step(ids, tg, hparams(step=step_no[0], **hp0))
+            runner.loss.item()
+    elif cfg.is_lm:
         lm = dict(wte=rand((cfg.vocab, cfg.d_model), 0.02), wpe=rand((cfg.seq, cfg.d_model), 0.02),
                   blocks=[block_params() for _ in range(cfg.n_layers)],
                   lnf_g=torch.ones(cfg.d_model), lnf_b=torch.zeros(cfg.d_model))
@@ -386,7 +419,12 @@ def run_ours(args):
     # per-phase split (the paper's Fig. 3 reports forward, loss and backward separately): the phase
     # entry points timed on their own, outside the step's timed region
     ph_steps = max(1, min(args.steps, 5))
-    if cfg.is_lm:
+    if data_parallel:
+        fb = timed(lambda: runner.local_gradients(ids, tg), ph_steps, tag="phases") / ph_steps
+        phases = {"forward_loss_backward_ms": fb, "exchange_and_adamw_ms": max(ms / args.steps - fb, 0.0),
+                  "note": "local forward + loss + backward; the rest of the step is reduce-scatter, sharded AdamW, all-gather"}
+        sum_phases = None
+    elif cfg.is_lm:
         fb = timed(lambda: runner.forward_backward(ids, tg), ph_steps, tag="phases") / ph_steps
         phases = {"forward_loss_backward_ms": fb, "adamw_ms": max(ms / args.steps - fb, 0.0),
                   "note": "forward + loss + backward through fax_lm_forward_backward; AdamW = step - that"}
@@ -409,9 +447,9 @@ def run_ours(args):
 
     ms_step = ms / args.steps
     tokens = cfg.tokens
-    tps = dist_util.whole_job_rate(tokens, world, ms_step)
+    tps = tokens / (ms_step * 1e-3) if data_parallel else dist_util.whole_job_rate(tokens, world, ms_step)
     flops = cfg.step_flops()
-    achieved_tf = flops / (ms_step * 1e-3) / 1e12
+    achieved_tf = flops / (ms_step * 1e-3) / 1e12 / (world if data_parallel else 1)     # per GPU
     # which measured GEMM peak fits this run: the burst figure unless the run sat in the power-capped state
     # the sustained figure was taken in (a timed region of a second or more AND the SM clock sampled low)
     timed_mhz = clocks["timed"].get("sm_mhz")
@@ -463,10 +501,13 @@ def run_ours(args):
         "metric": METRIC, "value": tps, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step,
         "ms_step_median": sorted(step_marks)[len(step_marks) // 2], "ms_step_min": min(step_marks),
-        "higher_is_better": True, "scaling": "weak",
+        "higher_is_better": True, "scaling": "strong" if data_parallel else "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": workload_name(cfg), "tokens_per_step": tokens, "params": cfg.n_params,
-                   "replicas": world, "fused_update": args.fused_update, "recompute": bool(args.recompute), "l2": "working set per step far exceeds the 126 MB L2"
+                   "replicas": 1 if data_parallel else world,
+                   "parallelism": f"dp{world}: batch sharded, gradients reduce-scattered, AdamW on shards, bf16 weights all-gathered"
+                   if data_parallel else ("single GPU" if world == 1 else f"{world} independent replicas"),
+                   "fused_update": args.fused_update, "recompute": bool(args.recompute), "l2": "working set per step far exceeds the 126 MB L2"
                    if cfg.n_params * 2 > 200e6 else "working set is L2-resident (small parity config)"},
         "mfu": {"step_flops": flops, "achieved_tflops": achieved_tf,
                 "vs_nominal_2250": achieved_tf / NOMINAL_BF16_TFLOPS,
@@ -476,7 +517,8 @@ def run_ours(args):
         "roofline": roofline, "kernels": kernels, "phases": phases, "accounting": accounting,
         "cpu_baseline": {"value": cfg.tokens / cpu_sec, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": what,
                          "extrapolated": extrap, "extrapolation_factors": factors, "seconds_per_step": cpu_sec},
-        "e2e": {"value": dist_util.whole_job_rate(tokens, world, ms_e2e / e2e_steps), "unit": UNIT,
+        "e2e": {"value": (tokens / (ms_e2e / e2e_steps * 1e-3) if data_parallel
+                          else dist_util.whole_job_rate(tokens, world, ms_e2e / e2e_steps)), "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": launches, "clocks": clocks["timed"], "clocks_by_pass": clocks,
     }

@@ -217,6 +217,14 @@ fax_status fax_set_gemm_two_cta(fax_ctx* ctx, int32_t enable);
  * enable = 0 launches every kernel fully serialised.  Default: enabled. */
 fax_status fax_set_dependent_launch(fax_ctx* ctx, int32_t enable);
 
+/* Tile order of the GEMMs.  The output tiles are visited in groups that keep
+ * one operand's panels (a tile's rows or columns over all of K) in L2 from one
+ * wave of tiles to the next while the other operand streams past once per
+ * group; the group is as large as `bytes` of L2 allow, along the dimension
+ * that costs fewer DRAM reads.  bytes = 0 restores the fixed order (groups of
+ * 8 row-tiles).  Results are bit-identical for every value.  Default: 48e6. */
+fax_status fax_set_gemm_l2_budget(fax_ctx* ctx, int64_t bytes);
+
 /* Attention backward at head_dim 128 walks the queries of a key tile in
  * sub-tiles of 64 with two of them in flight (the row warps work on one while
  * the tensor cores run the other's products); enable = 0 keeps the kernel with

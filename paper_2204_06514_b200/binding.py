@@ -98,6 +98,7 @@ _SIGNATURES = {
     "fax_set_dependent_launch": (C.c_int32, [_P, C.c_int32]),
     "fax_set_graph_replay": (C.c_int32, [_P, C.c_int32]),
     "fax_set_attention_backward_two_chains": (C.c_int32, [_P, C.c_int32]),
+    "fax_set_gemm_l2_budget": (C.c_int32, [_P, C.c_int64]),
     "fax_set_fused_update": (C.c_int32, [_P, C.c_int32, C.c_int32]),
     "fax_profile_begin": (C.c_int32, [_P]),
     "fax_profile_end": (C.c_int32, [_P, C.POINTER(ProfileEntry), C.c_int32]),
@@ -208,6 +209,10 @@ def fax_set_gemm_two_cta(ctx, enable: bool):
 
 def fax_set_dependent_launch(ctx, enable: bool):
     _check(load_library().fax_set_dependent_launch(ctx, int(bool(enable))), "fax_set_dependent_launch")
+
+
+def fax_set_gemm_l2_budget(ctx, nbytes: int):
+    _check(load_library().fax_set_gemm_l2_budget(ctx, int(nbytes)), "fax_set_gemm_l2_budget")
 
 
 def fax_set_attention_backward_two_chains(ctx, enable: bool):

@@ -41,6 +41,7 @@ extern "C" fax_status fax_create(fax_ctx** out, int32_t device_ordinal, void* cu
   c->use_2cta = true;
   c->use_pdl = true;
   c->attn_bwd_two_chains = true;
+  c->gemm_l2_budget = 48e6;
   c->use_graphs = true;
   c->fused_update = false;
   c->keep_fused_grads = false;
@@ -142,6 +143,14 @@ extern "C" fax_status fax_set_gemm_two_cta(fax_ctx* ctx, int32_t enable) {
 extern "C" fax_status fax_set_dependent_launch(fax_ctx* ctx, int32_t enable) {
   if (!ctx) return FAX_ERR_INVALID_ARG;
   ctx->use_pdl = enable != 0;
+  cudaStreamSynchronize(ctx->stream);
+  fax_graph_clear(ctx);
+  return FAX_OK;
+}
+
+extern "C" fax_status fax_set_gemm_l2_budget(fax_ctx* ctx, int64_t bytes) {
+  if (!ctx || bytes < 0) return FAX_ERR_INVALID_ARG;
+  ctx->gemm_l2_budget = (double)bytes;
   cudaStreamSynchronize(ctx->stream);
   fax_graph_clear(ctx);
   return FAX_OK;

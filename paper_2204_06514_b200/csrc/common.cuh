@@ -60,6 +60,7 @@ struct fax_ctx {
   bool keep_fused_grads;     // ... and still store those gradients
   bool use_2cta;             // GEMMs whose M and N are multiples of 256 use the two-CTA kernel
   bool use_pdl;              // kernels are launched with programmatic stream serialization allowed
+  double gemm_l2_budget;     // bytes of L2 a GEMM may count on for the operand panels it keeps between waves (0: fixed raster)
   bool attn_bwd_two_chains;  // head_dim-128 attention backward runs the kernel with two query sub-tiles in flight
 };
 

@@ -18,7 +18,8 @@ struct GemmParams {
   int32_t* status;
   float* ad_w; float* ad_m; float* ad_v; bf16* ad_wc;   // EPI_ADAMW: state of the weight this GEMM's result updates
   float ad_wd; float ad_sc[8]; int ad_keep;
-  int group_m;         // row-tiles per raster group
+  int group_m;         // tiles per raster group along the grouped dimension
+  int group_along_n;   // 0: groups of row-tiles swept across the columns; 1: groups of column-tiles swept down the rows
   int splits;          // > 1: each work item covers a slice of K and adds its partial tile into a float C
 };
 
@@ -39,16 +40,21 @@ __device__ __forceinline__ float gelu_grad_fast(float h) {
   return 0.5f * (1.0f + t) + 0.5f * h * (1.0f - t * t) * c * (1.0f + 3.0f * a * h * h);
 }
 
-// Tile order: groups of group_m row-tiles are swept across all column-tiles before the next
-// group starts, so the ~148 tiles in flight share few A row-panels and B column-panels in L2.
-__device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int group_m, int& tm, int& tn) {
-  const int per_group = group_m * tiles_n;
+// Tile order: groups of `group` row-tiles are swept across all column-tiles before the next group
+// starts (along_n: groups of column-tiles swept down all row-tiles), so the tiles in flight share
+// few A row-panels and B column-panels in L2, and the group's own panels stay in L2 from one wave
+// of tiles to the next while the other operand streams past once per group.
+__device__ __forceinline__ void tile_coords(int tile, int tiles_m, int tiles_n, int group, int along_n, int& tm, int& tn) {
+  const int t_g = along_n ? tiles_n : tiles_m;      // tiles along the grouped dimension
+  const int t_s = along_n ? tiles_m : tiles_n;      // tiles along the swept dimension
+  const int per_group = group * t_s;
   const int g = tile / per_group;
-  const int first_m = g * group_m;
-  const int rows = min(group_m, tiles_m - first_m);
+  const int first = g * group;
+  const int width = min(group, t_g - first);
   const int in = tile - g * per_group;
-  tm = first_m + in % rows;
-  tn = in / rows;
+  const int ig = first + in % width, is = in / width;
+  tm = along_n ? is : ig;
+  tn = along_n ? ig : is;
 }
 
 // Epilogue of one 32-column chunk held in registers: row `row`, columns col .. col+31.
@@ -217,7 +223,7 @@ static inline void fill_gemm_params(GemmParams& p, const FaxGemm& g, int32_t* st
   p.C = g.C; p.ldc = g.ldc; p.c_f32 = g.c_f32; p.accumulate = g.accumulate; p.epi = g.epi;
   p.bias = (const bf16*)g.bias; p.resid = (const bf16*)g.resid; p.ldr = g.ldr; p.aux = (bf16*)g.aux; p.ldaux = g.ldaux;
   p.alpha = g.alpha; p.status = status;
-  p.group_m = 8;
+  p.group_m = 8; p.group_along_n = 0;
   p.splits = 1;
   p.ad_w = p.ad_m = p.ad_v = nullptr; p.ad_wc = nullptr; p.ad_wd = 0.f; p.ad_keep = 0;
   for (int i = 0; i < 8; ++i) p.ad_sc[i] = 0.f;
@@ -227,6 +233,37 @@ static inline void fill_gemm_params(GemmParams& p, const FaxGemm& g, int32_t* st
     p.ad_wd = g.adam->weight_decay; p.ad_keep = g.adam->keep_grad ? 1 : 0;
     for (int i = 0; i < 8; ++i) p.ad_sc[i] = g.adam->sc[i];
   }
+}
+
+// Raster order of a problem with tile_m x tile_n tiles, `units` of them in flight.  DRAM reads are
+// (panel = one tile's rows or columns of an operand over all of K):
+//   grouped along M, G row-panels of A kept in L2:  A once + B once per group  = A + B * ceil(tiles_m / G)
+//   grouped along N, G column-panels of B kept:      B once + A once per group  = B + A * ceil(tiles_n / G)
+// as long as the group's panels fit the share of L2 that is left to them (l2_budget bytes); when even
+// a few panels do not fit (long K), nothing survives from wave to wave and the square-ish 8-tile group,
+// which minimises the panels one wave touches, stays.
+static inline void gemm_choose_raster(GemmParams& p, int tile_m, int tile_n, int units, double l2_budget) {
+  const int tiles_m = p.M / tile_m, tiles_n = p.N / tile_n;
+  const double a_bytes = 2.0 * p.M * p.K, b_bytes = 2.0 * p.N * p.K;
+  const double pa = 2.0 * tile_m * p.K, pb = 2.0 * tile_n * p.K;
+  p.group_m = 8; p.group_along_n = 0;
+  if (tiles_m * tiles_n <= units) return;                          // a single wave
+  const int g0 = tiles_m < 8 ? tiles_m : 8;
+  const double waves = (double)tiles_m * tiles_n / units;
+  double best = waves * (g0 * pa + ((double)units / g0) * pb);     // no reuse between waves
+  auto consider = [&](bool along_n) {
+    const int t_g = along_n ? tiles_n : tiles_m;
+    const double panel = along_n ? pb : pa;
+    int g = (int)(l2_budget / panel);
+    if (g < 4) return;                                             // too few panels in a wave to be worth keeping
+    if (g > t_g) g = t_g;
+    const int groups = (t_g + g - 1) / g;
+    g = (t_g + groups - 1) / groups;                               // even groups
+    const double traffic = along_n ? b_bytes + a_bytes * groups : a_bytes + b_bytes * groups;
+    if (traffic < best) { best = traffic; p.group_m = g; p.group_along_n = along_n ? 1 : 0; }
+  };
+  consider(false);
+  consider(true);
 }
 
 // Number of K slices the launchers use for a problem with `tiles` output tiles on `units`

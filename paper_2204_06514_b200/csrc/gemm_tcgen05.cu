@@ -88,7 +88,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       bool ok = true;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
         int tm, tn;
-        tile_coords(tile % out_tiles, tiles_m, tiles_n, p.group_m, tm, tn);
+        tile_coords(tile % out_tiles, tiles_m, tiles_n, p.group_m, p.group_along_n, tm, tn);
         const int m0 = tm * BM, n0 = tn * BN;
         const int kb0 = (tile / out_tiles) * kb_per, kb1 = min(kb_total, kb0 + kb_per);
         for (int kb = kb0; kb < kb1; ++kb) {
@@ -163,7 +163,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     bool ok = true;
     for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
       int tm, tn;
-      tile_coords(tile % out_tiles, tiles_m, tiles_n, p.group_m, tm, tn);
+      tile_coords(tile % out_tiles, tiles_m, tiles_n, p.group_m, p.group_along_n, tm, tn);
       const int m0 = tm * BM, n0 = tn * BN;
       const long long row = m0 + 32 * q + lane;
       U8 x0[2];
@@ -206,6 +206,7 @@ fax_status launch(fax_ctx* ctx, const FaxGemm& g) {
   // Few output tiles and a long K (the weight-gradient shapes of narrow models): slice K so that
   // the machine is filled; partial tiles are added into the float output with vector atomics.
   p.splits = gemm_split_count(g, tiles, ctx->sm_count, BK);
+  if (p.splits == 1 && ctx->gemm_l2_budget > 0) gemm_choose_raster(p, BM, BN, ctx->sm_count, ctx->gemm_l2_budget);
   if (p.splits > 1 && !g.accumulate)
     FAX_CUDA_TRY(ctx, cudaMemset2DAsync(g.C, (size_t)g.ldc * 4, 0, (size_t)g.N * 4, (size_t)g.M, ctx->stream));
   const int items = tiles * p.splits;

@@ -126,7 +126,7 @@ gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
       bool ok = true;
       for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
         int tm, tn;
-        tile_coords(tile % out_tiles, tiles_m, tiles_n, p.group_m, tm, tn);
+        tile_coords(tile % out_tiles, tiles_m, tiles_n, p.group_m, p.group_along_n, tm, tn);
         const int m0 = tm * 2 * BM + (int)rank * BM, n0 = tn * BN + (int)rank * BNH;
         const int kb0 = (tile / out_tiles) * kb_per, kb1 = min(kb_total, kb0 + kb_per);
         for (int kb = kb0; kb < kb1; ++kb) {
@@ -198,7 +198,7 @@ gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
     bool ok = true;
     for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
       int tm, tn;
-      tile_coords(tile % out_tiles, tiles_m, tiles_n, p.group_m, tm, tn);
+      tile_coords(tile % out_tiles, tiles_m, tiles_n, p.group_m, p.group_along_n, tm, tn);
       const int m0 = tm * 2 * BM + (int)rank * BM, n0 = tn * BN;
       const long long row = m0 + 32 * q + lane;
       U8 x0[2];
@@ -256,6 +256,7 @@ fax_status fax_gemm_tc2(fax_ctx* ctx, const FaxGemm& g) {
   const int tiles = (g.M / 256) * (g.N / 256);
   const int max_pairs = ctx->sm_count / 2;
   p.splits = gemm_split_count(g, tiles, max_pairs, BK);
+  if (p.splits == 1 && ctx->gemm_l2_budget > 0) gemm_choose_raster(p, 256, 256, max_pairs, ctx->gemm_l2_budget);
   if (p.splits > 1 && !g.accumulate)
     FAX_CUDA_TRY(ctx, cudaMemset2DAsync(g.C, (size_t)g.ldc * 4, 0, (size_t)g.N * 4, (size_t)g.M, ctx->stream));
   const int items = tiles * p.splits;

@@ -39,9 +39,12 @@ def main():
     ap.add_argument("--heads", type=int, default=32); ap.add_argument("--hd", type=int, default=128)
     ap.add_argument("--rows", type=int, default=8192); ap.add_argument("--d", type=int, default=4096)
     ap.add_argument("--iters", type=int, default=20); ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--l2-budget-mb", type=float, default=-1.0, help="GEMM raster: L2 bytes for resident panels (0: fixed order)")
     a = ap.parse_args()
     build.build()
     s = Session(0)
+    if a.l2_budget_mb >= 0:
+        fx.fax_set_gemm_l2_budget(s.ctx, int(a.l2_budget_mb * 1e6))
     dev, bf = s.device, torch.bfloat16
     g = torch.Generator(device=dev); g.manual_seed(1)
     rn = lambda *shape: torch.randn(shape, generator=g, device=dev).to(bf)

@@ -18,7 +18,7 @@ def lib():
 
 def declared_symbols():
     names = set()
-    for h in ("fax.h", "fax_ops.h"):
+    for h in ("fax.h", "fax_ops.h", "fax_dp.h"):
         text = open(os.path.join(ROOT, "include", h)).read()
         text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
         names |= set(re.findall(r"\b(fax_[a-z0-9_]+)\s*\(", text))
@@ -33,8 +33,8 @@ def test_every_declared_symbol_is_exported(lib):
 
 
 def test_binding_covers_every_declared_symbol(lib):
-    from paper_2204_06514_b200 import binding, binding_ops
-    have = set(binding._SIGNATURES) | set(binding_ops._SIGNATURES)
+    from paper_2204_06514_b200 import binding, binding_ops, dp
+    have = set(binding._SIGNATURES) | set(binding_ops._SIGNATURES) | set(dp._SIGNATURES)
     assert set(declared_symbols()) <= have
 
 
