@@ -386,12 +386,12 @@ def run_ours(args):
                 prev = e
         return dist_util.max_over_ranks(e0.elapsed_time(e1), dev)
 
-    sampler = ClockSampler(local)
-    sampler.start()
     for _ in range(max(args.warmup, 3)):
         step()
     torch.cuda.synchronize()
-    time.sleep(0.1)
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.25)              # the sampler's first readings; same pause before the timed region as ever
     l0 = sess.launches()
     ms = timed(step, args.steps, step_marks, tag="timed")
     launches = sess.launches() - l0

@@ -41,14 +41,14 @@ struct Bwd3Params {
   int32_t* status;
 };
 
-struct B3 {
-  static constexpr int HD = 128;
-  static constexpr int TILE_BYTES = 128 * HD * 2;         // 32 KB: two panels of 128 rows x 128 B
+template <int HD_> struct B3 {
+  static constexpr int HD = HD_;
+  static constexpr int TILE_BYTES = 128 * HD * 2;         // HD / 64 panels of 128 rows x 128 B
   static constexpr int K_OFF = 0, V_OFF = TILE_BYTES;
   static constexpr int Q_OFF = 2 * TILE_BYTES;            // two stages
   static constexpr int DO_OFF = 4 * TILE_BYTES;           // two stages
   static constexpr int DS_OFF = 6 * TILE_BYTES;           // dS^T: two panels (query halves) of 128 key rows x 128 B
-  static constexpr int STAT_OFF = 7 * TILE_BYTES;         // [2 stages][0: log2e * lse, 1: D][128] floats
+  static constexpr int STAT_OFF = DS_OFF + 32768;         // [2 stages][0: log2e * lse, 1: D][128] floats
   static constexpr int BAR_OFF = STAT_OFF + 2 * 1024;
   // a dQ tile is staged as 2 x 4 boxes of 64 rows x 32 floats (32 KB per query half): first half in the tile's
   // dO stage, second half in the dS^T tile
@@ -56,16 +56,17 @@ struct B3 {
                        PREADY = 12, DSREADY = 14, DQFULL = 16, DQREAD = 17, STGFULL = 18 /* per half */,
                        STGFREE_DO = 20 /* per stage */, STGFREE_DS = 22, ALLDONE = 23, DKVREAD = 24, NBARS = 25;
   static constexpr int LAYOUT_BYTES = BAR_OFF + NBARS * 8 + 16;
-  static constexpr int SMEM_BYTES = 227 * 1024;           // the layout plus slack for aligning it to 1024 bytes
+  // the layout plus slack for aligning it to 1024 bytes, capped at the 227 KB a block may have (head_dim 128)
+  static constexpr int SMEM_BYTES = (LAYOUT_BYTES + 1024 < 227 * 1024) ? LAYOUT_BYTES + 1024 : 227 * 1024;
   static constexpr int TMEM_COLS = 512;
 };
-static_assert(B3::LAYOUT_BYTES + 512 <= B3::SMEM_BYTES, "shared-memory layout does not fit");
+static_assert(B3<128>::LAYOUT_BYTES + 512 <= B3<128>::SMEM_BYTES, "shared-memory layout does not fit");
 
+template <int HD>
 __global__ void __launch_bounds__(B3_THREADS, 1)
 attn_bwd3_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_constant__ CUtensorMap tmap_do,
                     const __grid_constant__ CUtensorMap tmap_dq, const Bwd3Params p) {
-  using C_ = B3;
-  constexpr int HD = C_::HD;
+  using C_ = B3<HD>;
   constexpr uint32_t HALF_WARPS = B3_ROW_WARPS / 2;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -176,7 +177,9 @@ attn_bwd3_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_c
     if (lane == 0) {
       const uint32_t idesc_s = idesc_bf16(128, false, false);      // S^T, dP^T: both operands K-major
       const uint32_t idesc_acc = idesc_bf16(HD, false, true);      // dV, dK: A in tensor memory, B MN-major
-      const uint32_t idesc_dq = idesc_bf16(128, true, true);       // dQ^T: K^T and dS^T both MN-major
+      // dQ^T = K^T dS^T (128 x 128) at head_dim 128; dQ = dS K (128 queries x 64) at head_dim 64, where the
+      // transposed form would have only 64 rows: both operands MN-major either way
+      const uint32_t idesc_dq = idesc_bf16(HD == 128 ? 128 : 64, true, true);
       // A descriptor = {low word, high word}; only the 14-bit start-address field (16-byte units) of the
       // low word changes between stages and k-steps.  K-major tiles: a k-step is 32 bytes inside a
       // 64-column panel (panels 16 KB apart); MN-major: a k-step is 16 rows (2048 bytes).
@@ -244,7 +247,10 @@ attn_bwd3_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_c
           if (!mbar_wait(bar(C_::DSREADY + 1), ph, abort_flag, p.status, 347)) { ok = false; break; }
           tc_fence_after();
 #pragma unroll
-          for (int k = 0; k < 8; ++k) tc_mma_bf16(tm_dp, mk(k_mn + k * 128), mk(ds_mn + k * 128), idesc_dq, k ? 1u : 0u);
+          for (int k = 0; k < 8; ++k) {
+            if (HD == 128) tc_mma_bf16(tm_dp, mk(k_mn + k * 128), mk(ds_mn + k * 128), idesc_dq, k ? 1u : 0u);
+            else tc_mma_bf16(tm_dp, mk(ds_mn + k * 128), mk(k_mn + k * 128), idesc_dq, k ? 1u : 0u);
+          }
           tc_commit(bar(C_::DQFULL));
 #pragma unroll
           for (int k = 4; k < 8; ++k) tc_mma_bf16_ts(tm_dk, tm_s + 16u + acol(k), mk(bq + k * 128), idesc_acc, 1u);
@@ -271,7 +277,7 @@ attn_bwd3_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_c
           // second query half first: its staging bytes (the dS^T tile) are needed again soonest
           if (!mbar_wait(bar(C_::STGFULL + 1), gs & 1u, abort_flag, p.status, 351)) { ok = false; break; }
 #pragma unroll
-          for (int i = 0; i < HD / 32; ++i) tma_reduce_add_2d(&tmap_dq, ds_s + i * 8192, h * HD + 32 * i, qrow + 64);
+          for (int i = 0; i < HD / 32; ++i) tma_reduce_add_2d(&tmap_dq, ds_s + i * 8192, h * HD + 32 * i, qrow + 64);   // boxes of 64 rows x 32 floats
           bulk_commit_group();
           if (!mbar_wait(bar(C_::STGFULL), gs & 1u, abort_flag, p.status, 351)) { ok = false; break; }
 #pragma unroll
@@ -376,7 +382,7 @@ attn_bwd3_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_c
         // ---- dQ^T (lane = head column kr, this quarter's 32 queries) -> staging boxes (row = query) ----
         if (!mbar_wait_warp(bar(C_::DQFULL), ph, abort_flag, p.status, 355)) { ok = false; break; }
         tc_fence_after();
-        {
+        if (HD == 128) {
           uint32_t v[32];
           tc_ld32(tm_dp + lane_base + 32u * qr, v);
           tc_wait_ld();
@@ -391,27 +397,53 @@ attn_bwd3_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_c
             const int q = 32 * (int)(qr & 1u) + j;
             *reinterpret_cast<uint32_t*>(box + q * 128 + (((lane >> 2) ^ (q & 7)) << 4)) = v[j];
           }
+          fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar(C_::STGFULL + half));
+        } else {
+          // head_dim 64: dQ (lane = query row kr, 64 head columns); this thread takes columns 16 qr .. 16 qr + 15.
+          // Query rows 0..63 (lane quarters 0, 1) are staged in the dO stage, rows 64..127 in the dS^T tile,
+          // each as two boxes of 64 rows x 32 floats.
+          uint32_t v[16];
+          tc_ld16(tm_dp + lane_base + 16u * qr, v);
+          tc_wait_ld();
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar(C_::DQREAD));
+          const uint32_t qhalf = (uint32_t)(warp & 3) >> 1;
+          const int r = kr & 63;
+          uint8_t* box = gbase + (qhalf ? (uint32_t)C_::DS_OFF : (uint32_t)C_::DO_OFF + sq * C_::TILE_BYTES) + (qr >> 1) * 8192 + r * 128;
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            *reinterpret_cast<uint4*>(box + (((4 * (int)(qr & 1u) + k) ^ (r & 7)) << 4)) =
+                make_uint4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
+          fence_proxy_async();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar(C_::STGFULL + qhalf));
         }
-        fence_proxy_async();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(bar(C_::STGFULL + half));
       }
       if (!ok) break;
       if (!mbar_wait_warp(bar(C_::ALLDONE), (uint32_t)(it_n & 1), abort_flag, p.status, 357)) { ok = false; break; }
       tc_fence_after();
       {
+        constexpr int CW = HD / 4;                 // head columns per thread: 32 or 16
         const long long tok = (long long)row0 + kj * 128 + kr;
-        bf16* dk_row = p.dqkv + tok * 3 * d + d + h * HD + 32 * qr;
-        bf16* dv_row = p.dqkv + tok * 3 * d + 2 * d + h * HD + 32 * qr;
-        uint32_t kv[32], vv[32];
-        tc_ld32(tm_dk + lane_base + 32u * qr, kv);
-        tc_ld32(tm_dv + lane_base + 32u * qr, vv);
+        bf16* dk_row = p.dqkv + tok * 3 * d + d + h * HD + CW * qr;
+        bf16* dv_row = p.dqkv + tok * 3 * d + 2 * d + h * HD + CW * qr;
+        uint32_t kv[CW], vv[CW];
+        if (HD == 128) {
+          tc_ld32(tm_dk + lane_base + 32u * qr, reinterpret_cast<uint32_t(&)[32]>(kv));
+          tc_ld32(tm_dv + lane_base + 32u * qr, reinterpret_cast<uint32_t(&)[32]>(vv));
+        } else {
+          tc_ld16(tm_dk + lane_base + 16u * qr, reinterpret_cast<uint32_t(&)[16]>(kv));
+          tc_ld16(tm_dv + lane_base + 16u * qr, reinterpret_cast<uint32_t(&)[16]>(vv));
+        }
         tc_wait_ld();
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar(C_::DKVREAD));
 #pragma unroll
-        for (int c = 0; c < 32; c += 16) {        // 16 columns = one 32-byte sector per store
+        for (int c = 0; c < CW; c += 16) {        // 16 columns = one 32-byte sector per store
           U8 uk, uv;
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
@@ -434,14 +466,13 @@ attn_bwd3_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_c
 }  // namespace
 
 bool fax_attention_bwd3_supported(int B, int T, int H, int hd) {
-  return hd == 128 && T % 128 == 0 && B > 0 && H > 0;
+  return (hd == 128 || hd == 64) && T % 128 == 0 && B > 0 && H > 0;
 }
 
-// The main kernel only: D = rowsum(dO o O) must be in Dv and dq_acc cleared (both by the row-dot
-// kernel), and dq_acc is converted to bf16 by the caller afterwards.
-fax_status fax_attention_bwd3_tc(fax_ctx* ctx, int B, int T, int H, const void* qkv, const float* lse,
-                                 const void* d_o, void* dqkv, const float* Dv, float* dq_acc) {
-  constexpr int HD = B3::HD;
+namespace {
+template <int HD>
+fax_status launch_bwd3(fax_ctx* ctx, int B, int T, int H, const void* qkv, const float* lse, const void* d_o,
+                       void* dqkv, const float* Dv, float* dq_acc) {
   CUtensorMap mq, md, mdq;
   const uint64_t d = (uint64_t)H * HD;
   const uint64_t n_tok = (uint64_t)B * T;
@@ -454,9 +485,18 @@ fax_status fax_attention_bwd3_tc(fax_ctx* ctx, int B, int T, int H, const void* 
   p.scale_log2 = 1.4426950408889634f * p.scale;
   p.status = ctx->dev_status;
   static bool attr_set[FAX_MAX_DEVICES] = {};
-  FAX_TRY(fax_opt_in_shared_memory(ctx, attn_bwd3_tc_kernel, B3::SMEM_BYTES, attr_set));
+  FAX_TRY(fax_opt_in_shared_memory(ctx, attn_bwd3_tc_kernel<HD>, B3<HD>::SMEM_BYTES, attr_set));
   const long long items = (long long)B * H * (T / 128);
   const int grid = (int)(items < ctx->sm_count ? items : ctx->sm_count);
-  fax_launch(ctx, attn_bwd3_tc_kernel, dim3(grid), dim3(B3_THREADS), B3::SMEM_BYTES, mq, md, mdq, p);
+  fax_launch(ctx, attn_bwd3_tc_kernel<HD>, dim3(grid), dim3(B3_THREADS), B3<HD>::SMEM_BYTES, mq, md, mdq, p);
   return fax_after_launch(ctx);
+}
+}  // namespace
+
+// The main kernel only: D = rowsum(dO o O) must be in Dv and dq_acc cleared (both by the row-dot
+// kernel), and dq_acc is converted to bf16 by the caller afterwards.
+fax_status fax_attention_bwd3_tc(fax_ctx* ctx, int B, int T, int H, int hd, const void* qkv, const float* lse,
+                                 const void* d_o, void* dqkv, const float* Dv, float* dq_acc) {
+  return hd == 128 ? launch_bwd3<128>(ctx, B, T, H, qkv, lse, d_o, dqkv, Dv, dq_acc)
+                   : launch_bwd3<64>(ctx, B, T, H, qkv, lse, d_o, dqkv, Dv, dq_acc);
 }

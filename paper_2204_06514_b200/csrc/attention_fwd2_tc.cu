@@ -118,6 +118,14 @@ attn_fwd2_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnFwd2Para
     if (lane == 0) {
       const uint32_t idesc_s = idesc_bf16(128, false, false);
       const uint32_t idesc_o = idesc_bf16(HD, false, true);
+      // descriptors = {low word, high word}; only the start-address field (16-byte units) of the low word
+      // differs between tiles and k-steps, so each product adds a constant to a precomputed word (the
+      // instructions of this one thread between two products are on the critical path)
+      const uint32_t d_hi = (uint32_t)(smem_desc(0, 16, 1024) >> 32);
+      const uint32_t q_lo0 = (uint32_t)smem_desc(q_s(0), 16, 1024), k_lo0 = (uint32_t)smem_desc(k_s(0), 16, 1024);
+      const uint32_t v_lo0 = (uint32_t)smem_desc(v_s(0), 16384, 1024);
+      constexpr uint32_t TILE16 = C_::TILE_BYTES >> 4;
+      auto mk = [&](uint32_t lo) -> uint64_t { return ((uint64_t)d_hi << 32) | lo; };
       uint32_t kc0 = 0;                 // K / V tiles of the pairs before this one
       uint32_t pc[2] = {0u, 0u};        // P tiles consumed per query tile
       bool ok = true;
@@ -132,11 +140,12 @@ attn_fwd2_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnFwd2Para
           const int s = (int)(c % NS);
           if (!mbar_wait(bar(C_::KFULL + s), (c / NS) & 1u, abort_flag, p.status, 224)) return false;
           tc_fence_after();
+          const uint32_t qlo = q_lo0 + (uint32_t)x * TILE16, klo = k_lo0 + (uint32_t)s * TILE16;
+          const uint32_t dst = tmem + (uint32_t)(x * 128);
 #pragma unroll
           for (int k = 0; k < HD / 16; ++k) {
-            const uint32_t off = (k / 4) * 16384 + (k % 4) * 32;
-            tc_mma_bf16(tmem + (uint32_t)(x * 128), smem_desc(q_s(x) + off, 16, 1024), smem_desc(k_s(s) + off, 16, 1024),
-                        idesc_s, k ? 1u : 0u);
+            const uint32_t off = (k / 4) * 1024 + (k % 4) * 2;
+            tc_mma_bf16(dst, mk(qlo + off), mk(klo + off), idesc_s, k ? 1u : 0u);
           }
           tc_commit(bar(C_::SFULL + x));
           return true;
@@ -148,10 +157,11 @@ attn_fwd2_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnFwd2Para
           if (j == 0 && !mbar_wait(bar(C_::OFREE + x), iph ^ 1u, abort_flag, p.status, 226)) return false;
           tc_fence_after();
           const int s = (int)((kc0 + (uint32_t)j) % NS);
+          const uint32_t vlo = v_lo0 + (uint32_t)s * TILE16;
+          const uint32_t dst = tmem + 256u + (uint32_t)(x * 128), src = tmem + (uint32_t)(x * 128);
 #pragma unroll
           for (int k = 0; k < 8; ++k)
-            tc_mma_bf16_ts(tmem + 256u + (uint32_t)(x * 128), tmem + (uint32_t)(x * 128 + 8 * k),
-                           smem_desc(v_s(s) + k * 2048, 16384, 1024), idesc_o, (j | k) ? 1u : 0u);
+            tc_mma_bf16_ts(dst, src + 8 * k, mk(vlo + k * 128), idesc_o, (j | k) ? 1u : 0u);
           return true;
         };
         if (!mbar_wait(bar(C_::QFULL), iph, abort_flag, p.status, 227)) { ok = false; break; }

@@ -752,8 +752,8 @@ fax_status launch_bwd(fax_ctx* ctx, int B, int T, int H, const void* qkv, const 
   p.scale = 1.0f / sqrtf((float)HD);
   p.scale_log2 = 1.4426950408889634f * p.scale;
   p.status = ctx->dev_status;
-  if (HD == 128 && ctx->attn_bwd_two_chains && fax_attention_bwd3_supported(B, T, H, HD)) {
-    FAX_TRY(fax_attention_bwd3_tc(ctx, B, T, H, qkv, lse, d_o, dqkv, Dv, dq_acc));
+  if (ctx->attn_bwd_two_chains && fax_attention_bwd3_supported(B, T, H, HD)) {
+    FAX_TRY(fax_attention_bwd3_tc(ctx, B, T, H, HD, qkv, lse, d_o, dqkv, Dv, dq_acc));
   } else {
     static bool attr_set[FAX_MAX_DEVICES] = {};
     FAX_TRY(fax_opt_in_shared_memory(ctx, attn_bwd2_tc_kernel<HD>, Bwd2Cfg<HD>::SMEM_BYTES, attr_set));

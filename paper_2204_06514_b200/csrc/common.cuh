@@ -61,7 +61,7 @@ struct fax_ctx {
   bool use_2cta;             // GEMMs whose M and N are multiples of 256 use the two-CTA kernel
   bool use_pdl;              // kernels are launched with programmatic stream serialization allowed
   double gemm_l2_budget;     // bytes of L2 a GEMM may count on for the operand panels it keeps between waves (0: fixed raster)
-  bool attn_bwd_two_chains;  // head_dim-128 attention backward runs the kernel with two query sub-tiles in flight
+  bool attn_bwd_two_chains;  // attention backward runs the sixteen-row-warp kernel (half-tile hand-offs)
 };
 
 // Brackets the launches of one operator with CUDA events while profiling is on.
@@ -305,9 +305,9 @@ fax_status fax_gelu_fwd(fax_ctx* ctx, int prec, size_t n, const void* h, void* g
 bool fax_attention_fwd2_supported(int B, int T, int H, int hd);
 fax_status fax_attention_fwd2_tc(fax_ctx* ctx, int B, int T, int H, int hd, const void* qkv, void* o, float* lse);
 size_t fax_attention_bwd_tc_scratch_bytes(int B, int T, int H, int hd);
-// head_dim-128 backward with two query sub-tiles in flight (the main kernel only; see its definition)
+// backward with sixteen row warps and half-tile hand-offs (the main kernel only; see its definition)
 bool fax_attention_bwd3_supported(int B, int T, int H, int hd);
-fax_status fax_attention_bwd3_tc(fax_ctx* ctx, int B, int T, int H, const void* qkv, const float* lse,
+fax_status fax_attention_bwd3_tc(fax_ctx* ctx, int B, int T, int H, int hd, const void* qkv, const float* lse,
                                  const void* d_o, void* dqkv, const float* Dv, float* dq_acc);
 fax_status fax_attention_bwd_tc(fax_ctx* ctx, int B, int T, int H, int hd, const void* qkv, const void* o,
                                 const float* lse, const void* d_o, void* dqkv, void* scratch, size_t scratch_bytes);
