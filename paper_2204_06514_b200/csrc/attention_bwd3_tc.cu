@@ -1,4 +1,7 @@
-// Causal attention backward (step B5) at head_dim 128: sixteen row warps, half-tile hand-offs.
+// Causal attention backward (step B5), head_dim 128 and 64: sixteen row warps, half-tile hand-offs.
+// (Written for head_dim 128 below; at head_dim 64 the operand tiles are one 64-column panel, dV and dK
+// take 64 tensor-memory columns each, and dQ is formed untransposed, dQ = dS K with the queries in the
+// lanes, because the transposed form would have only 64 rows; its staging is by query rows.)
 //
 // A CTA owns a 128-key tile j (K_j, V_j resident in shared memory) and walks the 128-query tiles
 // i >= j.  Everything is formed transposed (keys in the tensor-memory lanes): S^T = K_j Q_i^T and
