@@ -81,16 +81,11 @@ __device__ __forceinline__ void gemm_epilogue_fetch(const GemmParams& p, long lo
   }
 }
 
+// Values of one chunk before they are stored: alpha * accumulator (+ bias) (+ residual) (* GELU'(pre-activation));
+// xv holds the chunk's 32 residual / pre-activation values where the mode reads any.
 template <int EPI>
-__device__ __forceinline__ void gemm_epilogue_chunk(const GemmParams& pr, const uint32_t (&r)[32], const U8 (&x)[2],
-                                                    long long row, int col) {
-        const GemmParams& p = pr;
-        const int p_epi = EPI == EPI_STATIC_F32 ? (int)EPI_NONE : (EPI >= 0 ? EPI : pr.epi);
-        const bool p_c_f32 = EPI == EPI_STATIC_F32 ? true : (EPI >= 0 ? false : (pr.c_f32 != 0));
-        U8 xn[2];
-        if (EPI < 0) gemm_epilogue_fetch<EPI, true>(pr, row, col, xn);
-        const U8* xv = EPI < 0 ? xn : x;
-        float v[32];
+__device__ __forceinline__ void gemm_epilogue_values(const GemmParams& p, const uint32_t (&r)[32], const U8* xv, int p_epi,
+                                                     int col, float (&v)[32]) {
 #pragma unroll
         for (int j = 0; j < 32; ++j) v[j] = __uint_as_float(r[j]) * p.alpha;
         if (p_epi == EPI_BIAS || p_epi == EPI_BIAS_GELU || p_epi == EPI_BIAS_RESID) {
@@ -126,6 +121,19 @@ __device__ __forceinline__ void gemm_epilogue_chunk(const GemmParams& pr, const 
             }
           }
         }
+}
+
+template <int EPI>
+__device__ __forceinline__ void gemm_epilogue_chunk(const GemmParams& pr, const uint32_t (&r)[32], const U8 (&x)[2],
+                                                    long long row, int col) {
+        const GemmParams& p = pr;
+        const int p_epi = EPI == EPI_STATIC_F32 ? (int)EPI_NONE : (EPI >= 0 ? EPI : pr.epi);
+        const bool p_c_f32 = EPI == EPI_STATIC_F32 ? true : (EPI >= 0 ? false : (pr.c_f32 != 0));
+        U8 xn[2];
+        if (EPI < 0) gemm_epilogue_fetch<EPI, true>(pr, row, col, xn);
+        const U8* xv = EPI < 0 ? xn : x;
+        float v[32];
+        gemm_epilogue_values<EPI>(p, r, xv, p_epi, col, v);
         if (p_epi == EPI_ADAMW) {
           // the accumulator is the gradient of w[row, col..]: AdamW here, w / m / v in place
           const long long off = row * p.ldc + col;
@@ -267,16 +275,25 @@ static inline void gemm_choose_raster(GemmParams& p, int tile_m, int tile_n, int
 }
 
 // Number of K slices the launchers use for a problem with `tiles` output tiles on `units`
-// tile-processing units (SMs, or SM pairs).
+// tile-processing units (SMs, or SM pairs).  Only plain float outputs are sliced (the partial tiles
+// are added into C).  Cost model in K blocks: waves of work items x (K blocks per item + a per-item
+// overhead for the epilogue and the pipeline refill); slicing pays when the tiles alone leave units
+// idle (fewer tiles than units) or fill the last wave badly.
 static inline int gemm_split_count(const FaxGemm& g, int tiles, int units, int bk) {
   const int kb_total = g.K / bk;
-  if (!(g.c_f32 && g.epi == EPI_NONE && g.alpha == 1.f && !g.adam && tiles * 2 <= units && kb_total >= 16)) return 1;
-  int sp = units / tiles;
-  if (sp > kb_total / 8) sp = kb_total / 8;
-  if (sp > 16) sp = 16;
-  if (sp <= 1) return 1;
-  const int kb_per = (kb_total + sp - 1) / sp;
-  return (kb_total + kb_per - 1) / kb_per;          // no empty slices
+  if (!(g.c_f32 && g.epi == EPI_NONE && g.alpha == 1.f && !g.adam && kb_total >= 16)) return 1;
+  if (tiles >= 4 * units) return 1;
+  auto slices = [&](int sp) { const int kb_per = (kb_total + sp - 1) / sp; return (kb_total + kb_per - 1) / kb_per; };
+  auto cost = [&](int sp) {
+    const int kb_per = (kb_total + sp - 1) / sp;
+    const long long items = (long long)tiles * slices(sp);
+    const long long waves = (items + units - 1) / units;
+    return (double)waves * (kb_per + (sp > 1 ? 6 : 3));
+  };
+  int best = 1;
+  for (int sp = 2; sp <= 16 && kb_total / sp >= 8; ++sp)
+    if (cost(sp) < 0.95 * cost(best)) best = sp;
+  return slices(best);                              // no empty slices
 }
 
 // One warp's share of a tile: NCH chunks of 32 columns starting at tensor-memory address
@@ -303,6 +320,50 @@ __device__ __forceinline__ void gemm_epilogue_warp(const GemmParams& p, uint32_t
       tc_wait_ld();
       if (i + 2 < NCH) tc_ld32(t_base + 32 * (i + 2), ra); else drained();
       gemm_epilogue_chunk<EPI>(p, rb, xb, row, col0 + 32 * (i + 1));
+    }
+  }
+}
+
+// ---- K-sliced float output: partial tiles added into C by bulk tensor reductions ----
+//
+// A warp owns 32 rows x 128 columns of the tile, four chunks of 32 columns, and one 4 KB staging buffer.
+// Each thread writes its own row of a chunk (32 floats) into the buffer in the 128-byte-swizzled layout
+// the tensor map expects; one lane then issues the bulk add-reduction (float add at L2), which replaces
+// eight float4 atomics per thread and chunk.  Only this mode stages its output: for the stored outputs
+// the shared-memory traffic of a staged tile (written once, read once by the copy engine) slows the main
+// loop, whose operand staging already uses the shared-memory bandwidth, by more than the scattered
+// 32-byte stores from registers cost.
+constexpr int EPI_STAGING_BYTES = 4096;      // per epilogue warp
+constexpr int EPI_TMA_CHUNKS = 4;
+
+// Byte offset of the 16-byte unit `unit` of row `r` in a staging buffer (128-byte rows, 128-byte swizzle;
+// buffers are 1024-byte aligned).
+__device__ __forceinline__ uint32_t epi_sw128(int r, int unit) { return (uint32_t)(r * 128 + ((unit ^ (r & 7)) << 4)); }
+
+template <typename Drained>
+__device__ __forceinline__ void gemm_epilogue_warp_reduce(const GemmParams& p, const CUtensorMap* mc, uint32_t t_base,
+                                                          int row0, int col0, int lane, uint32_t stg, Drained drained) {
+  uint32_t rr[2][32];
+  tc_ld32(t_base, rr[0]);
+#pragma unroll
+  for (int i = 0; i < EPI_TMA_CHUNKS; ++i) {
+    tc_wait_ld();
+    if (i + 1 < EPI_TMA_CHUNKS) tc_ld32(t_base + 32 * (i + 1), rr[(i + 1) & 1]); else drained();
+    if (lane == 0) bulk_wait_read<0>();        // the previous chunk's reduction has read the buffer
+    __syncwarp();
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const uint32_t* r = rr[i & 1];
+      st_shared_v4(stg + epi_sw128(lane, u), __float_as_uint(__uint_as_float(r[4 * u]) * p.alpha),
+                   __float_as_uint(__uint_as_float(r[4 * u + 1]) * p.alpha),
+                   __float_as_uint(__uint_as_float(r[4 * u + 2]) * p.alpha),
+                   __float_as_uint(__uint_as_float(r[4 * u + 3]) * p.alpha));
+    }
+    fence_proxy_async();
+    __syncwarp();
+    if (lane == 0) {
+      tma_reduce_add_2d(mc, stg, col0 + 32 * i, row0);
+      bulk_commit_group();
     }
   }
 }

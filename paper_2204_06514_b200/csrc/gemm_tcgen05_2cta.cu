@@ -11,7 +11,9 @@
 //   warp 1      : tensor-memory allocation (both CTAs); MMA issue (even CTA only);
 //                 tcgen05.commit multicasts "stage empty" / "accumulator full" to both
 //   warps 2..9  : epilogue of the CTA's own 128 x 256 half; "accumulator empty" is
-//                 signalled to the even CTA's barrier
+//                 signalled to the even CTA's barrier.  Outputs are stored from registers; the
+//                 partial tiles of a K-sliced float GEMM are staged in shared memory and added
+//                 into C by bulk tensor reductions.
 // Every TMA load is a plain load into the issuing CTA's own shared memory.  Every wait is bounded.
 #include "gemm_common.cuh"
 
@@ -30,7 +32,13 @@ constexpr int NUM_THREADS = 32 * (2 + NUM_EPI_WARPS);
 constexpr int A_BYTES = BM * BK * 2, B_BYTES = BNH * BK * 2, STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int STAGES = 6;
 constexpr int TMEM_COLS = 512;
-constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
+constexpr int STAGING_BYTES = NUM_EPI_WARPS * EPI_STAGING_BYTES;
+constexpr int BAR_BYTES = 256;
+// Only the float-output instantiation stages partial tiles; the others leave that shared memory to L1,
+// which the epilogue's residual / pre-activation loads go through.
+constexpr int smem_bytes(int epi) { return STAGES * STAGE_BYTES + (epi == EPI_STATIC_F32 ? STAGING_BYTES : 0) + 1024 + BAR_BYTES; }
+static_assert(smem_bytes(EPI_STATIC_F32) <= 227 * 1024, "shared memory per CTA");
+static_assert(8 * (2 * STAGES + 4) + 8 <= BAR_BYTES, "barrier area");
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
   uint32_t r;
@@ -75,13 +83,15 @@ __device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint64_t adesc
 template <int EPI>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                         const GemmParams p) {
+                         const GemmParams p, const __grid_constant__ CUtensorMap tmap_c) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t tiles_base = (raw + 1023u) & ~1023u;
   uint8_t* gen_base = smem_raw + (tiles_base - raw);
-  uint8_t* bar_mem = gen_base + STAGES * STAGE_BYTES;
-  const uint32_t bars = tiles_base + STAGES * STAGE_BYTES;
+  const uint32_t staging = tiles_base + STAGES * STAGE_BYTES;
+  constexpr int STG = EPI == EPI_STATIC_F32 ? STAGING_BYTES : 0;
+  uint8_t* bar_mem = gen_base + STAGES * STAGE_BYTES + STG;
+  const uint32_t bars = staging + STG;
   auto full_bar = [&](int s) { return bars + 8u * s; };                         // used in the even CTA
   auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };             // one per CTA
   auto tfull_bar = [&](int a) { return bars + 8u * (2 * STAGES + a); };         // one per CTA
@@ -106,6 +116,7 @@ gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_a) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_b) : "memory");
+    if (EPI == EPI_STATIC_F32) asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap_c) : "memory");
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -194,25 +205,32 @@ gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
     const int q = warp & 3;
     const int half = (warp - 2) >> 2;
     constexpr int NCH = BN / 64;
+    static_assert(NCH == EPI_TMA_CHUNKS, "a warp's share is four chunks");
     int acc = 0; uint32_t acc_phase = 0;
+    const uint32_t stg = staging + (uint32_t)(warp - 2) * EPI_STAGING_BYTES;
+    const bool reduce_out = EPI == EPI_STATIC_F32 && p.splits > 1;
     bool ok = true;
     for (int tile = pair; tile < num_tiles && ok; tile += num_pairs) {
       int tm, tn;
       tile_coords(tile % out_tiles, tiles_m, tiles_n, p.group_m, p.group_along_n, tm, tn);
       const int m0 = tm * 2 * BM + (int)rank * BM, n0 = tn * BN;
       const long long row = m0 + 32 * q + lane;
+      const int col0 = n0 + half * (BN / 2);
       U8 x0[2];
-      gemm_epilogue_fetch<EPI>(p, row, n0 + half * (BN / 2), x0);     // in flight while the accumulator fills
+      gemm_epilogue_fetch<EPI>(p, row, col0, x0);     // in flight while the accumulator fills
       if (!mbar_wait_warp(tfull_bar(acc), acc_phase, abort_flag, p.status, 114)) { ok = false; break; }
       tc_fence_after();
       const uint32_t t_base = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(acc * BN + half * (BN / 2));
-      gemm_epilogue_warp<NCH, EPI>(p, t_base, row, n0 + half * (BN / 2), x0, [&]() {
+      auto drained = [&]() {
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive_cluster(leader_addr(tempty_bar(acc)));
-      });
+      };
+      if (reduce_out) gemm_epilogue_warp_reduce(p, &tmap_c, t_base, m0 + 32 * q, col0, lane, stg, drained);
+      else gemm_epilogue_warp<NCH, EPI>(p, t_base, row, col0, x0, drained);
       if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
+    if (reduce_out && lane == 0) bulk_wait_all();     // the staging buffers have been read and the additions are complete
   }
 
   tc_fence_before();
@@ -244,11 +262,13 @@ fax_status fax_gemm_tc2(fax_ctx* ctx, const FaxGemm& g) {
   ok = ok && (g.b_mn_major ? make_map(ctx, &mb, g.B, g.N, g.K, g.ldb, 64, BK)
                            : make_map(ctx, &mb, g.B, g.K, g.N, g.ldb, BK, BNH));
   if (!ok) return FAX_ERR_INVALID_ARG;
+  CUtensorMap mc = ma;                                   // read only by the K-sliced float epilogue
+  if (g.c_f32 && !make_map_f32(ctx, &mc, g.C, g.N, g.M, g.ldc, 32, 32)) return FAX_ERR_INVALID_ARG;
   GemmParams p;
   fill_gemm_params(p, g, ctx->dev_status);
   {
     static bool attr_set[7][FAX_MAX_DEVICES] = {};
-#define FAX_SET_SMEM(I, E) FAX_TRY(fax_opt_in_shared_memory(ctx, gemm_tcgen05_2cta_kernel<E>, SMEM_BYTES, attr_set[I]))
+#define FAX_SET_SMEM(I, E) FAX_TRY(fax_opt_in_shared_memory(ctx, gemm_tcgen05_2cta_kernel<E>, smem_bytes(E), attr_set[I]))
     FAX_SET_SMEM(0, -1); FAX_SET_SMEM(1, 0); FAX_SET_SMEM(2, 1); FAX_SET_SMEM(3, 2); FAX_SET_SMEM(4, 3); FAX_SET_SMEM(5, 4);
     FAX_SET_SMEM(6, EPI_STATIC_F32);
 #undef FAX_SET_SMEM
@@ -262,9 +282,9 @@ fax_status fax_gemm_tc2(fax_ctx* ctx, const FaxGemm& g) {
   const int items = tiles * p.splits;
   const int pairs = items < max_pairs ? items : max_pairs;
   switch (gemm_static_epi(g)) {
-#define FAX_LAUNCH(E) case E: fax_launch(ctx, gemm_tcgen05_2cta_kernel<E>, dim3(2 * pairs), dim3(NUM_THREADS), SMEM_BYTES, ma, mb, p); break
+#define FAX_LAUNCH(E) case E: fax_launch(ctx, gemm_tcgen05_2cta_kernel<E>, dim3(2 * pairs), dim3(NUM_THREADS), smem_bytes(E), ma, mb, p, mc); break
     FAX_LAUNCH(0); FAX_LAUNCH(1); FAX_LAUNCH(2); FAX_LAUNCH(3); FAX_LAUNCH(4); FAX_LAUNCH(EPI_STATIC_F32);
-    default: fax_launch(ctx, gemm_tcgen05_2cta_kernel<-1>, dim3(2 * pairs), dim3(NUM_THREADS), SMEM_BYTES, ma, mb, p); break;
+    default: fax_launch(ctx, gemm_tcgen05_2cta_kernel<-1>, dim3(2 * pairs), dim3(NUM_THREADS), smem_bytes(-1), ma, mb, p, mc); break;
 #undef FAX_LAUNCH
   }
   return fax_after_launch(ctx);
