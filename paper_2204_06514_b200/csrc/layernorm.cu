@@ -388,6 +388,134 @@ layernorm_bwd_ring_kernel(int rows, int d, const T* __restrict__ da, const T* __
   for (int c = threadIdx.x; c < NS * d / 4; c += blockDim.x) dst[c] = reinterpret_cast<const float4*>(fuse_sm)[c];
 }
 
+// Backward, fused, rows of 513 .. 2048 vectors: the same one pass as the ring kernel with the whole block
+// (16 warps) on one row at a time.  Thread t owns vectors t + 512 i, i < VPT, of every row the block walks
+// (blockIdx.x + k * gridDim.x), so the column sums stay in registers and each block writes its slab
+// straight from them.  The ring holds RING rows of da, x (and add) per block; the second pass over a row
+// re-reads the slot (it stays valid until the next iteration's copy is issued) instead of keeping the
+// row in registers, which leaves the registers to the column sums.  One block-wide barrier per row.
+// Dynamic shared memory: [slot][da | x | add][512 * VPT vectors].
+template <typename T, int VPT, int RING, bool SUMS>
+__global__ void __launch_bounds__(512, 1)
+layernorm_bwd_wide_kernel(int rows, int d, const T* __restrict__ da, const T* __restrict__ x,
+                          const float* __restrict__ mu_in, const float* __restrict__ rstd_in,
+                          const T* __restrict__ gamma, const T* __restrict__ add, T* __restrict__ dx,
+                          float* __restrict__ partial) {
+  fax_grid_dependency_wait();
+  constexpr int VN = Vec<T>::N;
+  constexpr int PER = 512 * VPT;
+  constexpr int NS = SUMS ? 4 : 2;
+  extern __shared__ uint4 ring_sm_raw[];
+  uint4* ring = ring_sm_raw;
+  __shared__ float2 red[2][16];
+  const int t = threadIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int nvec = d / VN;
+  const int stride = gridDim.x;
+  const float inv_d = 1.f / (float)d;
+  float ag[VPT][VN], ab[VPT][VN], aa[SUMS ? VPT : 1][VN], ao[SUMS ? VPT : 1][VN];
+  uint4 gm[VPT];
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) {
+#pragma unroll
+    for (int j = 0; j < VN; ++j) { ag[i][j] = 0.f; ab[i][j] = 0.f; if (SUMS) { aa[i][j] = 0.f; ao[i][j] = 0.f; } }
+    const int vi = t + 512 * i;
+    gm[i] = (vi < nvec) ? reinterpret_cast<const uint4*>(gamma)[vi] : make_uint4(0, 0, 0, 0);
+  }
+  auto issue = [&](int r, int slot) {
+    if (r < rows) {
+      uint4* s0 = ring + (size_t)slot * 3 * PER;
+      const uint4* dar = reinterpret_cast<const uint4*>(da + (size_t)r * d);
+      const uint4* xr = reinterpret_cast<const uint4*>(x + (size_t)r * d);
+      const uint4* adr = reinterpret_cast<const uint4*>(add + (size_t)r * d);
+#pragma unroll
+      for (int i = 0; i < VPT; ++i) {
+        const int vi = t + 512 * i;
+        if (vi < nvec) {
+          cp_async16(s0 + vi, dar + vi);
+          cp_async16(s0 + PER + vi, xr + vi);
+          if (add) cp_async16(s0 + 2 * PER + vi, adr + vi);
+        }
+      }
+    }
+    cp_async_commit();          // one group per call, empty past the last row, so the counting stays uniform
+  };
+  int row = blockIdx.x;
+#pragma unroll
+  for (int k = 0; k < RING - 1; ++k) issue(row + k * stride, k);
+  int slot = 0;
+  float mu_next = 0.f, rstd_next = 0.f;                                     // the row statistics, one row ahead
+  if (row < rows) { mu_next = mu_in[row]; rstd_next = rstd_in[row]; }
+  for (int it = 0; row < rows; row += stride, ++it) {
+    issue(row + (RING - 1) * stride, slot >= 1 ? slot - 1 : RING - 1);      // the slot read in the iteration before this one
+    const float mu = mu_next, rstd = rstd_next;
+    if (row + stride < rows) { mu_next = mu_in[row + stride]; rstd_next = rstd_in[row + stride]; }
+    cp_async_wait<RING - 1>();                                              // all but the newest groups: this row has landed
+    const uint4* s0 = ring + (size_t)slot * 3 * PER;
+    float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+      const int vi = t + 512 * i;
+      if (vi < nvec) {
+        float fd[VN], fx[VN], g[VN];
+        unpack<T>(s0[vi], fd); unpack<T>(s0[PER + vi], fx); unpack<T>(gm[i], g);
+#pragma unroll
+        for (int j = 0; j < VN; ++j) { const float u = fd[j] * g[j]; s1 += u; s2 += u * (fx[j] - mu) * rstd; }
+      }
+    }
+    s1 = warp_sum(s1); s2 = warp_sum(s2);
+    if (lane == 0) red[it & 1][warp] = make_float2(s1, s2);
+    __syncthreads();
+    s1 = 0.f; s2 = 0.f;
+#pragma unroll
+    for (int k = 0; k < 16; ++k) { const float2 v = red[it & 1][k]; s1 += v.x; s2 += v.y; }
+    const float c1 = s1 * inv_d, c2 = s2 * inv_d;
+#pragma unroll
+    for (int i = 0; i < VPT; ++i) {
+      const int vi = t + 512 * i;
+      if (vi < nvec) {
+        float fd[VN], fx[VN], g[VN], o[VN];
+        unpack<T>(s0[vi], fd); unpack<T>(s0[PER + vi], fx); unpack<T>(gm[i], g);
+#pragma unroll
+        for (int j = 0; j < VN; ++j) {
+          const float xh = (fx[j] - mu) * rstd;
+          o[j] = rstd * (fd[j] * g[j] - c1 - xh * c2);
+          ag[i][j] += fd[j] * xh;
+          ab[i][j] += fd[j];
+        }
+        if (add) {
+          float av[VN];
+          unpack<T>(s0[2 * PER + vi], av);
+#pragma unroll
+          for (int j = 0; j < VN; ++j) { o[j] += av[j]; if (SUMS) aa[i][j] += av[j]; }
+        }
+        if (SUMS) {
+#pragma unroll
+          for (int j = 0; j < VN; ++j) ao[i][j] += o[j];
+        }
+        store_vec<T>(dx + (size_t)row * d + vi * VN, o);
+      }
+    }
+    slot = (slot + 1 == RING) ? 0 : slot + 1;
+  }
+  cp_async_wait<0>();
+  float* slab = partial + (size_t)blockIdx.x * NS * d;
+#pragma unroll
+  for (int i = 0; i < VPT; ++i) {
+    const int vi = t + 512 * i;
+    if (vi < nvec) {
+#pragma unroll
+      for (int j = 0; j < VN; j += 4) {
+        *reinterpret_cast<float4*>(slab + vi * VN + j) = make_float4(ag[i][j], ag[i][j + 1], ag[i][j + 2], ag[i][j + 3]);
+        *reinterpret_cast<float4*>(slab + d + vi * VN + j) = make_float4(ab[i][j], ab[i][j + 1], ab[i][j + 2], ab[i][j + 3]);
+        if (SUMS) {
+          *reinterpret_cast<float4*>(slab + 2 * d + vi * VN + j) = make_float4(aa[i][j], aa[i][j + 1], aa[i][j + 2], aa[i][j + 3]);
+          *reinterpret_cast<float4*>(slab + 3 * d + vi * VN + j) = make_float4(ao[i][j], ao[i][j + 1], ao[i][j + 2], ao[i][j + 3]);
+        }
+      }
+    }
+  }
+}
+
 // Backward dx, one block per row (wide rows).
 template <typename T, int VPT>
 __global__ void __launch_bounds__(512)
@@ -547,11 +675,14 @@ int colreduce_slabs(fax_ctx* ctx, int rows, int nvec, int blocks_per_sm) {
 // Resident 256-thread blocks per SM: 8 for the plain column sum (32 registers), 5 for the
 // LayerNorm variant (48 registers).
 constexpr int kColsumBlocksPerSm = 8, kLnColBlocksPerSm = 5;
-// The fused backward covers rows of up to 512 vectors; one slab per block, one block per SM.
-bool ln_bwd_is_fused(int nvec) { return nvec <= 512; }
+// The fused backward covers rows of up to 2048 vectors (up to 512: row groups inside a block, above: one
+// row per block at a time); one slab per block, one block per SM.  The bias-gradient sums ride along up
+// to 1024 vectors (wider rows have no registers left for four sums per column).
+bool ln_bwd_is_fused(int nvec) { return nvec <= 2048; }
+bool ln_bwd_fuses_sums(int nvec) { return nvec <= 1024; }
 int ln_row_groups(int nvec) { return nvec <= 64 ? 16 : nvec <= 128 ? 8 : nvec <= 256 ? 4 : 2; }
 int ln_bwd_fused_grid(fax_ctx* ctx, int rows, int nvec) {
-  const int ng = ln_row_groups(nvec);
+  const int ng = nvec > 512 ? 1 : ln_row_groups(nvec);
   int grid = (rows + ng - 1) / ng;
   if (grid > ctx->sm_count) grid = ctx->sm_count;
   if (grid > 256) grid = 256;
@@ -623,6 +754,26 @@ fax_status ln_bwd_fused_t(fax_ctx* ctx, int rows, int d, const void* da, const v
   const int grid = ln_bwd_fused_grid(ctx, rows, nvec);
   const bool sums = sum_add && sum_out && add;
   const int ns = sums ? 4 : 2;
+  if (nvec > 512) {
+    // one row per block at a time: ring of R slots x 3 arrays x 512 * V vectors of 16 bytes
+#define LN_WIDE_S(V, R, S)                                                                             \
+    {                                                                                                  \
+      const size_t smem = (size_t)(R) * 3 * 512 * (V) * 16;                                            \
+      static bool attr_set[FAX_MAX_DEVICES] = {};                                                      \
+      FAX_TRY(fax_opt_in_shared_memory(ctx, layernorm_bwd_wide_kernel<T, V, R, S>, (int)smem, attr_set)); \
+      fax_launch(ctx, layernorm_bwd_wide_kernel<T, V, R, S>, dim3(grid), dim3(512), smem,              \
+                 rows, d, (const T*)da, (const T*)x, mu, rstd, (const T*)gamma, (const T*)add, (T*)dx, partial); \
+    }
+    if (nvec <= 1024) { if (sums) LN_WIDE_S(2, 3, true) else LN_WIDE_S(2, 3, false) }
+    else if (sums) return FAX_ERR_INVALID_ARG;
+    else if (nvec <= 1536) LN_WIDE_S(3, 3, false)
+    else LN_WIDE_S(4, 2, false)
+#undef LN_WIDE_S
+    FAX_TRY(fax_after_launch(ctx));
+    fax_launch(ctx, colreduce_fold_kernel, dim3((ns * d + 31) / 32), dim3(256), 0, grid, ns * d, d, (const float*)partial,
+               dgamma, dbeta, sum_add, sum_out, accumulate ? 1 : 0);
+    return fax_after_launch(ctx);
+  }
   // dynamic shared memory: 2 * d floats for the final reduction (rounded up to whole 16-byte vectors),
   // then the ring: 16 / W groups x LN_RING slots x 3 arrays x 32 * W * V vectors of 16 bytes; the
   // opt-in limit covers the widest row an instantiation serves (512 vectors)
@@ -693,9 +844,11 @@ fax_status fax_layernorm_bwd(fax_ctx* ctx, int prec, int rows, int d, const void
                              size_t partial_floats, float* sum_add, float* sum_out) {
   if (d % (prec == FAX_PREC_BF16 ? 8 : 4)) return FAX_ERR_UNSUPPORTED_SHAPE;
   const bool sums = sum_add && sum_out && add;
-  const bool fused = ln_bwd_is_fused(d / (prec == FAX_PREC_BF16 ? 8 : 4));
-  if (partial_floats < (size_t)(sums && fused ? 4 : 2) * ln_bwd_slabs(ctx, rows, d, prec) * d) return FAX_ERR_WORKSPACE_TOO_SMALL;
-  if (sums && !fused) {
+  const int nvec_all = d / (prec == FAX_PREC_BF16 ? 8 : 4);
+  const bool fused = ln_bwd_is_fused(nvec_all);
+  const bool fused_sums = fused && ln_bwd_fuses_sums(nvec_all);
+  if (partial_floats < (size_t)(sums && fused_sums ? 4 : 2) * ln_bwd_slabs(ctx, rows, d, prec) * d) return FAX_ERR_WORKSPACE_TOO_SMALL;
+  if (sums && !fused_sums) {
     // wide rows: the column sums of add and dx as reductions of their own, after the LayerNorm kernels
     FAX_TRY(fax_layernorm_bwd(ctx, prec, rows, d, da, x, mu, rstd, gamma, add, dx, dgamma, dbeta, accumulate, partial,
                               partial_floats, nullptr, nullptr));

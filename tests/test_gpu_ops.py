@@ -64,8 +64,13 @@ def test_adamw_many_tensors_and_bf16_grads(sess):
         assert relerr(host(tw), r) <= TOL_ADAMW
 
 
+# rows wider than 4096 bf16 / 2048 float elements take the one-row-per-block backward (2, 3 or 4 vectors per
+# thread); 20480 bf16 and 16384 float are past it (separate dx and column-sum kernels)
 @pytest.mark.parametrize("prec,rows,d", [(0, 256, 256), (0, 515, 768), (0, 64, 4096), (0, 33, 12288),
-                                         (1, 10, 8), (1, 300, 1000), (1, 17, 4096)])
+                                         (0, 300, 5120), (0, 515, 8192), (0, 161, 10240), (0, 310, 12288),
+                                         (0, 150, 16384), (0, 20, 20480),
+                                         (1, 10, 8), (1, 300, 1000), (1, 17, 4096), (1, 160, 2052), (1, 40, 8192),
+                                         (1, 9, 16384)])
 def test_layernorm_forward_backward(sess, prec, rows, d):
     rng = np.random.default_rng(rows + d)
     dt = torch.bfloat16 if prec == 0 else torch.float32
