@@ -225,11 +225,13 @@ fax_status fax_set_dependent_launch(fax_ctx* ctx, int32_t enable);
  * 8 row-tiles).  Results are bit-identical for every value.  Default: 48e6. */
 fax_status fax_set_gemm_l2_budget(fax_ctx* ctx, int64_t bytes);
 
-/* Attention backward at head_dim 128 walks the queries of a key tile in
- * sub-tiles of 64 with two of them in flight (the row warps work on one while
- * the tensor cores run the other's products); enable = 0 keeps the kernel with
- * one 128-query tile in flight, which also serves head_dim 64.  Same arithmetic
- * (the float32 dQ additions arrive in another order).  Default: enabled. */
+/* Which attention-backward kernel runs.  mode 0: one 128-query tile in flight,
+ * four row warps (head_dim 64 and 128).  mode 1: sixteen row warps with half-tile
+ * hand-offs (both head dims).  mode 2 (default): as 1, and at head_dim 64 the
+ * kernel that keeps two score tiles in flight (the exponentials of the next
+ * query tile run while the tensor core works on the current one).  Same
+ * arithmetic in every mode (the float32 dQ additions arrive in another order).
+ * Other values: FAX_ERR_INVALID_ARG. */
 fax_status fax_set_attention_backward_two_chains(fax_ctx* ctx, int32_t enable);
 
 /* One trainable tensor of a training state: float32 master, compute-precision

@@ -215,8 +215,8 @@ def fax_set_gemm_l2_budget(ctx, nbytes: int):
     _check(load_library().fax_set_gemm_l2_budget(ctx, int(nbytes)), "fax_set_gemm_l2_budget")
 
 
-def fax_set_attention_backward_two_chains(ctx, enable: bool):
-    _check(load_library().fax_set_attention_backward_two_chains(ctx, int(bool(enable))),
+def fax_set_attention_backward_two_chains(ctx, mode: int):
+    _check(load_library().fax_set_attention_backward_two_chains(ctx, int(mode)),
            "fax_set_attention_backward_two_chains")
 
 

@@ -40,7 +40,7 @@ extern "C" fax_status fax_create(fax_ctx** out, int32_t device_ordinal, void* cu
   c->overlap_adamw = true;
   c->use_2cta = true;
   c->use_pdl = true;
-  c->attn_bwd_two_chains = true;
+  c->attn_bwd_mode = 2;
   c->gemm_l2_budget = 48e6;
   c->use_graphs = true;
   c->fused_update = false;
@@ -158,7 +158,8 @@ extern "C" fax_status fax_set_gemm_l2_budget(fax_ctx* ctx, int64_t bytes) {
 
 extern "C" fax_status fax_set_attention_backward_two_chains(fax_ctx* ctx, int32_t enable) {
   if (!ctx) return FAX_ERR_INVALID_ARG;
-  ctx->attn_bwd_two_chains = enable != 0;
+  if (enable < 0 || enable > 2) return FAX_ERR_INVALID_ARG;
+  ctx->attn_bwd_mode = enable;
   cudaStreamSynchronize(ctx->stream);
   fax_graph_clear(ctx);
   return FAX_OK;

@@ -10,6 +10,13 @@
 // operand from tensor memory.  The CTA loops over its share of the work list (heaviest pairs
 // first); the next pair's Q, K and V tiles are requested as soon as their buffers are free, so
 // the set-up of one pair hides under the tail of the one before.  Every wait is bounded.
+//
+// head_dim 64 leaves 128 tensor-memory columns free, which hold P beside S (EARLY_S): a group's softmax
+// threads signal "S read" as soon as the scores are in registers, the MMA thread issues the NEXT key
+// tile's S product right then, and the group goes from one tile's softmax straight into the next
+// without waiting for a product.  With that the exponentials (1024 clocks of the special-function
+// units per 128 x 128 tile, more than the tile's 876 tensor-core clocks at head_dim 64) are the bound;
+// before, each group's loop was softmax + both products + the hand-offs, about 2900 clocks per tile.
 #include "tc_common.cuh"
 
 namespace {
@@ -34,10 +41,13 @@ template <int HD> struct Fwd2Cfg {
   static constexpr int BAR_OFF = V_OFF + NS * TILE_BYTES;
   static constexpr int SMEM_BYTES = BAR_OFF + 512 + 1024;
   static constexpr int TMEM_COLS = 512;                  // S_A [0,128) S_B [128,256) O_A [256,..) O_B [384,..)
+  static constexpr bool EARLY_S = (HD == 64);            // then O_A [256,320) O_B [320,384) P_A [384,448) P_B [448,512)
+  static constexpr int O_STRIDE = EARLY_S ? 64 : 128;
   // barriers
-  static constexpr int QFULL = 0, QFREE = 2, SFULL = 4, PREADY = 6, OFULL = 8, OFREE = 10;
-  static constexpr int KFULL = 12, KFREE = KFULL + NS, VFULL = KFREE + NS, VFREE = VFULL + NS;
+  static constexpr int QFULL = 0, QFREE = 2, SFULL = 4, PREADY = 6, OFULL = 8, OFREE = 10, SREAD = 12, PFREE = 14;
+  static constexpr int KFULL = 16, KFREE = KFULL + NS, VFULL = KFREE + NS, VFREE = VFULL + NS;
   static constexpr int NBARS = VFREE + NS;
+  static_assert(NBARS <= 32, "barrier area");
 };
 
 template <int HD>
@@ -69,7 +79,8 @@ attn_fwd2_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnFwd2Para
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < C_::NBARS; ++i) {
-      const bool four = (i == C_::PREADY || i == C_::PREADY + 1 || i == C_::OFREE || i == C_::OFREE + 1);
+      const bool four = (i == C_::PREADY || i == C_::PREADY + 1 || i == C_::OFREE || i == C_::OFREE + 1 ||
+                         i == C_::SREAD || i == C_::SREAD + 1);
       mbar_init(bar(i), four ? 4u : 1u);
     }
     *abort_flag = 0;
@@ -128,6 +139,7 @@ attn_fwd2_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnFwd2Para
       auto mk = [&](uint32_t lo) -> uint64_t { return ((uint64_t)d_hi << 32) | lo; };
       uint32_t kc0 = 0;                 // K / V tiles of the pairs before this one
       uint32_t pc[2] = {0u, 0u};        // P tiles consumed per query tile
+      uint32_t ns[2] = {0u, 0u};        // S tiles issued per query tile
       bool ok = true;
       int it = 0;
       for (int t = blockIdx.x; t < n_items && ok; t += gridDim.x, ++it) {
@@ -138,6 +150,9 @@ attn_fwd2_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnFwd2Para
         auto issue_s = [&](int x, int j) -> bool {
           const uint32_t c = kc0 + (uint32_t)j;
           const int s = (int)(c % NS);
+          if (C_::EARLY_S && ns[x] > 0 &&
+              !mbar_wait(bar(C_::SREAD + x), (ns[x] - 1u) & 1u, abort_flag, p.status, 232)) return false;
+          ++ns[x];
           if (!mbar_wait(bar(C_::KFULL + s), (c / NS) & 1u, abort_flag, p.status, 224)) return false;
           tc_fence_after();
           const uint32_t qlo = q_lo0 + (uint32_t)x * TILE16, klo = k_lo0 + (uint32_t)s * TILE16;
@@ -158,10 +173,12 @@ attn_fwd2_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnFwd2Para
           tc_fence_after();
           const int s = (int)((kc0 + (uint32_t)j) % NS);
           const uint32_t vlo = v_lo0 + (uint32_t)s * TILE16;
-          const uint32_t dst = tmem + 256u + (uint32_t)(x * 128), src = tmem + (uint32_t)(x * 128);
+          const uint32_t dst = tmem + 256u + (uint32_t)(x * C_::O_STRIDE);
+          const uint32_t src = C_::EARLY_S ? tmem + 384u + (uint32_t)(x * 64) : tmem + (uint32_t)(x * 128);
 #pragma unroll
           for (int k = 0; k < 8; ++k)
             tc_mma_bf16_ts(dst, src + 8 * k, mk(vlo + k * 128), idesc_o, (j | k) ? 1u : 0u);
+          if (C_::EARLY_S) tc_commit(bar(C_::PFREE + x));
           return true;
         };
         if (!mbar_wait(bar(C_::QFULL), iph, abort_flag, p.status, 227)) { ok = false; break; }
@@ -173,6 +190,27 @@ attn_fwd2_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnFwd2Para
         for (int j = 0; j < nkv && ok; ++j) {
           const uint32_t c = kc0 + (uint32_t)j;
           const int s = (int)(c % NS);
+          if (C_::EARLY_S) {
+            // the next key tile's scores first (they wait only for "S read"), then this tile's P V products
+            if (j + 1 <= lastA) {
+              if (!issue_s(0, j + 1)) { ok = false; break; }
+              if (j + 1 == lastA) tc_commit(bar(C_::QFREE));
+            }
+            if (j + 1 <= lastB) {
+              if (!issue_s(1, j + 1)) { ok = false; break; }
+              tc_commit(bar(C_::KFREE + (int)((c + 1) % NS)));
+              if (j + 1 == lastB) tc_commit(bar(C_::QFREE + 1));
+            }
+            if (!mbar_wait(bar(C_::VFULL + s), (c / NS) & 1u, abort_flag, p.status, 229)) { ok = false; break; }
+            if (j <= lastA) {
+              if (!issue_pv(0, j)) { ok = false; break; }
+              if (j == lastA) tc_commit(bar(C_::OFULL));
+            }
+            if (!issue_pv(1, j)) { ok = false; break; }
+            tc_commit(bar(C_::VFREE + s));
+            if (j == lastB) tc_commit(bar(C_::OFULL + 1));
+            continue;
+          }
           if (!mbar_wait(bar(C_::VFULL + s), (c / NS) & 1u, abort_flag, p.status, 229)) { ok = false; break; }
           if (j <= lastA) {
             if (!issue_pv(0, j)) { ok = false; break; }
@@ -200,7 +238,8 @@ attn_fwd2_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnFwd2Para
     const int r = 32 * wq + lane;
     const uint32_t lane_base = (uint32_t)(32 * wq) << 16;
     const uint32_t tm_s = tmem + (uint32_t)(x * 128) + lane_base;
-    const uint32_t tm_o = tmem + 256u + (uint32_t)(x * 128) + lane_base;
+    const uint32_t tm_o = tmem + 256u + (uint32_t)(x * C_::O_STRIDE) + lane_base;
+    const uint32_t tm_p = C_::EARLY_S ? tmem + 384u + (uint32_t)(x * 64) + lane_base : tm_s;
     uint32_t sc = 0;                  // S tiles consumed
     bool ok = true;
     int it = 0;
@@ -216,6 +255,13 @@ attn_fwd2_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnFwd2Para
 #pragma unroll
         for (int c = 0; c < 4; ++c) tc_ld32(tm_s + (uint32_t)(32 * c), sv[c]);
         tc_wait_ld();
+        if (C_::EARLY_S) {
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar(C_::SREAD + x));       // the next key tile's scores may overwrite S
+        }
+        // EARLY_S: P V of the tile before (global count sc - 1) must be complete before O is rescaled or P overwritten
+        bool pv_done = !C_::EARLY_S || sc == 0;
         if (j == qx) {
 #pragma unroll
           for (int c = 0; c < 4; ++c)
@@ -231,10 +277,15 @@ attn_fwd2_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnFwd2Para
             mxa[(e >> 1) & 3] = max3(mxa[(e >> 1) & 3], __uint_as_float(sv[c][e]), __uint_as_float(sv[c][e + 1]));
         const float mx = fmaxf(fmaxf(mxa[0], mxa[1]), fmaxf(mxa[2], mxa[3]));
         const float m_new = fmaxf(m_used, mx * p.scale_log2);
-        // O is rescaled only when a row maximum of the warp has grown by more than 2^8; S_j complete
-        // implies P V of tile j-1 complete (the MMA thread issues them in that order)
+        // O is rescaled only when a row maximum of the warp has grown by more than 2^8.  Without EARLY_S,
+        // S_j complete implies P V of tile j-1 complete (the MMA thread issues them in that order)
         if (__any_sync(0xffffffffu, m_new > m_used + 8.0f)) {
           if (j > 0) {
+            if (!pv_done) {
+              if (!mbar_wait_warp(bar(C_::PFREE + x), (sc - 1u) & 1u, abort_flag, p.status, 233)) { ok = false; break; }
+              tc_fence_after();
+              pv_done = true;
+            }
             const float factor = ex2_approx(m_used - m_new);
             l *= factor;
 #pragma unroll 1
@@ -263,8 +314,14 @@ attn_fwd2_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnFwd2Para
               __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
               packed[16 * cc + (e >> 1)] = *reinterpret_cast<uint32_t*>(&h2);
             }
-          tc_st32(tm_s + (uint32_t)(32 * half), packed);
+          if (half == 0 && !pv_done) {
+            if (!mbar_wait_warp(bar(C_::PFREE + x), (sc - 1u) & 1u, abort_flag, p.status, 233)) { ok = false; break; }
+            tc_fence_after();
+            pv_done = true;
+          }
+          tc_st32(tm_p + (uint32_t)(32 * half), packed);
         }
+        if (!ok) break;
         l += rowsum;
         tc_wait_st();
         tc_fence_before();

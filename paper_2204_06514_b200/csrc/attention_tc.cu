@@ -752,7 +752,9 @@ fax_status launch_bwd(fax_ctx* ctx, int B, int T, int H, const void* qkv, const 
   p.scale = 1.0f / sqrtf((float)HD);
   p.scale_log2 = 1.4426950408889634f * p.scale;
   p.status = ctx->dev_status;
-  if (ctx->attn_bwd_two_chains && fax_attention_bwd3_supported(B, T, H, HD)) {
+  if (ctx->attn_bwd_mode >= 2 && fax_attention_bwd4_supported(B, T, H, HD)) {
+    FAX_TRY(fax_attention_bwd4_tc(ctx, B, T, H, HD, qkv, lse, d_o, dqkv, Dv, dq_acc));
+  } else if (ctx->attn_bwd_mode >= 1 && fax_attention_bwd3_supported(B, T, H, HD)) {
     FAX_TRY(fax_attention_bwd3_tc(ctx, B, T, H, HD, qkv, lse, d_o, dqkv, Dv, dq_acc));
   } else {
     static bool attr_set[FAX_MAX_DEVICES] = {};

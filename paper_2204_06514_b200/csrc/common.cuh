@@ -61,7 +61,7 @@ struct fax_ctx {
   bool use_2cta;             // GEMMs whose M and N are multiples of 256 use the two-CTA kernel
   bool use_pdl;              // kernels are launched with programmatic stream serialization allowed
   double gemm_l2_budget;     // bytes of L2 a GEMM may count on for the operand panels it keeps between waves (0: fixed raster)
-  bool attn_bwd_two_chains;  // attention backward runs the sixteen-row-warp kernel (half-tile hand-offs)
+  int attn_bwd_mode;         // attention backward: 0 one-tile kernel, 1 sixteen row warps, 2 also two score tiles in flight at head_dim 64
 };
 
 // Brackets the launches of one operator with CUDA events while profiling is on.
@@ -306,6 +306,9 @@ bool fax_attention_fwd2_supported(int B, int T, int H, int hd);
 fax_status fax_attention_fwd2_tc(fax_ctx* ctx, int B, int T, int H, int hd, const void* qkv, void* o, float* lse);
 size_t fax_attention_bwd_tc_scratch_bytes(int B, int T, int H, int hd);
 // backward with sixteen row warps and half-tile hand-offs (the main kernel only; see its definition)
+bool fax_attention_bwd4_supported(int B, int T, int H, int hd);
+fax_status fax_attention_bwd4_tc(fax_ctx* ctx, int B, int T, int H, int hd, const void* qkv, const float* lse,
+                                 const void* d_o, void* dqkv, const float* Dv, float* dq_acc);
 bool fax_attention_bwd3_supported(int B, int T, int H, int hd);
 fax_status fax_attention_bwd3_tc(fax_ctx* ctx, int B, int T, int H, int hd, const void* qkv, const float* lse,
                                  const void* d_o, void* dqkv, const float* Dv, float* dq_acc);

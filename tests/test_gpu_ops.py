@@ -356,11 +356,12 @@ def test_attention_forward_backward(sess, prec, B, T, H, hd):
     assert st == fx.FAX_OK
 
 
-def test_attention_backward_kernels_agree(sess):
-    """head_dim 128 has two backward kernels (half-tile hand-offs, and the older single hand-off one
-    that also serves head_dim 64): the same inputs through both, each against the oracle."""
-    B, T, H, hd = 2, 640, 5, 128
-    rng = np.random.default_rng(77)
+@pytest.mark.parametrize("B,T,H,hd", [(2, 640, 5, 128), (2, 640, 6, 64), (1, 1152, 3, 64)])
+def test_attention_backward_kernels_agree(sess, B, T, H, hd):
+    """The three backward kernels (mode 2: two score tiles in flight at head_dim 64; mode 1: sixteen row
+    warps with half-tile hand-offs; mode 0: the single hand-off kernel): the same inputs through each,
+    each against the oracle."""
+    rng = np.random.default_rng(77 + hd + T)
     d = H * hd
     qkv = synth.round_to_bf16(rng.standard_normal((B * T, 3 * d)).astype(np.float32))
     do = synth.round_to_bf16(rng.standard_normal((B * T, d)).astype(np.float32))
@@ -373,7 +374,7 @@ def test_attention_backward_kernels_agree(sess):
     nb = ops.fax_op_attention_backward_scratch_bytes(0, B, T, H, hd)
     scratch = sess.arena(nb)
     try:
-        for enable in (1, 0):
+        for enable in (2, 1, 0):
             fx.fax_set_attention_backward_two_chains(sess.ctx, enable)
             dqkv = torch.full_like(tq, float("nan"))
             ops.fax_op_attention_backward(sess.ctx, 0, B, T, H, hd, ptr(tq), ptr(o), ptr(lse), ptr(tdo), ptr(dqkv),
@@ -382,6 +383,6 @@ def test_attention_backward_kernels_agree(sess):
             for i, name in enumerate("qkv"):
                 assert relerr(got[:, i * d:(i + 1) * d], rd[:, i * d:(i + 1) * d]) <= TOL_GRAD_BF16, (enable, name)
     finally:
-        fx.fax_set_attention_backward_two_chains(sess.ctx, 1)
+        fx.fax_set_attention_backward_two_chains(sess.ctx, 2)
     st, _ = fx.fax_check_device_status(sess.ctx)
     assert st == fx.FAX_OK
