@@ -19,9 +19,12 @@
 // of phase n + 1 depends, through another barrier, on the consumer having passed phase n); "P ready"
 // alternates between two barriers because at the start of a key tile two S^T products are issued
 // before the first of them is waited for.
-// Shared memory: K, V, three Q stages (a Q tile lives from S^T, two iterations ahead, to dK), two dO
-// stages, the dS tile (B operand of dQ), two 32 KB dQ staging buffers, per-stage query statistics.
-// Every wait is bounded.
+// K and V of the next key tile are prefetched into a second buffer while the current one is walked, and
+// the MMA thread issues the next key tile's first two S^T products right after the last products of the
+// current one, so the row warps find their scores ready when they come back from the dV / dK read-out.
+// Shared memory: two (K, V) buffers, three Q stages (a Q tile lives from S^T, two iterations ahead, to
+// dK), two dO stages, the dS tile (B operand of dQ), a 32 KB dQ staging buffer, per-stage query
+// statistics.  Every wait is bounded.
 #include "tc_common.cuh"
 
 namespace {
@@ -42,16 +45,16 @@ struct Bwd4Params {
 
 struct B4 {
   static constexpr int TILE_BYTES = 128 * B4_HD * 2;      // one panel of 128 rows x 128 B
-  static constexpr int K_OFF = 0, V_OFF = TILE_BYTES;
-  static constexpr int Q_OFF = 2 * TILE_BYTES;            // three stages
-  static constexpr int DO_OFF = 5 * TILE_BYTES;           // two stages
-  static constexpr int DS_OFF = 7 * TILE_BYTES;           // dS^T: two panels (query halves) of 128 key rows x 128 B
-  static constexpr int STG_OFF = DS_OFF + 32768;          // two dQ staging buffers: 4 boxes of 64 rows x 32 floats each
-  static constexpr int STAT_OFF = STG_OFF + 2 * 32768;    // [3 stages][0: log2e * lse, 1: D][128] floats
+  static constexpr int KV_OFF = 0;                        // two buffers of (K, V): the next key tile is prefetched
+  static constexpr int Q_OFF = 4 * TILE_BYTES;            // three stages
+  static constexpr int DO_OFF = 7 * TILE_BYTES;           // two stages
+  static constexpr int DS_OFF = 9 * TILE_BYTES;           // dS^T: two panels (query halves) of 128 key rows x 128 B
+  static constexpr int STG_OFF = DS_OFF + 32768;          // dQ staging: 4 boxes of 64 rows x 32 floats
+  static constexpr int STAT_OFF = STG_OFF + 32768;        // [3 stages][0: log2e * lse, 1: D][128] floats
   static constexpr int BAR_OFF = STAT_OFF + 3 * 1024;
-  static constexpr int KVFULL = 0, KVFREE = 1, QFULL = 2 /* 3 */, QFREE = 5 /* 3 */, DOFULL = 8 /* 2 */, DOFREE = 10 /* 2 */,
-                       SFULL = 12 /* 2 */, DPFULL = 14, PREADY = 15 /* 2 */, DSREADY = 17, DQFULL = 18, DQREAD = 19,
-                       STGFULL = 20 /* 2 */, STGFREE = 22 /* 2 */, ALLDONE = 24, DKVREAD = 25, NBARS = 26;
+  static constexpr int KVFULL = 0 /* 2 */, KVFREE = 2 /* 2 */, QFULL = 4 /* 3 */, QFREE = 7 /* 3 */, DOFULL = 10 /* 2 */,
+                       DOFREE = 12 /* 2 */, SFULL = 14 /* 2 */, DPFULL = 16, PREADY = 17 /* 2 */, DSREADY = 19, DQFULL = 20,
+                       DQREAD = 21, STGFULL = 22, STGFREE = 23, ALLDONE = 24, DKVREAD = 25, NBARS = 26;
   static constexpr int LAYOUT_BYTES = BAR_OFF + NBARS * 8 + 16;
   static constexpr int SMEM_BYTES = LAYOUT_BYTES + 1024;
   static constexpr int TMEM_COLS = 512;
@@ -81,7 +84,7 @@ attn_bwd4_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_c
   if (threadIdx.x == 0) {
     for (int i = 0; i < C_::NBARS; ++i) {
       uint32_t count = 1;
-      if (i == C_::PREADY || i == C_::PREADY + 1 || i == C_::DSREADY || i == C_::DQREAD || i == C_::DKVREAD || i == C_::STGFULL || i == C_::STGFULL + 1)
+      if (i == C_::PREADY || i == C_::PREADY + 1 || i == C_::DSREADY || i == C_::DQREAD || i == C_::DKVREAD || i == C_::STGFULL)
         count = B4_ROW_WARPS;
       if (i >= C_::QFULL && i < C_::QFULL + 3) count = 2;       // the tile's bytes and its statistics
       mbar_init(bar(i), count);
@@ -100,10 +103,11 @@ attn_bwd4_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_c
   fax_grid_dependency_wait();
   auto tm_s = [&](uint32_t g) { return tmem + 128u * (g & 1u); };
   const uint32_t tm_dp = tmem + 256, tm_dv = tmem + 384, tm_dk = tmem + 448;
-  const uint32_t k_s = base + C_::K_OFF, v_s = base + C_::V_OFF, ds_s = base + C_::DS_OFF;
+  const uint32_t ds_s = base + C_::DS_OFF, stg_s = base + C_::STG_OFF;
+  auto k_s = [&](uint32_t i) { return base + C_::KV_OFF + 2 * i * C_::TILE_BYTES; };
+  auto v_s = [&](uint32_t i) { return base + C_::KV_OFF + (2 * i + 1) * C_::TILE_BYTES; };
   auto q_s = [&](uint32_t i) { return base + C_::Q_OFF + i * C_::TILE_BYTES; };
   auto do_s = [&](uint32_t i) { return base + C_::DO_OFF + i * C_::TILE_BYTES; };
-  auto stg_s = [&](uint32_t i) { return base + C_::STG_OFF + i * 32768u; };
   float* stat = reinterpret_cast<float*>(gbase + C_::STAT_OFF);
 
   if (warp == B4_ROW_WARPS + 1) {
@@ -113,16 +117,32 @@ attn_bwd4_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_c
       const int kj = t / bh_count, bh = t % bh_count;
       return reinterpret_cast<const float4*>(src + (long long)bh * p.T + (kj + it) * 128) + lane;
     };
+    // K, V of work item t (the CTA's item number n) into buffer n & 1, free once item n - 2 has finished
+    auto load_kv = [&](int t, int n) -> bool {
+      const uint32_t kb = (uint32_t)n & 1u;
+      if (!mbar_wait_warp(bar(C_::KVFREE + kb), (((uint32_t)n >> 1) & 1u) ^ 1u, abort_flag, p.status, 441)) return false;
+      if (lane == 0) {
+        const int kj = t / bh_count, bh = t % bh_count;
+        const int b = bh / p.H, h = bh % p.H;
+        mbar_expect_tx(bar(C_::KVFULL + kb), 2 * C_::TILE_BYTES);
+        tma_load_2d(k_s(kb), &tmap_qkv, bar(C_::KVFULL + kb), d + h * HD, b * p.T + kj * 128);
+        tma_load_2d(v_s(kb), &tmap_qkv, bar(C_::KVFULL + kb), 2 * d + h * HD, b * p.T + kj * 128);
+      }
+      return true;
+    };
     uint32_t gs = 0;
     bool ok = true;
     int it_n = 0;
     float4 l_next = make_float4(0.f, 0.f, 0.f, 0.f), d_next = l_next;
-    if ((int)blockIdx.x < n_items) { l_next = *stat_ptr(p.lse, blockIdx.x, 0); d_next = *stat_ptr(p.Dv, blockIdx.x, 0); }
+    if ((int)blockIdx.x < n_items) {
+      l_next = *stat_ptr(p.lse, blockIdx.x, 0); d_next = *stat_ptr(p.Dv, blockIdx.x, 0);
+      ok = load_kv(blockIdx.x, 0);
+    }
     for (int t = blockIdx.x; t < n_items && ok; t += gridDim.x, ++it_n) {
       const int kj = t / bh_count, bh = t % bh_count;
       const int b = bh / p.H, h = bh % p.H;
       const int row0 = b * p.T;
-      const int qcol = h * HD, kcol = d + h * HD, vcol = 2 * d + h * HD;
+      const int qcol = h * HD;
       const int nsteps = nq - kj;
       for (int it = 0; it < nsteps; ++it, ++gs) {
         const int qrow = row0 + (kj + it) * 128;
@@ -131,14 +151,6 @@ attn_bwd4_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_c
         const float4 d_cur = d_next;
         if (it + 1 < nsteps) { l_next = *stat_ptr(p.lse, t, it + 1); d_next = *stat_ptr(p.Dv, t, it + 1); }
         else if (t + (int)gridDim.x < n_items) { l_next = *stat_ptr(p.lse, t + gridDim.x, 0); d_next = *stat_ptr(p.Dv, t + gridDim.x, 0); }
-        if (it == 0) {
-          if (!mbar_wait_warp(bar(C_::KVFREE), (uint32_t)(it_n & 1) ^ 1u, abort_flag, p.status, 441)) { ok = false; break; }
-          if (lane == 0) {
-            mbar_expect_tx(bar(C_::KVFULL), 2 * C_::TILE_BYTES);
-            tma_load_2d(k_s, &tmap_qkv, bar(C_::KVFULL), kcol, row0 + kj * 128);
-            tma_load_2d(v_s, &tmap_qkv, bar(C_::KVFULL), vcol, row0 + kj * 128);
-          }
-        }
         if (!mbar_wait_warp(bar(C_::QFREE + s3), (u3 & 1u) ^ 1u, abort_flag, p.status, 442)) { ok = false; break; }
         if (lane == 0) {
           mbar_expect_tx(bar(C_::QFULL + s3), C_::TILE_BYTES);
@@ -154,6 +166,8 @@ attn_bwd4_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_c
           mbar_expect_tx(bar(C_::DOFULL + s2), C_::TILE_BYTES);
           tma_load_2d(do_s(s2), &tmap_do, bar(C_::DOFULL + s2), qcol, qrow);
         }
+        // K, V of the next key tile, once this one's second query tile is requested (the first, if it has one)
+        if (it == (nsteps > 1 ? 1 : 0) && t + (int)gridDim.x < n_items && !load_kv(t + gridDim.x, it_n + 1)) { ok = false; break; }
       }
     }
     if (!ok && lane == 0) { const long long t0 = clock64(); while (clock64() - t0 < 2000000LL) { } }
@@ -167,8 +181,9 @@ attn_bwd4_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_c
       // changes between stages and k-steps.  K-major tiles: a k-step is 32 bytes inside the 64-column
       // panel; MN-major: a k-step is 16 rows (2048 bytes).
       const uint32_t hi = (uint32_t)(smem_desc(0, 16, 1024) >> 32);
-      const uint32_t k_kmaj = (uint32_t)smem_desc(k_s, 16, 1024), v_kmaj = (uint32_t)smem_desc(v_s, 16, 1024);
-      const uint32_t k_mn = (uint32_t)smem_desc(k_s, 16384, 1024), ds_mn = (uint32_t)smem_desc(ds_s, 16384, 1024);
+      const uint32_t k_kmaj0 = (uint32_t)smem_desc(k_s(0), 16, 1024), v_kmaj0 = (uint32_t)smem_desc(v_s(0), 16, 1024);
+      const uint32_t k_mn0 = (uint32_t)smem_desc(k_s(0), 16384, 1024), ds_mn = (uint32_t)smem_desc(ds_s, 16384, 1024);
+      uint32_t k_kmaj = k_kmaj0, v_kmaj = v_kmaj0, k_mn = k_mn0;      // of the key tile being walked
       const uint32_t q_kmaj0 = (uint32_t)smem_desc(q_s(0), 16, 1024), q_mn0 = (uint32_t)smem_desc(q_s(0), 16384, 1024);
       const uint32_t do_kmaj0 = (uint32_t)smem_desc(do_s(0), 16, 1024), do_mn0 = (uint32_t)smem_desc(do_s(0), 16384, 1024);
       auto mk = [&](uint32_t lo) -> uint64_t { return ((uint64_t)hi << 32) | lo; };
@@ -176,13 +191,13 @@ attn_bwd4_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_c
       // A k-step of P^T / dS^T in tensor memory: 16 queries = 8 columns inside the quarter's 32
       auto acol = [](int k) { return (uint32_t)(32 * (k / 2) + 8 * (k % 2)); };
       bool ok = true;
-      auto issue_s = [&](uint32_t g) -> bool {
+      auto issue_s = [&](uint32_t g, uint32_t kk) -> bool {         // kk: K (K-major words) of the key tile that tile g belongs to
         const uint32_t s3 = g % 3u;
         if (!mbar_wait(bar(C_::QFULL + s3), (g / 3u) & 1u, abort_flag, p.status, 444)) return false;
         tc_fence_after();
         const uint32_t bq = q_kmaj0 + s3 * TILE16;
 #pragma unroll
-        for (int s = 0; s < HD / 16; ++s) tc_mma_bf16(tm_s(g), mk(k_kmaj + s * 2), mk(bq + s * 2), idesc_s, s ? 1u : 0u);
+        for (int s = 0; s < HD / 16; ++s) tc_mma_bf16(tm_s(g), mk(kk + s * 2), mk(bq + s * 2), idesc_s, s ? 1u : 0u);
         tc_commit(bar(C_::SFULL + (g & 1u)));
         return true;
       };
@@ -208,12 +223,19 @@ attn_bwd4_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_c
       };
       uint32_t gs = 0;
       int it_n = 0;
+      // S^T of the first two query tiles of work item t (number n of this CTA, first tile g), K from buffer n & 1
+      auto open_item = [&](int t, int n, uint32_t g) -> bool {
+        const uint32_t kb = (uint32_t)n & 1u;
+        if (!mbar_wait(bar(C_::KVFULL + kb), ((uint32_t)n >> 1) & 1u, abort_flag, p.status, 449)) return false;
+        const uint32_t kk = k_kmaj0 + kb * 2 * TILE16;
+        return issue_s(g, kk) && (nq - t / bh_count < 2 || issue_s(g + 1, kk));
+      };
+      if ((int)blockIdx.x < n_items && !open_item(blockIdx.x, 0, 0)) ok = false;
       for (int t = blockIdx.x; t < n_items && ok; t += gridDim.x, ++it_n) {
         const int kj = t / bh_count;
         const uint32_t nsteps = (uint32_t)(nq - kj);
-        if (!mbar_wait(bar(C_::KVFULL), (uint32_t)(it_n & 1), abort_flag, p.status, 449)) { ok = false; break; }
-        if (!issue_s(gs)) { ok = false; break; }
-        if (nsteps > 1 && !issue_s(gs + 1)) { ok = false; break; }
+        const uint32_t kb = (uint32_t)it_n & 1u;
+        k_kmaj = k_kmaj0 + kb * 2 * TILE16; v_kmaj = v_kmaj0 + kb * 2 * TILE16; k_mn = k_mn0 + kb * 2 * TILE16;
         // the first dV product of a key tile overwrites: dV and dK of the tile before must have been read out
         if (!mbar_wait(bar(C_::DKVREAD), (uint32_t)(it_n & 1) ^ 1u, abort_flag, p.status, 450)) { ok = false; break; }
         if (!issue_dv(gs, true)) { ok = false; break; }
@@ -230,11 +252,13 @@ attn_bwd4_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_c
           for (int k = 0; k < 8; ++k) tc_mma_bf16_ts(tm_dk, tm_s(gs) + 16u + acol(k), mk(bq + k * 128), idesc_acc, (it | (uint32_t)k) ? 1u : 0u);
           tc_commit(bar(C_::QFREE + gs % 3u));
           if (it + 1 == nsteps) {
-            tc_commit(bar(C_::KVFREE));
+            tc_commit(bar(C_::KVFREE + kb));
             tc_commit(bar(C_::ALLDONE));         // every product of this key tile is complete: dV and dK are final
+            // the next key tile's first scores, ready when the row warps come back from the read-out
+            if (t + (int)gridDim.x < n_items && !open_item(t + gridDim.x, it_n + 1, gs + 1)) { ok = false; break; }
             continue;
           }
-          if (it + 2 < nsteps && !issue_s(gs + 2)) { ok = false; break; }
+          if (it + 2 < nsteps && !issue_s(gs + 2, k_kmaj)) { ok = false; break; }
           if (!issue_dp(gs + 1)) { ok = false; break; }
           if (it + 2 < nsteps && !issue_dv(gs + 2, false)) { ok = false; break; }
         }
@@ -251,16 +275,13 @@ attn_bwd4_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_c
         const int nsteps = nq - kj;
         for (int it = 0; it < nsteps; ++it, ++gs) {
           const int qrow = b * p.T + (kj + it) * 128;
-          const uint32_t sb = gs & 1u;
-          if (!mbar_wait(bar(C_::STGFULL + sb), (gs >> 1) & 1u, abort_flag, p.status, 451)) { ok = false; break; }
+          if (!mbar_wait(bar(C_::STGFULL), gs & 1u, abort_flag, p.status, 451)) { ok = false; break; }
 #pragma unroll
           for (int i = 0; i < 4; ++i)             // boxes of 64 rows x 32 floats: (row half i / 2, column half i % 2)
-            tma_reduce_add_2d(&tmap_dq, stg_s(sb) + i * 8192, h * HD + 32 * (i & 1), qrow + 64 * (i >> 1));
+            tma_reduce_add_2d(&tmap_dq, stg_s + i * 8192, h * HD + 32 * (i & 1), qrow + 64 * (i >> 1));
           bulk_commit_group();
-          if (gs > 0) {                           // the group before this one has read the other buffer
-            asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-            mbar_arrive(bar(C_::STGFREE + (sb ^ 1u)));
-          }
+          bulk_wait_read_all();                   // the buffer has been read: the next tile may be staged
+          mbar_arrive(bar(C_::STGFREE));
         }
       }
       bulk_wait_all();
@@ -312,8 +333,8 @@ attn_bwd4_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_c
       if (lane == 0) mbar_arrive(bar(C_::PREADY + (g & 1u)));
       return true;
     };
-    // C: dQ of tile g (lane = query row kr, columns 16 qr .. 16 qr + 15) -> staging buffer g & 1 as four
-    // boxes of 64 rows x 32 floats (row half, column half)
+    // C: dQ of tile g (lane = query row kr, columns 16 qr .. 16 qr + 15) -> the staging buffer as four boxes
+    // of 64 rows x 32 floats (row half, column half)
     auto phase_dq = [&](uint32_t g) -> bool {
       if (!mbar_wait_warp(bar(C_::DQFULL), g & 1u, abort_flag, p.status, 455)) return false;
       tc_fence_after();
@@ -323,16 +344,17 @@ attn_bwd4_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_c
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar(C_::DQREAD));
-      if (!mbar_wait_warp(bar(C_::STGFREE + (g & 1u)), ((g >> 1) & 1u) ^ 1u, abort_flag, p.status, 456)) return false;
+      // the reduction of the tile before has read the buffer
+      if (g > 0 && !mbar_wait_warp(bar(C_::STGFREE), (g - 1u) & 1u, abort_flag, p.status, 456)) return false;
       const int r = kr & 63;
-      uint8_t* box = gbase + C_::STG_OFF + (g & 1u) * 32768u + (2u * ((uint32_t)kr >> 6) + (qr >> 1)) * 8192u + r * 128;
+      uint8_t* box = gbase + C_::STG_OFF + (2u * ((uint32_t)kr >> 6) + (qr >> 1)) * 8192u + r * 128;
 #pragma unroll
       for (int k = 0; k < 4; ++k)
         *reinterpret_cast<uint4*>(box + (((4 * (int)(qr & 1u) + k) ^ (r & 7)) << 4)) =
             make_uint4(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
       fence_proxy_async();
       __syncwarp();
-      if (lane == 0) mbar_arrive(bar(C_::STGFULL + (g & 1u)));
+      if (lane == 0) mbar_arrive(bar(C_::STGFULL));
       return true;
     };
     // B: dS^T = P^T * (dP^T - D[q]) of tile g, from the bf16 P^T that the products use
