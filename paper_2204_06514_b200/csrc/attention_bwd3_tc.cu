@@ -27,7 +27,7 @@
 // tiles later).  Staging in the Q stage instead delayed the next Q tile and with it S^T.
 // Per-query statistics (log2e * LSE, D) travel with the Q stage they belong to.  The MMA thread
 // builds every shared-memory descriptor from precomputed words with one addition.  Every wait is bounded.
-#include "attention_common.cuh"
+#include "tc_common.cuh"
 
 namespace {
 
@@ -332,7 +332,7 @@ attn_bwd3_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_c
             float p0 = ex2_approx(__uint_as_float(sv[e]) * p.scale_log2 - l4.x);
             float p1 = ex2_approx(__uint_as_float(sv[e + 1]) * p.scale_log2 - l4.y);
             float p2 = ex2_approx(__uint_as_float(sv[e + 2]) * p.scale_log2 - l4.z);
-            float p3 = ex2_poly(__uint_as_float(sv[e + 3]) * p.scale_log2 - l4.w);     // one in four off the special-function unit
+            float p3 = ex2_approx(__uint_as_float(sv[e + 3]) * p.scale_log2 - l4.w);
             if (it == 0) {                   // diagonal tile: a query before the key is masked
               const int q0 = 32 * (int)qr + e;
               if (q0 < kr) p0 = 0.f;

@@ -25,7 +25,7 @@
 // Shared memory: two (K, V) buffers, three Q stages (a Q tile lives from S^T, two iterations ahead, to
 // dK), two dO stages, the dS tile (B operand of dQ), a 32 KB dQ staging buffer, per-stage query
 // statistics.  Every wait is bounded.
-#include "attention_common.cuh"
+#include "tc_common.cuh"
 
 namespace {
 
@@ -314,7 +314,7 @@ attn_bwd4_tc_kernel(const __grid_constant__ CUtensorMap tmap_qkv, const __grid_c
         float p0 = ex2_approx(__uint_as_float(sv[e]) * p.scale_log2 - l4.x);
         float p1 = ex2_approx(__uint_as_float(sv[e + 1]) * p.scale_log2 - l4.y);
         float p2 = ex2_approx(__uint_as_float(sv[e + 2]) * p.scale_log2 - l4.z);
-        float p3 = ex2_poly(__uint_as_float(sv[e + 3]) * p.scale_log2 - l4.w);     // one in four off the special-function unit
+        float p3 = ex2_approx(__uint_as_float(sv[e + 3]) * p.scale_log2 - l4.w);
         if (diag) {
           const int q0 = 32 * (int)qr + e;
           if (q0 < kr) p0 = 0.f;

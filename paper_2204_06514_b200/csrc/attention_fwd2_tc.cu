@@ -17,7 +17,7 @@
 // without waiting for a product.  With that the exponentials (1024 clocks of the special-function
 // units per 128 x 128 tile, more than the tile's 876 tensor-core clocks at head_dim 64) are the bound;
 // before, each group's loop was softmax + both products + the hand-offs, about 2900 clocks per tile.
-#include "attention_common.cuh"
+#include "tc_common.cuh"
 
 namespace {
 
@@ -308,10 +308,8 @@ attn_fwd2_tc_kernel(const __grid_constant__ CUtensorMap tmap, const AttnFwd2Para
           for (int cc = 0; cc < 2; ++cc)
 #pragma unroll
             for (int e = 0; e < 32; e += 2) {
-              // one exponential in four on the FMA pipe: the special-function unit is the busiest unit of the tile
               const float p0 = ex2_approx(__uint_as_float(sv[2 * half + cc][e]) * p.scale_log2 - m_used);
-              const float x1 = __uint_as_float(sv[2 * half + cc][e + 1]) * p.scale_log2 - m_used;
-              const float p1 = (e & 2) ? ex2_poly(x1) : ex2_approx(x1);
+              const float p1 = ex2_approx(__uint_as_float(sv[2 * half + cc][e + 1]) * p.scale_log2 - m_used);
               rowsum += p0 + p1;
               __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
               packed[16 * cc + (e >> 1)] = *reinterpret_cast<uint32_t*>(&h2);
