@@ -34,10 +34,12 @@ constexpr int STAGES = 6;
 constexpr int TMEM_COLS = 512;
 constexpr int STAGING_BYTES = NUM_EPI_WARPS * EPI_STAGING_BYTES;
 constexpr int BAR_BYTES = 256;
-// Only the float-output instantiation stages partial tiles; the others leave that shared memory to L1,
-// which the epilogue's residual / pre-activation loads go through.
-constexpr int smem_bytes(int epi) { return STAGES * STAGE_BYTES + (epi == EPI_STATIC_F32 ? STAGING_BYTES : 0) + 1024 + BAR_BYTES; }
-static_assert(smem_bytes(EPI_STATIC_F32) <= 227 * 1024, "shared memory per CTA");
+// Only a K-sliced float output stages partial tiles; every other launch leaves that shared memory to L1 (which
+// the epilogue's residual / pre-activation loads go through) and to the blocks of the kernels that run beside
+// or right behind this one (the AdamW stream, the next kernel's blocks under programmatic dependent launch:
+// with the staging in every float-output launch a block step of hidden 5120 took 4.9 instead of 4.5 ms).
+constexpr int smem_bytes(bool staged) { return STAGES * STAGE_BYTES + (staged ? STAGING_BYTES : 0) + 1024 + BAR_BYTES; }
+static_assert(smem_bytes(true) <= 227 * 1024, "shared memory per CTA");
 static_assert(8 * (2 * STAGES + 4) + 8 <= BAR_BYTES, "barrier area");
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
@@ -89,9 +91,9 @@ gemm_tcgen05_2cta_kernel(const __grid_constant__ CUtensorMap tmap_a, const __gri
   const uint32_t tiles_base = (raw + 1023u) & ~1023u;
   uint8_t* gen_base = smem_raw + (tiles_base - raw);
   const uint32_t staging = tiles_base + STAGES * STAGE_BYTES;
-  constexpr int STG = EPI == EPI_STATIC_F32 ? STAGING_BYTES : 0;
-  uint8_t* bar_mem = gen_base + STAGES * STAGE_BYTES + STG;
-  const uint32_t bars = staging + STG;
+  const int stg_bytes = (EPI == EPI_STATIC_F32 && p.splits > 1) ? STAGING_BYTES : 0;      // as the launcher sized it
+  uint8_t* bar_mem = gen_base + STAGES * STAGE_BYTES + stg_bytes;
+  const uint32_t bars = staging + (uint32_t)stg_bytes;
   auto full_bar = [&](int s) { return bars + 8u * s; };                         // used in the even CTA
   auto empty_bar = [&](int s) { return bars + 8u * (STAGES + s); };             // one per CTA
   auto tfull_bar = [&](int a) { return bars + 8u * (2 * STAGES + a); };         // one per CTA
@@ -268,7 +270,7 @@ fax_status fax_gemm_tc2(fax_ctx* ctx, const FaxGemm& g) {
   fill_gemm_params(p, g, ctx->dev_status);
   {
     static bool attr_set[7][FAX_MAX_DEVICES] = {};
-#define FAX_SET_SMEM(I, E) FAX_TRY(fax_opt_in_shared_memory(ctx, gemm_tcgen05_2cta_kernel<E>, smem_bytes(E), attr_set[I]))
+#define FAX_SET_SMEM(I, E) FAX_TRY(fax_opt_in_shared_memory(ctx, gemm_tcgen05_2cta_kernel<E>, smem_bytes(E == EPI_STATIC_F32), attr_set[I]))
     FAX_SET_SMEM(0, -1); FAX_SET_SMEM(1, 0); FAX_SET_SMEM(2, 1); FAX_SET_SMEM(3, 2); FAX_SET_SMEM(4, 3); FAX_SET_SMEM(5, 4);
     FAX_SET_SMEM(6, EPI_STATIC_F32);
 #undef FAX_SET_SMEM
@@ -282,9 +284,9 @@ fax_status fax_gemm_tc2(fax_ctx* ctx, const FaxGemm& g) {
   const int items = tiles * p.splits;
   const int pairs = items < max_pairs ? items : max_pairs;
   switch (gemm_static_epi(g)) {
-#define FAX_LAUNCH(E) case E: fax_launch(ctx, gemm_tcgen05_2cta_kernel<E>, dim3(2 * pairs), dim3(NUM_THREADS), smem_bytes(E), ma, mb, p, mc); break
+#define FAX_LAUNCH(E) case E: fax_launch(ctx, gemm_tcgen05_2cta_kernel<E>, dim3(2 * pairs), dim3(NUM_THREADS), smem_bytes(E == EPI_STATIC_F32 && p.splits > 1), ma, mb, p, mc); break
     FAX_LAUNCH(0); FAX_LAUNCH(1); FAX_LAUNCH(2); FAX_LAUNCH(3); FAX_LAUNCH(4); FAX_LAUNCH(EPI_STATIC_F32);
-    default: fax_launch(ctx, gemm_tcgen05_2cta_kernel<-1>, dim3(2 * pairs), dim3(NUM_THREADS), smem_bytes(-1), ma, mb, p, mc); break;
+    default: fax_launch(ctx, gemm_tcgen05_2cta_kernel<-1>, dim3(2 * pairs), dim3(NUM_THREADS), smem_bytes(false), ma, mb, p, mc); break;
 #undef FAX_LAUNCH
   }
   return fax_after_launch(ctx);

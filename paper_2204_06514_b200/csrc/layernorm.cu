@@ -678,7 +678,11 @@ constexpr int kColsumBlocksPerSm = 8, kLnColBlocksPerSm = 5;
 // The fused backward covers rows of up to 2048 vectors (up to 512: row groups inside a block, above: one
 // row per block at a time); one slab per block, one block per SM.  The bias-gradient sums ride along up
 // to 1024 vectors (wider rows have no registers left for four sums per column).
-bool ln_bwd_is_fused(int nvec) { return nvec <= 2048; }
+// The one-row-per-block kernel takes every register of an SM, so it cannot be placed beside the persistent
+// AdamW blocks of the optimizer stream and waits for a whole AdamW launch to finish (measured: +1.7 % on the
+// step at hidden 5120 and 8192 with the overlap on): while that stream is busy the wide rows take the
+// block-per-row dx kernel and a column reduction, whose small blocks fit beside the optimizer's.
+bool ln_bwd_is_fused(const fax_ctx* ctx, int nvec) { return nvec <= 512 || (nvec <= 2048 && !ctx->side_busy); }
 bool ln_bwd_fuses_sums(int nvec) { return nvec <= 1024; }
 int ln_row_groups(int nvec) { return nvec <= 64 ? 16 : nvec <= 128 ? 8 : nvec <= 256 ? 4 : 2; }
 int ln_bwd_fused_grid(fax_ctx* ctx, int rows, int nvec) {
@@ -690,7 +694,7 @@ int ln_bwd_fused_grid(fax_ctx* ctx, int rows, int nvec) {
 }
 int ln_bwd_slabs(fax_ctx* ctx, int rows, int d, int prec) {
   const int nvec = d / (prec == FAX_PREC_BF16 ? 8 : 4);
-  return ln_bwd_is_fused(nvec) ? ln_bwd_fused_grid(ctx, rows, nvec) : colreduce_slabs(ctx, rows, nvec, kLnColBlocksPerSm);
+  return ln_bwd_is_fused(ctx, nvec) ? ln_bwd_fused_grid(ctx, rows, nvec) : colreduce_slabs(ctx, rows, nvec, kLnColBlocksPerSm);
 }
 
 template <typename T>
@@ -845,7 +849,7 @@ fax_status fax_layernorm_bwd(fax_ctx* ctx, int prec, int rows, int d, const void
   if (d % (prec == FAX_PREC_BF16 ? 8 : 4)) return FAX_ERR_UNSUPPORTED_SHAPE;
   const bool sums = sum_add && sum_out && add;
   const int nvec_all = d / (prec == FAX_PREC_BF16 ? 8 : 4);
-  const bool fused = ln_bwd_is_fused(nvec_all);
+  const bool fused = ln_bwd_is_fused(ctx, nvec_all);
   const bool fused_sums = fused && ln_bwd_fuses_sums(nvec_all);
   if (partial_floats < (size_t)(sums && fused_sums ? 4 : 2) * ln_bwd_slabs(ctx, rows, d, prec) * d) return FAX_ERR_WORKSPACE_TOO_SMALL;
   if (sums && !fused_sums) {
@@ -857,7 +861,7 @@ fax_status fax_layernorm_bwd(fax_ctx* ctx, int prec, int rows, int d, const void
   }
   // dx pass reads da, x (and add) and writes dx; the dgamma/dbeta pass reads da and x again
   FaxProfScope prof(ctx, KC_LN_BWD, 0.0, (double)rows * d * fax_elem_size(prec) * (add ? 4 : 3));
-  if (ln_bwd_is_fused(d / (prec == FAX_PREC_BF16 ? 8 : 4))) {
+  if (fused) {
     if (prec == FAX_PREC_BF16)
       return ln_bwd_fused_t<bf16>(ctx, rows, d, da, x, mu, rstd, gamma, add, dx, dgamma, dbeta, accumulate, partial,
                                   sum_add, sum_out);
