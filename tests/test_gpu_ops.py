@@ -178,7 +178,9 @@ def test_gemm_epilogues(sess, prec, force_simt):
     assert relerr(run(ops.FAX_EPI_NONE, c_f32=1, accumulate=1, C0=C0), acc + C0) <= (1e-5 if prec == 1 else tol)
 
 
-@pytest.mark.parametrize("M,N,K", [(128, 256, 4096), (768, 768, 16384), (256, 128, 1088)])
+# (768, 2304, 16384): 27 tiles on 74 SM pairs, five slices; (2560, 2560, 4096): 100 tiles, sliced to fill the second wave
+@pytest.mark.parametrize("M,N,K", [(128, 256, 4096), (768, 768, 16384), (256, 128, 1088), (768, 2304, 16384),
+                                   (2560, 2560, 4096)])
 @pytest.mark.parametrize("accumulate", [0, 1])
 def test_gemm_weight_gradient_shapes_split_k(sess, M, N, K, accumulate):
     """Few output tiles, long K: the kernel slices K and adds partial tiles into the float output."""
