@@ -358,7 +358,8 @@ def test_attention_forward_backward(sess, prec, B, T, H, hd):
     assert st == fx.FAX_OK
 
 
-@pytest.mark.parametrize("B,T,H,hd", [(2, 640, 5, 128), (2, 640, 6, 64), (1, 1152, 3, 64)])
+@pytest.mark.parametrize("B,T,H,hd", [(2, 640, 5, 128), (2, 640, 6, 64), (1, 1152, 3, 64), (1, 128, 1, 64), (3, 256, 2, 64),
+                                      (5, 2048, 31, 64)])
 def test_attention_backward_kernels_agree(sess, B, T, H, hd):
     """The three backward kernels (mode 2: two score tiles in flight at head_dim 64; mode 1: sixteen row
     warps with half-tile hand-offs; mode 0: the single hand-off kernel): the same inputs through each,
